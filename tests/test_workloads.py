@@ -1,0 +1,76 @@
+"""Seeded input generator and the closed-form byte counts (no GPU)."""
+import numpy as np
+import torch
+
+from paper_2512_20687_b200 import workloads as wl
+
+
+def test_streams_are_deterministic_and_sliceable():
+    a = wl.normal_bf16(3, "t", (1000,))
+    b = wl.normal_bf16(3, "t", (1000,))
+    assert np.array_equal(a, b)
+    assert np.array_equal(wl.normal_bf16(3, "t", (100,), offset=250), a[250:350])
+    assert not np.array_equal(a, wl.normal_bf16(4, "t", (1000,)))
+    assert not np.array_equal(a, wl.normal_bf16(3, "u", (1000,)))
+    big = wl.normal_bf16(5, "big", (3, 1 << 22))          # crosses the threaded block size
+    assert np.array_equal(big.reshape(-1)[(1 << 22) - 5:(1 << 22) + 5],
+                          wl.normal_bf16(5, "big", (10,), offset=(1 << 22) - 5))
+
+
+def test_distribution_and_bf16_rounding():
+    x = wl.bf16_bits_to_f64(wl.normal_bf16(0, "m", (1 << 20,)))
+    assert abs(x.mean()) < 5e-3 and abs(x.std() - 1.0) < 5e-3 and np.isfinite(x).all()
+    w = wl.bf16_bits_to_f64(wl.normal_bf16(0, "w", (1 << 18,), std=256 ** -0.5))
+    assert abs(w.var() * 256 - 1.0) < 2e-2
+    r = np.random.default_rng(0).standard_normal(50000).astype(np.float32)
+    t = torch.from_numpy(r).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(wl.f32_to_bf16_bits(r), t)
+    assert np.array_equal(wl.bf16_bits_to_f64(t), torch.from_numpy(r).to(torch.bfloat16).double().numpy())
+
+
+def test_config_table_matches_the_hierarchy():
+    """Cached coarse length is T / C_{<=L} (Section 2.3.3, inference cost)."""
+    for c in wl.CONFIGS:
+        assert c.S == c.context // c.compress and c.D == c.Hq * c.dh and c.Hq % c.Hkv == 0
+        if c.shared_S:
+            assert c.shared_S == c.shared_context // c.compress
+    assert [c.S for c in wl.CONFIGS] == [16, 512, 8192, 32, 128]
+    assert [c.Nc for c in wl.CONFIGS] == [16, 128, 32, 512, 16384]
+
+
+def test_kv_bytes_closed_forms():
+    """Per step the coarse cache is C_{<=L} times smaller than a token-level
+    cache; a coarse step happens once per C_{<=L} tokens, so per generated
+    token the ratio is C_{<=L}^2 (takeaway table of Section 2.3.3)."""
+    mib = 1 << 20
+    assert [wl.coarse_kv_bytes(c) // 1024 for c in wl.CONFIGS[:1]] == [16]
+    assert [wl.coarse_kv_bytes(c) / mib for c in wl.CONFIGS[1:]] == [64, 256, 20, 256]
+    assert [wl.flat_kv_bytes(c) / mib for c in wl.CONFIGS[1:]] == [1024, 4096, 320, 4096]
+    for c in wl.CONFIGS:
+        assert wl.flat_kv_bytes(c) == c.compress * wl.coarse_kv_bytes(c)
+        per_token_coarse = wl.coarse_kv_bytes(c) / c.compress
+        assert wl.flat_kv_bytes(c) / per_token_coarse == c.compress ** 2 == 256
+
+
+def test_chunk_inputs_structure():
+    cfg = wl.CONFIGS[0]
+    ch = wl.chunk_inputs(cfg, poison=True)
+    assert ch["kc"].shape == (16, 2, 8, 64) and ch["len"].min() >= cfg.P + 1 and ch["len"].max() <= 8
+    for c in range(cfg.Nc):
+        assert np.all(ch["kc"][c, :, ch["len"][c]:] == 0x7FC1)
+        assert not np.any(ch["kc"][c, :, : ch["len"][c]] == 0x7FC1)
+    strict = wl.chunk_inputs(cfg, strict_paper=True)
+    assert np.array_equal(strict["len"], ch["len"] - 1) and strict["len"].min() >= cfg.P
+    big = wl.chunk_inputs(wl.scaled(wl.CONFIGS[4], B=8))
+    assert set(np.unique(big["n_in"])) == set(range(1, 17))
+    assert wl.chunk_kv_bytes(cfg, ch["len"]) == int(ch["len"].sum()) * 2 * 64 * 4
+
+
+def test_shard_units_partitions_exactly():
+    for n in (0, 1, 7, 64, 16384):
+        for ws in (1, 2, 3, 8):
+            parts = [wl.shard_units(n, ws, r) for r in range(ws)]
+            assert parts[0][0] == 0 and parts[-1][1] == n
+            assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
+            sizes = [b - a for a, b in parts]
+            assert max(sizes) - min(sizes) <= 1
