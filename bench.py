@@ -1,0 +1,463 @@
+#!/usr/bin/env python
+"""Benchmark of the PHOTON decode step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
+
+A step is one pass of the whole hot path (append -> coarse attention ->
+converter -> chunk attention) over one batch of seeded synthetic input.  The
+metric is decode tokens/s = token-level in-flight chunks per step / step time.
+With N > 1 (launched by torchrun) every rank runs an independent replica of
+the same per-GPU batch (weak scaling, no data-path collective); time is the
+max over ranks.  Rank 0 prints ONE JSON line.
+
+`--impl reference` times the CPU oracle (a deliberately plain fp64 program)
+on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2512_20687_b200 import workloads as wl  # noqa: E402
+
+METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
+L2_BYTES = 126 * 1000 * 1000
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--config", type=int, default=1, help="index into the five workload configurations")
+    ap.add_argument("--impl", default="photon", choices=["photon", "reference"])
+    ap.add_argument("--layout", default="out_major", choices=["out_major", "in_major"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parts", action="store_true")
+    ap.add_argument("--max-splits", type=int, default=0)
+    return ap.parse_args()
+
+
+def workload_desc(cfg) -> dict:
+    d = {"workload": f"config {cfg.index} ({cfg.name}): batch {cfg.B}, context {cfg.context} tokens -> "
+                     f"{cfg.S} coarse latents, {cfg.Hq}q/{cfg.Hkv}kv heads x {cfg.dh}, d_model {cfg.D}, "
+                     f"converter {cfg.D}->{cfg.P}x{cfg.D}, chunk attention P={cfg.P} C={cfg.C}, "
+                     f"{cfg.chunks_per_seq} in-flight chunks per sequence",
+         "batch": cfg.B, "coarse_len": cfg.S, "context": cfg.context, "seed": cfg.seed,
+         "tokens_per_step": cfg.tokens_per_step}
+    if cfg.shared_S:
+        d["shared_prefix_len"] = cfg.shared_S
+    return d
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_sample(cfg, seconds: float, threads: int):
+    """The first b sequences (and their chunks) of the workload, b sized so that
+    one oracle step costs about `seconds` of wall time on `threads` cores."""
+    flops = (cfg.B * cfg.Hq * (cfg.S + cfg.shared_S) * cfg.dh * 4 + 2.0 * cfg.B * cfg.D * cfg.P * cfg.D
+             + cfg.Nc * cfg.Hq * (cfg.P + cfg.C) * cfg.dh * 4)
+    rate = 0.25e9 * max(1, threads)                      # plain fp64 loops: ~0.25 Gflop/s per core
+    b = int(max(1, min(cfg.B, cfg.B * seconds * rate / flops)))
+    sub = wl.scaled(cfg, B=b)
+    s = wl.step_inputs(sub)
+    return sub, s
+
+
+def time_oracle_step(cfg, sample_cfg, s, threads: int) -> float:
+    from oracle import photon_oracle as oracle
+    co = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in s["coarse"].items()}
+    scale = cfg.dh ** -0.5
+    t0 = time.perf_counter()
+    oracle.decode_step(co, s["converter"], s["chunks"], scale, scale, chain=True, w_out_major=True,
+                       n_threads=threads)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, seconds: float = 10.0) -> dict:
+    from oracle import photon_oracle as oracle
+    threads = oracle.hardware_threads() or os.cpu_count() or 1
+    sub, s = oracle_sample(cfg, seconds, threads)
+    dt = time_oracle_step(cfg, sub, s, threads)
+    tokens = cfg.tokens_per_step * sub.B / cfg.B
+    return {"value": tokens / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"one full decode step of the first {sub.B} of {cfg.B} sequences "
+                      f"({sub.Nc} chunks), {dt:.2f} s"}
+
+
+def run_reference(args, cfg) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import photon_oracle as oracle
+    oracle.build()
+    threads = oracle.hardware_threads() or os.cpu_count() or 1
+    per_step = max(0.05, min(10.0, 150.0 / max(1, args.steps + args.warmup)))
+    sub, s = oracle_sample(cfg, per_step, threads)
+    for _ in range(args.warmup):
+        time_oracle_step(cfg, sub, s, threads)
+    times = [time_oracle_step(cfg, sub, s, threads) for _ in range(args.steps)]
+    dt = sum(times) / len(times)
+    tokens = cfg.tokens_per_step * sub.B / cfg.B
+    val = tokens / dt
+    sample = (f"each step = one oracle decode step of the first {sub.B} of {cfg.B} sequences "
+              f"({sub.Nc} chunks)")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 * cfg.B / sub.B,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_desc(cfg),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid, self.proc, self.f = uuid, None, None
+
+    def start(self):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.f.flush()
+        self.f.seek(0)
+        rows = [r.strip().split(", ") for r in self.f.read().splitlines() if r.strip()]
+        self.f.close()
+        os.unlink(self.f.name)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def run_gpu(args, cfg) -> None:
+    import torch
+
+    import paper_2512_20687_b200 as ph
+    from paper_2512_20687_b200 import dist as pd
+
+    rank, local_rank, world = pd.init()
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    ph.load()
+
+    out_major = args.layout == "out_major"
+    layout = ph.PHOTON_W_OUT_MAJOR if out_major else ph.PHOTON_W_IN_MAJOR
+    scale = cfg.dh ** -0.5
+    s = wl.step_inputs(cfg)
+    co, cv, ch = s["coarse"], s["converter"], s["chunks"]
+
+    def dev_bf16(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    coarse_bytes = wl.coarse_kv_bytes(cfg)
+    chunk_bytes = wl.chunk_kv_bytes(cfg, ch["len"])
+    w_bytes = cv["w_in_major"].nbytes
+    per_replica = co["k"].nbytes * 2 + ch["kc"].nbytes * 2 + w_bytes
+    R = max(4, -(-3 * L2_BYTES // per_replica))
+    base = {"k": dev_bf16(co["k"]), "v": dev_bf16(co["v"]), "kc": dev_bf16(ch["kc"]),
+            "vc": dev_bf16(ch["vc"]), "w": dev_bf16(cv["w_out_major"] if out_major else cv["w_in_major"])}
+    k_new, v_new, q = dev_bf16(co["k_new"]), dev_bf16(co["v_new"]), dev_bf16(co["q"])
+    qc = dev_bf16(ch["q"])
+    lens0 = torch.from_numpy(np.tile(co["len"], (R, 1))).to(dev)
+    lens = lens0.clone()
+    clen = torch.from_numpy(ch["len"]).to(dev)
+    shared = {}
+    if cfg.shared_S:
+        shared = dict(k_shared=dev_bf16(co["k_shared"]), v_shared=dev_bf16(co["v_shared"]),
+                      shared_len=torch.from_numpy(co["shared_len"]).to(dev),
+                      shared_id=torch.from_numpy(co["shared_id"]).to(dev))
+    ctx = ph.photon_create(cfg.Hq, cfg.Hkv, cfg.dh, cfg.D, cfg.P, cfg.C, max(cfg.B, cfg.Nc),
+                           args.max_splits)
+    reps = []
+    for r in range(R):
+        t = {n: (b if r == 0 else b.clone()) for n, b in base.items()}
+        t["out"] = torch.empty_like(q)
+        t["U"] = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device=dev)
+        t["oc"] = torch.empty_like(qc)
+        t["kv"] = ph.make_kv(t["k"], t["v"], lens[r], max_len=cfg.S, **shared)
+        t["ckv"] = ph.make_kv(t["kc"], t["vc"], clen)
+        t["args"] = ph.make_step_args(t["kv"], k_new, v_new, q, t["out"], scale, t["w"], layout, t["U"],
+                                      cfg.B, chunks=t["ckv"], q_chunk=qc, out_chunk=t["oc"], Nc=cfg.Nc,
+                                      scale_chunk=scale)
+        reps.append(t)
+    torch.cuda.synchronize()
+
+    def step(i, a=None):
+        r = i % R
+        ph.photon_decode_step(ctx, a if a is not None else reps[r]["args"])
+        if r == R - 1:
+            lens.copy_(lens0)                     # undo the appends of one ring cycle
+
+    K, W = args.steps, args.warmup
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    n0 = ph.photon_launch_count(ctx)
+    step(0)
+    launches_per_step = ph.photon_launch_count(ctx) - n0
+    for i in range(1, R):
+        step(i)
+    torch.cuda.synchronize()
+    assert ph.photon_device_status(ctx) == 0, "device status word set during warm-up"
+
+    # CUDA graphs of one ring cycle each (R steps + the length reset); K steps = full cycles + a tail
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+
+    def capture(n_steps):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_steps):
+                    step(i)
+                if n_steps % R:
+                    lens.copy_(lens0)
+        return g
+
+    cycles_per_graph = max(1, 32 // R)
+    G = R * cycles_per_graph
+    g_full = capture(G) if K >= G else None
+    g_tail = capture(K % G) if K % G else None
+    n_full = K // G
+
+    def replay():
+        for _ in range(n_full):
+            g_full.replay()
+        if g_tail is not None:
+            g_tail.replay()
+
+    replay() if K <= 4096 else (g_full.replay() if g_full else g_tail.replay())     # untimed graph warm-up
+    torch.cuda.synchronize()
+
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pd.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record()
+    replay()
+    e1.record()
+    torch.cuda.synchronize()
+    pd.barrier()
+    sec = e0.elapsed_time(e1) * 1e-3
+    clocks = sampler.stop()
+    if clocks["samples"] < 3:                     # region too short to sample: repeat it untimed under the sampler
+        sampler = ClockSampler(sampler.uuid)
+        sampler.start()
+        t_end = time.time() + 1.0
+        while time.time() < t_end:
+            replay()
+            torch.cuda.synchronize()
+        clocks = sampler.stop()
+        clocks["note"] = "timed region shorter than the sampling period; sampled on an untimed repeat of it"
+    assert ph.photon_device_status(ctx) == 0, "device status word set during the timed region"
+    sec_max = pd.reduce_max(sec)
+    tokens_total = pd.reduce_sum(cfg.tokens_per_step * K)
+    value = tokens_total / sec_max
+
+    # dominant kernel in place: eager steps with events around the coarse attention launches
+    n_ev = min(K, 256)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+    for a, b in evs:
+        a.record(); b.record()                    # creates the underlying CUDA events
+    torch.cuda.synchronize()
+    ev_args = []
+    for i in range(n_ev):
+        t = reps[i % R]
+        ev_args.append(ph.make_step_args(t["kv"], k_new, v_new, q, t["out"], scale, t["w"], layout,
+                                         t["U"], cfg.B, chunks=t["ckv"], q_chunk=qc, out_chunk=t["oc"],
+                                         Nc=cfg.Nc, scale_chunk=scale, ev_attn_begin=evs[i][0],
+                                         ev_attn_end=evs[i][1]))
+    lens.copy_(lens0)
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ee0.record()
+    for i in range(n_ev):
+        step(i, ev_args[i])
+    ee1.record()
+    torch.cuda.synchronize()
+    lens.copy_(lens0)
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+    eager_ms_per_step = ee0.elapsed_time(ee1) / n_ev
+
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    qo_bytes = 2 * cfg.B * cfg.Hq * cfg.dh * 2
+    attn_alg_bytes = coarse_bytes + qo_bytes
+    traffic = None
+    try:
+        traffic = json.load(open(os.path.join(ROOT, "profiles", "roofline_traffic.json"))).get(
+            f"config{cfg.index}", {}).get("coarse_attn_dram_bytes_per_launch")
+    except OSError:
+        pass
+    achieved = attn_alg_bytes / (attn_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "coarse attention (split-K partial + merge launches)",
+                "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                "traffic": traffic, "algorithmic_bytes": attn_alg_bytes, "us_per_launch": attn_ms * 1e3,
+                "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback 6650 GB/s",
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # per-part times (eager, events around a batch of calls rotating over the replicas)
+    parts = {}
+    if not args.no_parts:
+        def time_part(fn, n=64):
+            for i in range(8):
+                fn(reps[i % R])
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for i in range(n):
+                fn(reps[i % R])
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / n
+        parts["coarse_attn_us"] = time_part(lambda t: ph.photon_coarse_attn(ctx, t["kv"], q, t["out"], None, scale))
+        parts["converter_us"] = time_part(lambda t: ph.photon_converter(ctx, t["out"].view(cfg.B, -1), t["w"], layout, None, t["U"]))
+        parts["chunk_attn_us"] = time_part(lambda t: ph.photon_chunk_attn(ctx, t["ckv"], qc, None, t["oc"], scale=scale))
+
+        def app(t):
+            ph.photon_kv_append(ctx, t["kv"], k_new, v_new)
+        lens.copy_(lens0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for i in range(R):
+            app(reps[i])
+        b.record()
+        torch.cuda.synchronize()
+        lens.copy_(lens0)
+        parts["kv_append_us"] = a.elapsed_time(b) * 1e3 / R
+        parts["note"] = "eager back-to-back calls; launch-rate bound below ~3 us"
+        parts["converter_gbs_weights"] = w_bytes / (parts["converter_us"] * 1e-6) / 1e9
+        parts["converter_tflops"] = 2.0 * cfg.B * cfg.D * cfg.P * cfg.D / (parts["converter_us"] * 1e-6) / 1e12
+        parts["chunk_attn_gbs"] = (chunk_bytes + 2 * cfg.Nc * cfg.Hq * cfg.dh * 2) / (parts["chunk_attn_us"] * 1e-6) / 1e9
+        parts["coarse_attn_gbs"] = attn_alg_bytes / (parts["coarse_attn_us"] * 1e-6) / 1e9
+
+    # end to end through the public API with host buffers: H2D of the step's inputs, D2H of its results
+    pin = lambda t: t.cpu().pin_memory()
+    h_in = [pin(k_new), pin(v_new), pin(q), pin(qc), pin(lens0[0])]
+    d_in = [k_new, v_new, q, qc]
+    h_out_c, h_out_t = pin(reps[0]["out"]), pin(reps[0]["oc"])
+    h2d = sum(t.numel() * t.element_size() for t in h_in)
+    d2h = h_out_c.numel() * 2 + h_out_t.numel() * 2
+    n_e2e = max(3, min(K, 2000))
+
+    def e2e_step(i):
+        r = i % R
+        for h, d in zip(h_in[:4], d_in):
+            d.copy_(h, non_blocking=True)
+        lens[r].copy_(h_in[4], non_blocking=True)
+        ph.photon_decode_step(ctx, reps[r]["args"])
+        h_out_c.copy_(reps[r]["out"], non_blocking=True)
+        h_out_t.copy_(reps[r]["oc"], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    pd.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_sec = pd.reduce_max(time.perf_counter() - t0)
+    e2e_val = pd.reduce_sum(cfg.tokens_per_step * n_e2e) / e2e_sec
+    lens.copy_(lens0)
+    torch.cuda.synchronize()
+    bits = ph.photon_device_status(ctx)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": sec_max * 1e3 / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(workload_desc(cfg),
+                       l2="inputs larger than L2: KV caches, chunk buffers and converter weight rotate over "
+                          f"{R} replicas ({R * per_replica / 2**20:.0f} MiB vs 126 MB L2)",
+                       launch="CUDA graph of %d steps replayed; per-rank batch fixed" % G,
+                       w_layout=args.layout),
+        "clocks": clocks,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": n_e2e, "note": "pinned host buffers -> device, decode step, results -> host, every step"},
+        "gpu_launches": launches_per_step * K,
+        "roofline": roofline,
+        "us_per_step": sec_max * 1e6 / K,
+        "eager_us_per_step": eager_ms_per_step * 1e3,
+        "parts": parts,
+        "kv_bytes_per_token": {
+            "photon_coarse_per_step": coarse_bytes,
+            "photon_per_token": coarse_bytes / cfg.compress / cfg.B + (chunk_bytes / cfg.Nc),
+            "flat_per_token": wl.flat_kv_bytes(cfg) / cfg.B,
+            "note": "per sequence and layer; coarse step amortised over %d tokens" % cfg.compress},
+        "device_status": bits,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(cfg)
+    ph.photon_destroy(ctx)
+    pd.barrier()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    pd.shutdown()
+
+
+def main():
+    args = parse()
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_gpu(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,194 @@
+/* photon.h - C boundary of the PHOTON decode-step library (sm_100a).
+ *
+ * One recursive-generation step of PHOTON (Section 2.3.3): the coarsest
+ * stream appends one latent to its KV cache and attends over it (the
+ * attention and cache halves of STEP, Eq. 12 / Eq. 13), the context converter
+ * expands the resulting latent into P prefix vectors (Section 2.1.2), and the
+ * local decoders run bounded causal attention over P prefix rows plus at most
+ * C in-chunk rows, independently for every in-flight chunk (Eq. 6-7).
+ *
+ * Conventions that hold for every call
+ *  - All tensor pointers are DEVICE pointers owned by the caller, 16-byte
+ *    aligned, bf16 stored as raw uint16 bits, C order.  The library owns only
+ *    the photon_ctx (split-K workspace and a 4-byte device status word).
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and
+ *    return at once; nothing synchronises except photon_device_status.
+ *  - The return value reports host-side problems only (bad arguments, a
+ *    failed launch).  Nothing is launched when it is not PHOTON_OK.
+ *  - Device-side anomalies never trap.  They set bits in the status word:
+ *    an append without room writes nothing (PHOTON_DEV_CAPACITY); an
+ *    out-of-range unit id, slot or shared id skips that item and zero-fills
+ *    its output row (PHOTON_DEV_BAD_INDEX); a bounded wait that ran out
+ *    (PHOTON_DEV_TIMEOUT) leaves the affected outputs undefined.
+ *  - q and k arrive already position-encoded; the library applies no rotary
+ *    or other positional transform.
+ *  - There is no CPU fallback: without a CUDA device photon_create fails.
+ */
+#ifndef PHOTON_H
+#define PHOTON_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t photon_bf16;            /* raw bf16 bits */
+typedef struct photon_ctx photon_ctx;
+typedef void *photon_stream;             /* cudaStream_t */
+typedef void *photon_event;              /* cudaEvent_t  */
+
+typedef enum {
+  PHOTON_OK = 0,
+  PHOTON_ERR_INVALID_ARG = 1,            /* NULL / misaligned pointer, size out of range */
+  PHOTON_ERR_UNSUPPORTED = 2,            /* shape the kernels are not built for */
+  PHOTON_ERR_CUDA = 3,                   /* a CUDA runtime call or launch failed */
+  PHOTON_ERR_WORKSPACE = 4               /* call needs more workspace than the ctx was created with */
+} photon_status;
+
+enum {                                   /* device status bits */
+  PHOTON_DEV_CAPACITY = 1,
+  PHOTON_DEV_BAD_INDEX = 2,
+  PHOTON_DEV_TIMEOUT = 4
+};
+
+enum {                                   /* storage order of the converter weight */
+  PHOTON_W_IN_MAJOR = 0,                 /* W[k][n]: [D, P*D], row k = input feature   */
+  PHOTON_W_OUT_MAJOR = 1                 /* W[n][k]: [P*D, D], row n = output column (the order of a
+                                            kernel-size-1 convolution weight)          */
+};
+
+/* Model shape, fixed per context.  Hq query heads share Hkv KV heads in
+ * contiguous groups (query head h reads KV head h / (Hq/Hkv)).  dh must be 64
+ * or 128, Hq/Hkv at most 16, D = d_model a multiple of 64, P + C at most 64.
+ * max_queries: largest number of queries (sequences, branches or chunks) any
+ * single attention call will carry; max_splits: upper bound on the number of
+ * key ranges one query's keys are split into (0 = library default).  Both
+ * only size the workspace. */
+typedef struct {
+  int32_t Hq, Hkv, dh, D, P, C;
+  int32_t max_queries;
+  int32_t max_splits;
+} photon_config;
+
+/* A KV cache: coarse (one unit per sequence), token-level (for
+ * photon_flat_attn) or chunk-local (one unit per chunk buffer, cap = P + C).
+ *   k, v        [n_units, Hkv, cap, dh]; rows [0, len[u]) of unit u are valid,
+ *               rows beyond may hold anything (including NaN bit patterns)
+ *               and never influence a result.
+ *   len         [n_units] device int32.
+ *   max_len     host-side upper bound on every len[u] during the call
+ *               (0 = cap); only steers how many key splits are launched.
+ * Optional shared prefixes (Section 1: long-context, multi-query serving; one
+ * document, many query branches): unit u with shared_id[u] = s >= 0 attends
+ * rows [0, shared_len[s]) of segment s followed by its own rows, exactly as
+ * if the prefix had been copied in front of its cache; the prefix is stored
+ * and read once.  k_shared = NULL disables this.
+ *   k_shared, v_shared [n_shared, Hkv, cap_shared, dh]; shared_len [n_shared];
+ *   shared_id [n_units], -1 = none; max_shared_len like max_len. */
+typedef struct {
+  photon_bf16 *k, *v;
+  int32_t *len;
+  int32_t n_units, cap, max_len;
+  const photon_bf16 *k_shared, *v_shared;
+  const int32_t *shared_len, *shared_id;
+  int32_t n_shared, cap_shared, max_shared_len;
+} photon_kv;
+
+/* Creates a context on the current CUDA device: validates cfg, allocates the
+ * split-K workspace and the status word.  The only allocating call besides
+ * photon_destroy's frees.  *out is NULL on failure. */
+photon_status photon_create(photon_ctx **out, const photon_config *cfg);
+photon_status photon_destroy(photon_ctx *ctx);
+
+/* Cache half of the streaming update STEP (Eq. 12, Eq. 13): KV_{<=g} is
+ * KV_{<=g-1} plus the new unit's K and V.  Item i (i < n) writes n_rows rows
+ * k_new, v_new [n, n_rows, Hkv, dh] into unit u = unit_ids ? unit_ids[i] : i
+ * at rows len[u] .. len[u]+n_rows-1 and adds n_rows to len[u].  A bit copy.
+ * Unit ids within one call must be distinct.  With n_rows = P the same call
+ * installs a chunk's prefix rows; with n_rows = 1 it appends an in-chunk row
+ * (chunk-local caches are discarded at chunk boundaries by resetting len,
+ * Section 2.3.3).  No room: nothing written, PHOTON_DEV_CAPACITY. */
+photon_status photon_kv_append(photon_ctx *ctx, photon_kv *cache, const photon_bf16 *k_new,
+                               const photon_bf16 *v_new, const int32_t *unit_ids, int32_t n,
+                               int32_t n_rows, photon_stream stream);
+
+/* Attention half of STEP for the coarsest stream (Eq. 12; causal Transformer
+ * F^(L) of Section 2.1.1 whose cache holds T / C_{<=L} units, Section 2.3.3):
+ * for unit u and query head h,
+ *   s_i = scale * <q[u,h], K[u,h/G,i]>,  i over the shared prefix rows (if any)
+ *   then rows [0, len[u]);  out[u,h] = sum_i softmax(s)_i V[u,h/G,i].
+ * For the newest position the causal mask selects exactly the valid rows, so
+ * a caller appends first and then attends.  q, out: [n_units, Hq, dh] bf16;
+ * lse: [n_units, Hq] float (log-sum-exp of the logits, natural log) or NULL.
+ * No valid key: out row = 0, lse = -inf.  fp32 accumulation, one rounding to
+ * bf16 at the output.  Keys are split into ranges whose partial results are
+ * merged by log-sum-exp; a shared prefix is read once for all its branches. */
+photon_status photon_coarse_attn(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
+                                 photon_bf16 *out, float *lse, float scale, photon_stream stream);
+
+/* The same operation on a token-level cache (what a flat Transformer reads
+ * per generated token, Section 2.3.1); exists to report KV bytes per token
+ * of the flat baseline next to the coarse stream's. */
+photon_status photon_flat_attn(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
+                               photon_bf16 *out, float *lse, float scale, photon_stream stream);
+
+/* Context converter U^(l) (Section 2.1.2): one latent -> P conditioning
+ * vectors, U[b, r, j] = sum_k x[b,k] * W[k, r*D + j] (+ bias[r*D + j]).
+ * x [B, D]; w in the order given by w_layout; bias [P*D] or NULL;
+ * U [B, P, D]; all bf16, fp32 accumulation, one rounding at the output. */
+photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w,
+                               int32_t w_layout, const photon_bf16 *bias, photon_bf16 *U, int32_t B,
+                               photon_stream stream);
+
+/* Bounded causal attention of the local decoders G^(l) (Eq. 6-7): query c
+ * (q [Nc, Hq, dh]) attends rows [0, len[u]) of chunk buffer u = slot ?
+ * slot[c] : c of `chunks` (cap = P + C; rows 0..P-1 the converter prefix,
+ * rows P.. the in-chunk positions written so far) and nothing else, so the
+ * span is bounded by P + C whatever the context length.  out [Nc, Hq, dh].
+ * Shared-prefix fields of `chunks` must be unset. */
+photon_status photon_chunk_attn(photon_ctx *ctx, const photon_kv *chunks, const photon_bf16 *q,
+                                const int32_t *slot, photon_bf16 *out, int32_t Nc, float scale,
+                                photon_stream stream);
+
+/* One decode step on one stream, in the order of Section 2.3.3: append
+ * (k_new, v_new) to `coarse`; coarse attention of q_coarse over the grown
+ * cache -> out_coarse (lse_coarse optional); converter on x, or, when x is
+ * NULL, on out_coarse viewed as [B, Hq*dh] (requires Hq*dh == D and
+ * B == coarse->n_units); chunk attention of q_chunk over `chunks`.
+ * ev_attn_begin / ev_attn_end, when not NULL, are recorded on the stream
+ * around the coarse attention launches (for timing that part in place). */
+typedef struct {
+  photon_kv *coarse;
+  const photon_bf16 *k_new, *v_new, *q_coarse;
+  photon_bf16 *out_coarse;
+  float *lse_coarse;
+  float scale_coarse;
+  const photon_bf16 *x, *w, *bias;
+  int32_t w_layout;
+  photon_bf16 *U;
+  int32_t B;
+  const photon_kv *chunks;
+  const photon_bf16 *q_chunk;
+  const int32_t *slot;
+  photon_bf16 *out_chunk;
+  int32_t Nc;
+  float scale_chunk;
+  photon_event ev_attn_begin, ev_attn_end;
+} photon_step_args;
+
+photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, photon_stream stream);
+
+/* Reads (and optionally clears) the device status word.  Synchronises the
+ * whole device; the only call that does. */
+photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear);
+
+/* Number of kernels the library has launched through this context so far. */
+int64_t photon_launch_count(const photon_ctx *ctx);
+
+const char *photon_status_str(photon_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PHOTON_H */

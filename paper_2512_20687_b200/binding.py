@@ -1,0 +1,220 @@
+"""Thin ctypes binding of libphoton.so: same names as include/photon.h,
+argument marshalling only.  Tensors are torch CUDA tensors (bf16 data held as
+torch.bfloat16 or as raw int16/uint16 bits; int32 index arrays); the binding
+passes their data pointers and the current (or a given) CUDA stream.  Every
+step of the path runs in the library's kernels; there is no fallback: if the
+shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_int64, c_void_p
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libphoton.so")
+
+PHOTON_OK, PHOTON_ERR_INVALID_ARG, PHOTON_ERR_UNSUPPORTED, PHOTON_ERR_CUDA, PHOTON_ERR_WORKSPACE = range(5)
+PHOTON_DEV_CAPACITY, PHOTON_DEV_BAD_INDEX, PHOTON_DEV_TIMEOUT = 1, 2, 4
+PHOTON_W_IN_MAJOR, PHOTON_W_OUT_MAJOR = 0, 1
+
+
+class PhotonError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {photon_status_str(code)} (status {code})")
+
+
+class photon_config(Structure):
+    _fields_ = [(n, c_int32) for n in ("Hq", "Hkv", "dh", "D", "P", "C", "max_queries", "max_splits")]
+
+
+class photon_kv(Structure):
+    _fields_ = [
+        ("k", c_void_p), ("v", c_void_p), ("len", c_void_p),
+        ("n_units", c_int32), ("cap", c_int32), ("max_len", c_int32),
+        ("k_shared", c_void_p), ("v_shared", c_void_p),
+        ("shared_len", c_void_p), ("shared_id", c_void_p),
+        ("n_shared", c_int32), ("cap_shared", c_int32), ("max_shared_len", c_int32),
+    ]
+
+
+class photon_step_args(Structure):
+    _fields_ = [
+        ("coarse", POINTER(photon_kv)),
+        ("k_new", c_void_p), ("v_new", c_void_p), ("q_coarse", c_void_p),
+        ("out_coarse", c_void_p), ("lse_coarse", c_void_p), ("scale_coarse", c_float),
+        ("x", c_void_p), ("w", c_void_p), ("bias", c_void_p), ("w_layout", c_int32),
+        ("U", c_void_p), ("B", c_int32),
+        ("chunks", POINTER(photon_kv)),
+        ("q_chunk", c_void_p), ("slot", c_void_p), ("out_chunk", c_void_p),
+        ("Nc", c_int32), ("scale_chunk", c_float),
+        ("ev_attn_begin", c_void_p), ("ev_attn_end", c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libphoton.so (built in-tree by paper_2512_20687_b200.build).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2512_20687_b200.build`; "
+            "there is no CPU fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    st = c_int32
+    lib.photon_create.restype = st
+    lib.photon_create.argtypes = [POINTER(c_void_p), POINTER(photon_config)]
+    lib.photon_destroy.restype = st
+    lib.photon_destroy.argtypes = [c_void_p]
+    lib.photon_kv_append.restype = st
+    lib.photon_kv_append.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
+                                     c_int32, c_int32, c_void_p]
+    for name in ("photon_coarse_attn", "photon_flat_attn"):
+        f = getattr(lib, name)
+        f.restype = st
+        f.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p, c_float, c_void_p]
+    lib.photon_converter.restype = st
+    lib.photon_converter.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
+                                     c_int32, c_void_p]
+    lib.photon_chunk_attn.restype = st
+    lib.photon_chunk_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
+                                      c_int32, c_float, c_void_p]
+    lib.photon_decode_step.restype = st
+    lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
+    lib.photon_device_status.restype = st
+    lib.photon_device_status.argtypes = [c_void_p, POINTER(c_int32), c_int32]
+    lib.photon_launch_count.restype = c_int64
+    lib.photon_launch_count.argtypes = [c_void_p]
+    lib.photon_status_str.restype = c_char_p
+    lib.photon_status_str.argtypes = [c_int32]
+    _lib = lib
+    return lib
+
+
+def _ptr(t) -> c_void_p:
+    """Device pointer of a tensor (None -> NULL, int -> as is)."""
+    if t is None:
+        return c_void_p(0)
+    if isinstance(t, int):
+        return c_void_p(t)
+    if not t.is_cuda:
+        raise ValueError("libphoton takes device tensors")
+    if not t.is_contiguous():
+        raise ValueError("libphoton takes contiguous tensors")
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> c_void_p:
+    if stream is None:
+        import torch
+        return c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return c_void_p(stream)
+    return c_void_p(stream.cuda_stream)
+
+
+def _check(code: int, where: str) -> None:
+    if code != PHOTON_OK:
+        raise PhotonError(code, where)
+
+
+def photon_status_str(code: int) -> str:
+    return load().photon_status_str(int(code)).decode()
+
+
+def make_kv(k, v, length, max_len: int = 0, k_shared=None, v_shared=None, shared_len=None,
+            shared_id=None, max_shared_len: int = 0) -> photon_kv:
+    """Fills a photon_kv from tensors k, v [n_units, Hkv, cap, dh], length [n_units]
+    (and the optional shared-prefix tensors).  The struct keeps the tensors alive."""
+    kv = photon_kv()
+    kv.k, kv.v, kv.len = _ptr(k), _ptr(v), _ptr(length)
+    kv.n_units, kv.cap, kv.max_len = k.shape[0], k.shape[2], max_len
+    if k_shared is not None:
+        kv.k_shared, kv.v_shared = _ptr(k_shared), _ptr(v_shared)
+        kv.shared_len, kv.shared_id = _ptr(shared_len), _ptr(shared_id)
+        kv.n_shared, kv.cap_shared, kv.max_shared_len = k_shared.shape[0], k_shared.shape[2], max_shared_len
+    kv._keep = (k, v, length, k_shared, v_shared, shared_len, shared_id)
+    return kv
+
+
+def photon_create(Hq, Hkv, dh, D, P, C, max_queries, max_splits=0) -> c_void_p:
+    cfg = photon_config(Hq, Hkv, dh, D, P, C, max_queries, max_splits)
+    ctx = c_void_p(0)
+    _check(load().photon_create(byref(ctx), byref(cfg)), "photon_create")
+    return ctx
+
+
+def photon_destroy(ctx) -> None:
+    _check(load().photon_destroy(ctx), "photon_destroy")
+
+
+def photon_kv_append(ctx, cache: photon_kv, k_new, v_new, unit_ids=None, n=None, n_rows=1,
+                     stream=None) -> None:
+    if n is None:
+        n = k_new.shape[0]
+    _check(load().photon_kv_append(ctx, byref(cache), _ptr(k_new), _ptr(v_new), _ptr(unit_ids),
+                                   int(n), int(n_rows), _stream(stream)), "photon_kv_append")
+
+
+def photon_coarse_attn(ctx, cache: photon_kv, q, out, lse=None, scale=1.0, stream=None) -> None:
+    _check(load().photon_coarse_attn(ctx, byref(cache), _ptr(q), _ptr(out), _ptr(lse),
+                                     c_float(scale), _stream(stream)), "photon_coarse_attn")
+
+
+def photon_flat_attn(ctx, cache: photon_kv, q, out, lse=None, scale=1.0, stream=None) -> None:
+    _check(load().photon_flat_attn(ctx, byref(cache), _ptr(q), _ptr(out), _ptr(lse),
+                                   c_float(scale), _stream(stream)), "photon_flat_attn")
+
+
+def photon_converter(ctx, x, w, w_layout, bias, U, B=None, stream=None) -> None:
+    if B is None:
+        B = x.shape[0]
+    _check(load().photon_converter(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(U), int(B),
+                                   _stream(stream)), "photon_converter")
+
+
+def photon_chunk_attn(ctx, chunks: photon_kv, q, slot, out, Nc=None, scale=1.0, stream=None) -> None:
+    if Nc is None:
+        Nc = q.shape[0]
+    _check(load().photon_chunk_attn(ctx, byref(chunks), _ptr(q), _ptr(slot), _ptr(out), int(Nc),
+                                    c_float(scale), _stream(stream)), "photon_chunk_attn")
+
+
+def make_step_args(coarse: photon_kv, k_new, v_new, q_coarse, out_coarse, scale_coarse, w, w_layout,
+                   U, B, chunks: photon_kv | None = None, q_chunk=None, out_chunk=None, Nc=0,
+                   scale_chunk=1.0, x=None, bias=None, lse_coarse=None, slot=None,
+                   ev_attn_begin=None, ev_attn_end=None) -> photon_step_args:
+    a = photon_step_args()
+    a.coarse = ctypes.pointer(coarse)
+    a.k_new, a.v_new, a.q_coarse = _ptr(k_new), _ptr(v_new), _ptr(q_coarse)
+    a.out_coarse, a.lse_coarse, a.scale_coarse = _ptr(out_coarse), _ptr(lse_coarse), scale_coarse
+    a.x, a.w, a.bias, a.w_layout = _ptr(x), _ptr(w), _ptr(bias), int(w_layout)
+    a.U, a.B = _ptr(U), int(B)
+    if chunks is not None:
+        a.chunks = ctypes.pointer(chunks)
+    a.q_chunk, a.slot, a.out_chunk = _ptr(q_chunk), _ptr(slot), _ptr(out_chunk)
+    a.Nc, a.scale_chunk = int(Nc), scale_chunk
+    a.ev_attn_begin = c_void_p(ev_attn_begin.cuda_event if ev_attn_begin is not None else 0)
+    a.ev_attn_end = c_void_p(ev_attn_end.cuda_event if ev_attn_end is not None else 0)
+    a._keep = (coarse, chunks, k_new, v_new, q_coarse, out_coarse, lse_coarse, x, w, bias, U,
+               q_chunk, slot, out_chunk, ev_attn_begin, ev_attn_end)
+    return a
+
+
+def photon_decode_step(ctx, args: photon_step_args, stream=None) -> None:
+    _check(load().photon_decode_step(ctx, byref(args), _stream(stream)), "photon_decode_step")
+
+
+def photon_device_status(ctx, clear=True) -> int:
+    bits = c_int32(0)
+    _check(load().photon_device_status(ctx, byref(bits), int(bool(clear))), "photon_device_status")
+    return bits.value
+
+
+def photon_launch_count(ctx) -> int:
+    return int(load().photon_launch_count(ctx))

@@ -1,0 +1,68 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "photon.h"
+
+typedef __nv_bfloat16 bf16;
+
+struct photon_ctx {
+    photon_config cfg;
+    int device;
+    int sm_count;
+    int max_splits;          // resolved upper bound on key ranges per query
+    float *partials;         // split-K workspace: [max_queries * Hq * max_splits * (dh + 2)] floats
+    size_t partial_floats;
+    int32_t *tickets;        // one arrival counter per (query, kv head); zero between calls
+    size_t n_tickets;
+    int32_t *status;         // device status word
+    long long launches;
+};
+
+// Everything an attention launch needs.  A "query" i uses cache unit
+// u = slot ? slot[i] : i.  Its keys are the shared segment's rows (if any)
+// followed by the unit's own rows; the shared part is cut into splits_sh key
+// ranges and the own part into splits_own.
+struct AttnParams {
+    const bf16 *q;
+    bf16 *out;
+    float *lse;
+    const bf16 *k, *v;
+    const int32_t *len;
+    int n_units, cap;
+    const bf16 *ks, *vs;
+    const int32_t *sh_len, *sh_id;
+    int n_shared, cap_sh;
+    const int32_t *slot;
+    int n_q, Hq, Hkv, dh;
+    int splits_own, splits_sh;
+    float scale_log2;        // scale * log2(e): logits are kept in the base-2 domain
+    float *partials;
+    int32_t *tickets;
+    int32_t *status;
+};
+
+struct ConvParams {
+    const bf16 *x, *w, *bias;
+    bf16 *U;
+    int B, D, N;             // N = P * D
+    int w_out_major;
+};
+
+// launchers: enqueue on `st`, add the number of kernels launched to *launches,
+// return the launch error (cudaSuccess when fine)
+cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,
+                             const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
+                             int n_rows, int32_t *status, cudaStream_t st, long long *launches);
+cudaError_t launch_attention(const photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+                             long long *launches);
+cudaError_t launch_chunk_attention(const photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+                                   long long *launches);
+cudaError_t launch_converter(const photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
+                             long long *launches);
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }

@@ -1,0 +1,47 @@
+// KV-cache append: the cache half of the streaming update STEP (Eq. 12, Eq. 13).
+// A bit copy of n_rows new rows per unit plus the length update.
+#include "common.cuh"
+
+// One CTA per appended item.  Every thread reads len[u] before the CTA-wide
+// barrier and only thread 0 writes it after, and unit ids within a call are
+// distinct, so no thread can observe the updated length.
+__global__ void __launch_bounds__(128)
+kv_append_kernel(uint4 *__restrict__ k, uint4 *__restrict__ v, int32_t *__restrict__ len, int n_units,
+                 int Hkv, int cap, int vec_per_row, const uint4 *__restrict__ k_new,
+                 const uint4 *__restrict__ v_new, const int32_t *__restrict__ unit_ids, int n_rows,
+                 int32_t *__restrict__ status) {
+    const int i = blockIdx.x;
+    const int u = unit_ids ? unit_ids[i] : i;
+    if (u < 0 || u >= n_units) {
+        if (threadIdx.x == 0) atomicOr(status, PHOTON_DEV_BAD_INDEX);
+        return;
+    }
+    const int at = len[u];
+    if (at < 0 || at + n_rows > cap) {
+        if (threadIdx.x == 0) atomicOr(status, PHOTON_DEV_CAPACITY);
+        return;
+    }
+    const int per_item = n_rows * Hkv * vec_per_row;
+    for (int t = threadIdx.x; t < per_item; t += blockDim.x) {
+        const int d = t % vec_per_row;
+        const int h = (t / vec_per_row) % Hkv;
+        const int r = t / (vec_per_row * Hkv);
+        const size_t src = (size_t)i * per_item + t;      // [n, n_rows, Hkv, dh]
+        const size_t dst = (((size_t)u * Hkv + h) * cap + (at + r)) * vec_per_row + d;
+        k[dst] = k_new[src];
+        v[dst] = v_new[src];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) len[u] = at + n_rows;
+}
+
+cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,
+                             const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
+                             int n_rows, int32_t *status, cudaStream_t st, long long *launches) {
+    if (n == 0) return cudaSuccess;
+    kv_append_kernel<<<n, 128, 0, st>>>((uint4 *)k, (uint4 *)v, len, n_units, Hkv, cap, dh / 8,
+                                        (const uint4 *)k_new, (const uint4 *)v_new, unit_ids, n_rows,
+                                        status);
+    ++*launches;
+    return cudaGetLastError();
+}

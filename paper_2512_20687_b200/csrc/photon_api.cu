@@ -1,0 +1,283 @@
+// C boundary: context management, argument validation, launch sequencing.
+#include <algorithm>
+#include <cstdio>
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kDefaultMaxSplits = 32;
+constexpr size_t kMaxPartialFloats = size_t(64) << 20;     // 256 MiB ceiling on the split-K workspace
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool kv_ok(const photon_ctx *ctx, const photon_kv *c, bool allow_shared) {
+    if (!c || !c->k || !c->v || !c->len) return false;
+    if (!aligned16(c->k) || !aligned16(c->v)) return false;
+    if (c->n_units < 0 || c->cap <= 0 || c->max_len < 0 || c->max_len > c->cap) return false;
+    if (c->k_shared) {
+        if (!allow_shared) return false;
+        if (!c->v_shared || !c->shared_len || !c->shared_id) return false;
+        if (!aligned16(c->k_shared) || !aligned16(c->v_shared)) return false;
+        if (c->n_shared <= 0 || c->cap_shared <= 0 || c->max_shared_len < 0 ||
+            c->max_shared_len > c->cap_shared)
+            return false;
+    }
+    (void)ctx;
+    return true;
+}
+
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Number of key ranges for a segment whose rows are bounded by max_rows:
+// enough CTAs to cover the SMs a few times over, but at least `min_rows` keys each.
+int choose_splits(const photon_ctx *ctx, int streams, int max_rows, int min_rows, int limit) {
+    if (max_rows <= 0 || streams <= 0) return 1;
+    const int want = ceil_div(ctx->sm_count * 4, streams);
+    const int by_rows = std::max(1, max_rows / min_rows);
+    return std::max(1, std::min(std::min(want, by_rows), limit));
+}
+
+photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
+                               const int32_t *slot, int n_q, photon_bf16 *out, float *lse,
+                               float scale, bool chunk, cudaStream_t st) {
+    if (!ctx) return PHOTON_ERR_INVALID_ARG;
+    if (!kv_ok(ctx, cache, !chunk)) return PHOTON_ERR_INVALID_ARG;
+    if (n_q < 0 || (n_q > 0 && (!q || !out))) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out)) return PHOTON_ERR_INVALID_ARG;
+    if (!(scale == scale)) return PHOTON_ERR_INVALID_ARG;
+    if (n_q == 0) return PHOTON_OK;
+    const photon_config &c = ctx->cfg;
+    AttnParams p{};
+    p.q = reinterpret_cast<const bf16 *>(q);
+    p.out = reinterpret_cast<bf16 *>(out);
+    p.lse = lse;
+    p.k = reinterpret_cast<const bf16 *>(cache->k);
+    p.v = reinterpret_cast<const bf16 *>(cache->v);
+    p.len = cache->len;
+    p.n_units = cache->n_units;
+    p.cap = cache->cap;
+    p.slot = slot;
+    p.n_q = n_q;
+    p.Hq = c.Hq; p.Hkv = c.Hkv; p.dh = c.dh;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.partials = ctx->partials;
+    p.tickets = ctx->tickets;
+    p.status = ctx->status;
+
+    const size_t per_part = size_t(n_q) * c.Hq * (c.dh + 2);
+    const int parts_allowed = (int)std::min<size_t>(ctx->partial_floats / per_part, 1 << 20);
+    const int streams = n_q * c.Hkv;
+    if (chunk) {
+        p.splits_own = 1; p.splits_sh = 0;
+    } else {
+        const int max_len = cache->max_len ? cache->max_len : cache->cap;
+        p.splits_own = choose_splits(ctx, streams, max_len, 128, ctx->max_splits);
+        p.splits_sh = 0;
+        if (cache->k_shared) {
+            p.ks = reinterpret_cast<const bf16 *>(cache->k_shared);
+            p.vs = reinterpret_cast<const bf16 *>(cache->v_shared);
+            p.sh_len = cache->shared_len; p.sh_id = cache->shared_id;
+            p.n_shared = cache->n_shared; p.cap_sh = cache->cap_shared;
+            const int ms = cache->max_shared_len ? cache->max_shared_len : cache->cap_shared;
+            p.splits_sh = choose_splits(ctx, streams, ms, 128, ctx->max_splits);
+        }
+        while (p.splits_own + p.splits_sh > std::min(parts_allowed, ctx->max_splits) &&
+               (p.splits_own > 1 || p.splits_sh > 1)) {
+            if (p.splits_own >= p.splits_sh && p.splits_own > 1) --p.splits_own;
+            else --p.splits_sh;
+        }
+    }
+    if (p.splits_own + p.splits_sh > parts_allowed) return PHOTON_ERR_WORKSPACE;
+    const cudaError_t e = chunk ? launch_chunk_attention(ctx, p, st, &ctx->launches)
+                                : launch_attention(ctx, p, st, &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
+    if (!out) return PHOTON_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = *cfg;
+    if (c.Hq <= 0 || c.Hkv <= 0 || c.dh <= 0 || c.D <= 0 || c.P <= 0 || c.C <= 0 ||
+        c.max_queries <= 0 || c.max_splits < 0)
+        return PHOTON_ERR_INVALID_ARG;
+    if (c.Hq % c.Hkv != 0) return PHOTON_ERR_INVALID_ARG;
+    if (c.dh != 64 && c.dh != 128) return PHOTON_ERR_UNSUPPORTED;
+    if (c.Hq / c.Hkv > 16 || c.D % 64 != 0 || c.P + c.C > 64) return PHOTON_ERR_UNSUPPORTED;
+
+    photon_ctx *ctx = new (std::nothrow) photon_ctx();
+    if (!ctx) return PHOTON_ERR_CUDA;
+    ctx->cfg = c;
+    ctx->max_splits = c.max_splits ? c.max_splits : kDefaultMaxSplits;
+    ctx->launches = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+        cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) {
+        delete ctx;
+        return PHOTON_ERR_CUDA;
+    }
+    if (prop.major != 10) {              // built for sm_100a only
+        delete ctx;
+        return PHOTON_ERR_UNSUPPORTED;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    const size_t per_part = size_t(c.max_queries) * c.Hq * (c.dh + 2);
+    ctx->partial_floats = std::max(per_part, std::min(per_part * ctx->max_splits, kMaxPartialFloats));
+    ctx->n_tickets = size_t(c.max_queries) * c.Hkv;
+    if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&ctx->tickets, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
+        cudaMalloc(&ctx->status, sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) {
+        cudaFree(ctx->partials); cudaFree(ctx->tickets); cudaFree(ctx->status);
+        cudaGetLastError();
+        delete ctx;
+        return PHOTON_ERR_CUDA;
+    }
+    *out = ctx;
+    return PHOTON_OK;
+}
+
+photon_status photon_destroy(photon_ctx *ctx) {
+    if (!ctx) return PHOTON_ERR_INVALID_ARG;
+    cudaFree(ctx->partials);
+    cudaFree(ctx->tickets);
+    cudaFree(ctx->status);
+    delete ctx;
+    return PHOTON_OK;
+}
+
+photon_status photon_kv_append(photon_ctx *ctx, photon_kv *cache, const photon_bf16 *k_new,
+                               const photon_bf16 *v_new, const int32_t *unit_ids, int32_t n,
+                               int32_t n_rows, photon_stream stream) {
+    if (!ctx || !kv_ok(ctx, cache, true)) return PHOTON_ERR_INVALID_ARG;
+    if (n < 0 || n_rows <= 0 || n_rows > cache->cap) return PHOTON_ERR_INVALID_ARG;
+    if (n > 0 && (!k_new || !v_new)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new)) return PHOTON_ERR_INVALID_ARG;
+    if (!unit_ids && n > cache->n_units) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    const cudaError_t e = launch_kv_append(
+        reinterpret_cast<bf16 *>(cache->k), reinterpret_cast<bf16 *>(cache->v), cache->len,
+        cache->n_units, c.Hkv, cache->cap, c.dh, reinterpret_cast<const bf16 *>(k_new),
+        reinterpret_cast<const bf16 *>(v_new), unit_ids, n, n_rows, ctx->status,
+        static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_coarse_attn(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
+                                 photon_bf16 *out, float *lse, float scale, photon_stream stream) {
+    if (!cache) return PHOTON_ERR_INVALID_ARG;
+    return attention_common(ctx, cache, q, nullptr, cache->n_units, out, lse, scale, false,
+                            static_cast<cudaStream_t>(stream));
+}
+
+photon_status photon_flat_attn(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
+                               photon_bf16 *out, float *lse, float scale, photon_stream stream) {
+    if (!cache) return PHOTON_ERR_INVALID_ARG;
+    return attention_common(ctx, cache, q, nullptr, cache->n_units, out, lse, scale, false,
+                            static_cast<cudaStream_t>(stream));
+}
+
+photon_status photon_chunk_attn(photon_ctx *ctx, const photon_kv *chunks, const photon_bf16 *q,
+                                const int32_t *slot, photon_bf16 *out, int32_t Nc, float scale,
+                                photon_stream stream) {
+    if (!ctx || !chunks) return PHOTON_ERR_INVALID_ARG;
+    if (chunks->cap > ctx->cfg.P + ctx->cfg.C) return PHOTON_ERR_INVALID_ARG;
+    if (!slot && Nc > chunks->n_units) return PHOTON_ERR_INVALID_ARG;
+    return attention_common(ctx, chunks, q, slot, Nc, out, nullptr, scale, true,
+                            static_cast<cudaStream_t>(stream));
+}
+
+photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w,
+                               int32_t w_layout, const photon_bf16 *bias, photon_bf16 *U, int32_t B,
+                               photon_stream stream) {
+    if (!ctx || B < 0) return PHOTON_ERR_INVALID_ARG;
+    if (B > 0 && (!x || !w || !U)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(U) || !aligned16(bias))
+        return PHOTON_ERR_INVALID_ARG;
+    if (w_layout != PHOTON_W_IN_MAJOR && w_layout != PHOTON_W_OUT_MAJOR)
+        return PHOTON_ERR_INVALID_ARG;
+    ConvParams p{};
+    p.x = reinterpret_cast<const bf16 *>(x);
+    p.w = reinterpret_cast<const bf16 *>(w);
+    p.bias = reinterpret_cast<const bf16 *>(bias);
+    p.U = reinterpret_cast<bf16 *>(U);
+    p.B = B; p.D = ctx->cfg.D; p.N = ctx->cfg.P * ctx->cfg.D;
+    p.w_out_major = (w_layout == PHOTON_W_OUT_MAJOR);
+    const cudaError_t e = launch_converter(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {
+    if (!ctx || !a || !a->coarse) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    const bool chain = (a->x == nullptr);
+    // validate everything before the first launch so that a bad argument leaves no partial step behind
+    if (!kv_ok(ctx, a->coarse, true) || !a->k_new || !a->v_new || !a->q_coarse || !a->out_coarse)
+        return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(a->k_new) || !aligned16(a->v_new) || !aligned16(a->q_coarse) ||
+        !aligned16(a->out_coarse))
+        return PHOTON_ERR_INVALID_ARG;
+    if (!a->w || !a->U || a->B < 0 || !aligned16(a->w) || !aligned16(a->U) || !aligned16(a->x) ||
+        !aligned16(a->bias))
+        return PHOTON_ERR_INVALID_ARG;
+    if (a->w_layout != PHOTON_W_IN_MAJOR && a->w_layout != PHOTON_W_OUT_MAJOR)
+        return PHOTON_ERR_INVALID_ARG;
+    if (chain && (c.Hq * c.dh != c.D || a->B != a->coarse->n_units)) return PHOTON_ERR_INVALID_ARG;
+    if (a->Nc < 0) return PHOTON_ERR_INVALID_ARG;
+    if (a->Nc > 0) {
+        if (!kv_ok(ctx, a->chunks, false) || !a->q_chunk || !a->out_chunk ||
+            !aligned16(a->q_chunk) || !aligned16(a->out_chunk))
+            return PHOTON_ERR_INVALID_ARG;
+        if (a->chunks->cap > c.P + c.C || (!a->slot && a->Nc > a->chunks->n_units))
+            return PHOTON_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    photon_status s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr,
+                                       a->coarse->n_units, 1, stream);
+    if (s != PHOTON_OK) return s;
+    if (a->ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_begin), st) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
+    s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse,
+                           a->scale_coarse, stream);
+    if (s != PHOTON_OK) return s;
+    if (a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
+    s = photon_converter(ctx, chain ? a->out_coarse : a->x, a->w, a->w_layout, a->bias, a->U, a->B,
+                         stream);
+    if (s != PHOTON_OK) return s;
+    if (a->Nc > 0)
+        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc,
+                              a->scale_chunk, stream);
+    return s;
+}
+
+photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear) {
+    if (!ctx || !bits_out) return PHOTON_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PHOTON_ERR_CUDA;
+    if (cudaMemcpy(bits_out, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
+    if (clear && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return PHOTON_ERR_CUDA;
+    return PHOTON_OK;
+}
+
+int64_t photon_launch_count(const photon_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *photon_status_str(photon_status s) {
+    switch (s) {
+        case PHOTON_OK: return "ok";
+        case PHOTON_ERR_INVALID_ARG: return "invalid argument";
+        case PHOTON_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case PHOTON_ERR_CUDA: return "CUDA runtime error";
+        case PHOTON_ERR_WORKSPACE: return "workspace too small for this call";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

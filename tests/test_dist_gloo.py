@@ -1,0 +1,45 @@
+"""The N > 1 path of the benchmark on CPU: two gloo ranks, independent shards,
+throughput = units summed over ranks / time maxed over ranks."""
+import os
+import socket
+
+import torch.multiprocessing as mp
+
+from paper_2512_20687_b200 import workloads as wl
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, q):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    from paper_2512_20687_b200 import dist as pd
+    r, lr, w = pd.init("gloo")
+    lo, hi = wl.shard_units(101, w, r)
+    pd.barrier()
+    mx = pd.reduce_max(1.0 + r)                # rank 1 is the slow one
+    total = pd.reduce_sum(hi - lo)
+    thr = pd.job_throughput(hi - lo, 1.0 + r)
+    pd.barrier()
+    pd.shutdown()
+    q.put((r, lo, hi, mx, total, thr))
+
+
+def test_two_gloo_ranks_reduce_time_by_max_and_units_by_sum():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [(r[1], r[2]) for r in res] == [(0, 51), (51, 101)]
+    for r in res:
+        assert r[3] == 2.0 and r[4] == 101.0 and abs(r[5] - 101.0 / 2.0) < 1e-12

@@ -1,0 +1,364 @@
+"""Parity of the CUDA path (through the C boundary) with the CPU oracle on the
+same seeded inputs.  Append and index work is bit-exact; bf16 outputs are held
+to max abs error 2e-2 and mean abs error 2e-3 against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_20687_b200 as ph
+from paper_2512_20687_b200 import workloads as wl
+
+from gpu_util import (Ctx, assert_close, chunks_to_dev, coarse_to_dev, dev_bf16, dev_i32, host_bits,
+                      host_f64, shared_of)
+
+pytestmark = pytest.mark.gpu
+
+NT = 16     # oracle threads
+
+
+def cfg_small(i, **kw):
+    return wl.scaled(wl.CONFIGS[i], **kw)
+
+
+# ------------------------------------------------------------------ append
+
+@pytest.mark.parametrize("idx", [0, 1, 4])
+def test_append_is_bit_exact(oracle, idx):
+    cfg = wl.CONFIGS[idx] if idx < 4 else cfg_small(4, B=64)
+    co = wl.coarse_inputs(cfg, poison=True)
+    with Ctx(cfg) as c:
+        d = coarse_to_dev(co)
+        ph.photon_kv_append(c.h, d["kv"], d["k_new"], d["v_new"])
+        assert c.status() == 0
+        flags = oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"])
+        assert flags == 0
+        assert np.array_equal(host_bits(d["k"]), co["k"])
+        assert np.array_equal(host_bits(d["v"]), co["v"])
+        assert np.array_equal(d["len"].cpu().numpy(), co["len"])
+
+
+def test_append_by_unit_index_blocks_overflow_and_bad_ids(oracle):
+    cfg = wl.CONFIGS[0]
+    n_units, cap, P = 9, cfg.P + cfg.C, cfg.P
+    k = wl.normal_bf16(7, "k", (n_units, cfg.Hkv, cap, cfg.dh))
+    v = wl.normal_bf16(7, "v", (n_units, cfg.Hkv, cap, cfg.dh))
+    ln = np.array([0, 0, 5, 0, 8, 2, 0, 0, 1], np.int32)
+    ids = np.array([6, 2, 0, 4, 11, -1, 8], np.int32)        # 2 and 4 lack room; 11 and -1 are bad
+    kn = wl.normal_bf16(7, "kn", (len(ids), P, cfg.Hkv, cfg.dh))
+    vn = wl.normal_bf16(7, "vn", (len(ids), P, cfg.Hkv, cfg.dh))
+    with Ctx(cfg) as c:
+        dk, dv, dl = dev_bf16(k), dev_bf16(v), dev_i32(ln)
+        kv = ph.make_kv(dk, dv, dl)
+        ph.photon_kv_append(c.h, kv, dev_bf16(kn), dev_bf16(vn), unit_ids=dev_i32(ids), n_rows=P)
+        bits = c.status()
+        flags = oracle.kv_append(k, v, ln, kn, vn, unit_ids=ids, n_rows=P)
+        assert bits == flags == (ph.PHOTON_DEV_CAPACITY | ph.PHOTON_DEV_BAD_INDEX)
+        assert np.array_equal(host_bits(dk), k) and np.array_equal(host_bits(dv), v)
+        assert np.array_equal(dl.cpu().numpy(), ln)
+        assert c.status() == 0          # cleared by the previous read
+
+
+# ------------------------------------------------------------------ coarse attention
+
+def run_coarse(c, co, scale, appended=True, flat=False):
+    d = coarse_to_dev(co)
+    out = torch.empty_like(d["q"])
+    lse = torch.empty(d["q"].shape[:2], dtype=torch.float32, device="cuda")
+    (ph.photon_flat_attn if flat else ph.photon_coarse_attn)(c.h, d["kv"], d["q"], out, lse, scale)
+    torch.cuda.synchronize()
+    return host_f64(out), lse.cpu().numpy().astype(np.float64), host_bits(out)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
+def test_coarse_attention_matches_oracle_at_full_size(oracle, idx):
+    cfg = wl.CONFIGS[idx]
+    co = wl.coarse_inputs(cfg, poison=True)
+    oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"])    # attend over S rows
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale,
+                                      shared=shared_of(co), n_threads=NT)
+    with Ctx(cfg) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, f"coarse cfg{idx}")
+    assert np.abs(lse - want_lse).max() < 2e-3
+
+
+@pytest.mark.parametrize("max_splits", [1, 2, 3, 7, 32])
+def test_split_count_does_not_change_the_result(oracle, max_splits):
+    """Ragged lengths incl. 0 and 1, more splits than keys, and splits that
+    receive no keys at all."""
+    cfg = cfg_small(1, B=9, S=700)
+    co = wl.coarse_inputs(cfg, poison=True)
+    lens = np.array([700, 0, 1, 2, 127, 128, 129, 513, 699], np.int32)
+    for u, n in enumerate(lens):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0xFFC1
+    co["len"] = lens
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], lens, scale, n_threads=NT)
+    with Ctx(cfg, max_splits=max_splits) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, f"splits<={max_splits}")
+    assert np.all(got[1] == 0) and np.all(np.isneginf(lse[1]))
+    fin = np.isfinite(want_lse)
+    assert np.abs(lse[fin] - want_lse[fin]).max() < 2e-3
+
+
+def test_shared_prefix_variants(oracle):
+    """Two shared segments of different length, units without a prefix, empty own caches."""
+    cfg = cfg_small(3, B=37, S=40, shared_S=300)
+    co = wl.coarse_inputs(cfg, poison=True)
+    ks = wl.normal_bf16(3, "ks2", (2, cfg.Hkv, 300, cfg.dh))
+    vs = wl.normal_bf16(3, "vs2", (2, cfg.Hkv, 300, cfg.dh))
+    sh_len = np.array([300, 77], np.int32)
+    ks[1, :, 77:] = 0x7FC1
+    vs[1, :, 77:] = 0x7FC1
+    sh_id = (np.arange(cfg.B) % 3 - 1).astype(np.int32)       # -1, 0, 1, -1, ...
+    lens = (np.arange(cfg.B) % 5 * 9).astype(np.int32)        # 0, 9, 18, 27, 36
+    for u, n in enumerate(lens):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0x7FC1
+    co.update(k_shared=ks, v_shared=vs, shared_len=sh_len, shared_id=sh_id, len=lens)
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], lens, scale, shared=shared_of(co),
+                                      n_threads=NT)
+    with Ctx(cfg) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, "shared prefix")
+    empty = (lens == 0) & (sh_id < 0)
+    assert empty.any() and np.all(got[empty] == 0) and np.all(np.isneginf(lse[empty]))
+    fin = np.isfinite(want_lse)
+    assert np.abs(lse[fin] - want_lse[fin]).max() < 2e-3
+
+
+def test_bad_shared_id_is_flagged_and_zeroed(oracle):
+    cfg = cfg_small(3, B=6, S=20, shared_S=50)
+    co = wl.coarse_inputs(cfg)
+    co["len"][:] = 20
+    co["shared_id"] = np.array([0, 0, 5, 0, -1, 0], np.int32)
+    scale = cfg.dh ** -0.5
+    want, _, flags = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale,
+                                      shared=shared_of(co), want_flags=True)
+    with Ctx(cfg) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == flags == ph.PHOTON_DEV_BAD_INDEX
+    assert np.all(got[2] == 0) and np.all(np.isneginf(lse[2]))
+    assert_close(got, want, "bad shared id")
+
+
+def test_attention_is_deterministic_and_batch_permutation_equivariant():
+    cfg = cfg_small(1, B=24, S=333)
+    co = wl.coarse_inputs(cfg)
+    co["len"] = wl.uniform_int(5, "lens", cfg.B, 0, 333)
+    scale = cfg.dh ** -0.5
+    perm = np.random.default_rng(0).permutation(cfg.B)
+    cp = dict(co, k=co["k"][perm], v=co["v"][perm], q=co["q"][perm], len=co["len"][perm])
+    with Ctx(cfg) as c:
+        _, _, b1 = run_coarse(c, co, scale)
+        _, _, b2 = run_coarse(c, co, scale)
+        _, _, b3 = run_coarse(c, cp, scale)
+    assert np.array_equal(b1, b2) and np.array_equal(b3, b1[perm])
+
+
+def test_flat_attention_on_a_token_level_cache(oracle):
+    cfg = cfg_small(1, B=3, S=4096 + 5)       # token-level cache: one row per token
+    co = wl.coarse_inputs(cfg, poison=True)
+    scale = cfg.dh ** -0.5
+    want, _ = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        got, _, _ = run_coarse(c, co, scale, flat=True)
+    assert_close(got, want, "flat")
+
+
+# ------------------------------------------------------------------ converter
+
+@pytest.mark.parametrize("idx,rows", [(0, None), (1, None), (2, None), (3, 24), (4, 24)])
+@pytest.mark.parametrize("layout", [ph.PHOTON_W_IN_MAJOR, ph.PHOTON_W_OUT_MAJOR])
+def test_converter_matches_oracle(oracle, idx, rows, layout):
+    """Full batch on the device; at the two large batches the oracle recomputes a
+    seeded sample of batch rows (each output row depends on its own x row only)."""
+    cfg = wl.CONFIGS[idx]
+    cv = wl.converter_inputs(cfg, with_bias=(idx == 0))
+    out_major = layout == ph.PHOTON_W_OUT_MAJOR
+    w = cv["w_out_major"] if out_major else cv["w_in_major"]
+    pick = np.arange(cfg.B) if rows is None else np.sort(
+        np.random.default_rng(idx).choice(cfg.B, rows, replace=False))
+    want = oracle.converter(cv["x"][pick], w, cv["bias"], w_out_major=out_major, n_threads=NT)
+    with Ctx(cfg) as c:
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        bias = None if cv["bias"] is None else dev_bf16(cv["bias"])
+        ph.photon_converter(c.h, dev_bf16(cv["x"]), dev_bf16(w), layout, bias, U)
+        torch.cuda.synchronize()
+    assert_close(host_f64(U)[pick], want, f"converter cfg{idx}")
+
+
+def test_converter_one_hot_rows_are_bit_exact_and_ragged_batches_work():
+    cfg = cfg_small(0, B=37)
+    cv = wl.converter_inputs(cfg)
+    x = np.zeros((cfg.B, cfg.D), np.uint16)
+    hot = (np.arange(cfg.B) * 7) % cfg.D
+    x[np.arange(cfg.B), hot] = 0x3F80                           # 1.0
+    with Ctx(cfg) as c:
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        ph.photon_converter(c.h, dev_bf16(x), dev_bf16(cv["w_out_major"]), ph.PHOTON_W_OUT_MAJOR, None, U)
+        torch.cuda.synchronize()
+    assert np.array_equal(host_bits(U).reshape(cfg.B, -1), cv["w_in_major"][hot])
+
+
+# ------------------------------------------------------------------ chunk attention
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_chunk_attention_matches_oracle(oracle, idx):
+    cfg = wl.CONFIGS[idx]
+    ch = wl.chunk_inputs(cfg, poison=True)
+    scale = cfg.dh ** -0.5
+    want, _ = oracle.chunk_attention(ch["q"], ch["kc"], ch["vc"], ch["len"], scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        out = torch.empty_like(d["q"])
+        ph.photon_chunk_attn(c.h, d["kv"], d["q"], None, out, scale=scale)
+        assert c.status() == 0
+    assert_close(host_f64(out), want, f"chunk cfg{idx}")
+
+
+def test_chunk_attention_full_size_chunk_parallel_config_sampled(oracle):
+    """All 16 384 chunks on the device in the benchmark's launch shape; the
+    oracle recomputes a seeded sample of chunks (each is independent of all others)."""
+    cfg = wl.CONFIGS[4]
+    ch = wl.chunk_inputs(cfg, poison=True)
+    scale = cfg.dh ** -0.5
+    pick = np.sort(np.random.default_rng(4).choice(cfg.Nc, 600, replace=False)).astype(np.int32)
+    pick[:3] = [0, 1, 2]
+    pick[-1] = cfg.Nc - 1
+    want, _ = oracle.chunk_attention(ch["q"][pick], ch["kc"], ch["vc"], ch["len"], scale, slot=pick,
+                                     n_threads=NT)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        out = torch.empty_like(d["q"])
+        ph.photon_chunk_attn(c.h, d["kv"], d["q"], None, out, scale=scale)
+        assert c.status() == 0
+    assert_close(host_f64(out)[pick], want, "chunk cfg4 sample")
+
+
+def test_chunk_attention_strict_positions_gather_and_bad_slots(oracle):
+    """n_in = j - 1 (query is the latent before in-chunk position j, incl. the
+    prefix-only case), a gather through `slot`, and an out-of-range slot."""
+    cfg = cfg_small(4, B=4)
+    ch = wl.chunk_inputs(cfg, poison=True, strict_paper=True)
+    assert ch["len"].min() == cfg.P
+    scale = cfg.dh ** -0.5
+    slot = np.random.default_rng(1).permutation(cfg.Nc).astype(np.int32)[:100]
+    slot[17] = cfg.Nc + 3
+    q = ch["q"][:100]
+    want, _, flags = oracle.attention(q, ch["kc"], ch["vc"], ch["len"], scale, slot=slot, want_flags=True)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        dq = dev_bf16(q)
+        out = torch.full_like(dq, 7.0)
+        ph.photon_chunk_attn(c.h, d["kv"], dq, dev_i32(slot), out, scale=scale)
+        assert c.status() == flags == ph.PHOTON_DEV_BAD_INDEX
+    got = host_f64(out)
+    assert np.all(got[17] == 0)
+    assert_close(got, want, "chunk gather")
+
+
+def test_chunk_attention_ignores_other_chunks_bit_exactly():
+    cfg = cfg_small(4, B=2)
+    ch = wl.chunk_inputs(cfg)
+    scale = cfg.dh ** -0.5
+    ch2 = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in ch.items()}
+    other = np.arange(cfg.Nc) != 11
+    ch2["kc"][other] = wl.normal_bf16(77, "a", ch2["kc"][other].shape)
+    ch2["vc"][other] = wl.normal_bf16(78, "a", ch2["vc"][other].shape)
+    ch2["q"][other] = wl.normal_bf16(79, "a", ch2["q"][other].shape)
+    with Ctx(cfg) as c:
+        outs = []
+        for x in (ch, ch2):
+            d = chunks_to_dev(x)
+            out = torch.empty_like(d["q"])
+            ph.photon_chunk_attn(c.h, d["kv"], d["q"], None, out, scale=scale)
+            outs.append(host_bits(out))
+    assert np.array_equal(outs[0][11], outs[1][11]) and not np.array_equal(outs[0][10], outs[1][10])
+
+
+# ------------------------------------------------------------------ the step
+
+@pytest.mark.parametrize("idx", [0, 1, 3])
+@pytest.mark.parametrize("layout", [ph.PHOTON_W_IN_MAJOR, ph.PHOTON_W_OUT_MAJOR])
+def test_decode_step_chain_matches_oracle(oracle, idx, layout):
+    cfg = wl.CONFIGS[idx] if idx != 3 else cfg_small(3, B=48, shared_S=512)
+    s = wl.step_inputs(cfg, poison=True)
+    co, cv, chk = s["coarse"], s["converter"], s["chunks"]
+    out_major = layout == ph.PHOTON_W_OUT_MAJOR
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        d, dc = coarse_to_dev(co), chunks_to_dev(chk)
+        out = torch.empty_like(d["q"])
+        lse = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device="cuda")
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        oc = torch.empty_like(dc["q"])
+        w = dev_bf16(cv["w_out_major"] if out_major else cv["w_in_major"])
+        args = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out, scale, w, layout, U,
+                                 cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc, Nc=cfg.Nc,
+                                 scale_chunk=scale, lse_coarse=lse)
+        n0 = ph.photon_launch_count(c.h)
+        ph.photon_decode_step(c.h, args)
+        assert c.status() == 0
+        assert ph.photon_launch_count(c.h) > n0
+        r = oracle.decode_step(co, cv, chk, scale, scale, chain=True, w_out_major=out_major,
+                               n_threads=NT)
+        assert np.array_equal(host_bits(d["k"]), co["k"]) and np.array_equal(host_bits(d["v"]), co["v"])
+        assert np.array_equal(d["len"].cpu().numpy(), co["len"])
+        assert_close(host_f64(out), r["out"], "step: coarse out")
+        assert_close(host_f64(U), r["U"], "step: U")
+        assert_close(host_f64(oc), r["chunk_out"], "step: chunk out")
+        assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
+
+
+def test_decode_step_with_given_x_and_no_chunks(oracle):
+    cfg = wl.CONFIGS[0]
+    s = wl.step_inputs(cfg)
+    co, cv = s["coarse"], s["converter"]
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        d = coarse_to_dev(co)
+        out = torch.empty_like(d["q"])
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        args = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out, scale,
+                                 dev_bf16(cv["w_in_major"]), ph.PHOTON_W_IN_MAJOR, U, cfg.B,
+                                 x=dev_bf16(cv["x"]))
+        ph.photon_decode_step(c.h, args)
+        assert c.status() == 0
+    want = oracle.converter(cv["x"], cv["w_in_major"])
+    assert_close(host_f64(U), want, "step: U from x")
+
+
+# ------------------------------------------------------------------ argument checks on a live context
+
+def test_invalid_arguments_launch_nothing():
+    cfg = wl.CONFIGS[0]
+    co = wl.coarse_inputs(cfg)
+    with Ctx(cfg) as c:
+        d = coarse_to_dev(co)
+        out = torch.empty_like(d["q"])
+        n0 = ph.photon_launch_count(c.h)
+        with pytest.raises(ph.PhotonError) as e:              # misaligned q
+            ph.photon_coarse_attn(c.h, d["kv"], d["q"].data_ptr() + 2, out, None, 1.0)
+        assert e.value.code == ph.PHOTON_ERR_INVALID_ARG
+        with pytest.raises(ph.PhotonError):                   # NULL out
+            ph.photon_coarse_attn(c.h, d["kv"], d["q"], None, None, 1.0)
+        with pytest.raises(ph.PhotonError):                   # NaN scale
+            ph.photon_coarse_attn(c.h, d["kv"], d["q"], out, None, float("nan"))
+        with pytest.raises(ph.PhotonError):                   # bad layout code
+            ph.photon_converter(c.h, d["q"], d["q"], 5, None, out, 2)
+        with pytest.raises(ph.PhotonError):                   # chunk cache wider than P + C
+            ph.photon_chunk_attn(c.h, d["kv"], d["q"], None, out, 2, 1.0)
+        with pytest.raises(ph.PhotonError):                   # append more rows than capacity
+            ph.photon_kv_append(c.h, d["kv"], d["k_new"], d["v_new"], n_rows=cfg.S + 1)
+        assert ph.photon_launch_count(c.h) == n0 and c.status() == 0
+    with pytest.raises(ph.PhotonError) as e:
+        ph.photon_create(4, 2, 96, 256, 4, 4, 16)
+    assert e.value.code == ph.PHOTON_ERR_UNSUPPORTED
