@@ -237,6 +237,7 @@ def run_gpu(args, cfg) -> None:
     K, W = args.steps, args.warmup
     for i in range(W):
         step(i)
+    lens.copy_(lens0)
     torch.cuda.synchronize()
     n0 = ph.photon_launch_count(ctx)
     step(0)

@@ -88,7 +88,7 @@ def test_coarse_attention_matches_oracle_at_full_size(oracle, idx):
 def test_split_count_does_not_change_the_result(oracle, max_splits):
     """Ragged lengths incl. 0 and 1, more splits than keys, and splits that
     receive no keys at all."""
-    cfg = cfg_small(1, B=9, S=700)
+    cfg = cfg_small(1, B=9, S=701)
     co = wl.coarse_inputs(cfg, poison=True)
     lens = np.array([700, 0, 1, 2, 127, 128, 129, 513, 699], np.int32)
     for u, n in enumerate(lens):
