@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -8,6 +9,22 @@
 #include "photon.h"
 
 typedef __nv_bfloat16 bf16;
+
+// Tensor maps keyed by (base pointer, shape); entries are copied out by value.
+struct TmapCache {
+    static constexpr int kEntries = 64;
+    struct Entry {
+        const void *base;
+        uint64_t rows, cols;
+        uint32_t box_rows;
+        CUtensorMap map;
+    };
+    Entry e[kEntries];
+    int n = 0, next = 0;
+    const CUtensorMap *get(const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+};
+bool make_tmap_bf16_rows(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                         uint32_t box_rows);
 
 struct photon_ctx {
     photon_config cfg;
@@ -20,6 +37,7 @@ struct photon_ctx {
     size_t n_tickets;
     int32_t *status;         // device status word
     long long launches;
+    TmapCache tmaps;
 };
 
 // Everything an attention launch needs.  A "query" i uses cache unit
@@ -39,6 +57,7 @@ struct AttnParams {
     const int32_t *slot;
     int n_q, Hq, Hkv, dh;
     int splits_own, splits_sh;
+    int ctas_own, upc;       // filled by the launcher: CTAs on own keys; units per CTA on shared keys
     float scale_log2;        // scale * log2(e): logits are kept in the base-2 domain
     float *partials;
     int32_t *tickets;
@@ -57,11 +76,11 @@ struct ConvParams {
 cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,
                              const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
                              int n_rows, int32_t *status, cudaStream_t st, long long *launches);
-cudaError_t launch_attention(const photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                              long long *launches);
-cudaError_t launch_chunk_attention(const photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);
-cudaError_t launch_converter(const photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
+cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }

@@ -45,7 +45,7 @@ converter_tile_kernel(const ConvParams p) {
 
 }  // namespace
 
-cudaError_t launch_converter(const photon_ctx *, const ConvParams &p, cudaStream_t st,
+cudaError_t launch_converter(photon_ctx *, const ConvParams &p, cudaStream_t st,
                              long long *launches) {
     if (p.B == 0) return cudaSuccess;
     dim3 grid(p.N / 64, (p.B + 15) / 16);

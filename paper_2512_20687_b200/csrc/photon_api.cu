@@ -49,6 +49,10 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
     if (!(scale == scale)) return PHOTON_ERR_INVALID_ARG;
     if (n_q == 0) return PHOTON_OK;
     const photon_config &c = ctx->cfg;
+    // TMA row coordinates are 32-bit
+    if ((uint64_t)cache->n_units * c.Hkv * cache->cap >= (1ull << 31)) return PHOTON_ERR_UNSUPPORTED;
+    if (cache->k_shared && (uint64_t)cache->n_shared * c.Hkv * cache->cap_shared >= (1ull << 31))
+        return PHOTON_ERR_UNSUPPORTED;
     AttnParams p{};
     p.q = reinterpret_cast<const bf16 *>(q);
     p.out = reinterpret_cast<bf16 *>(out);
