@@ -69,6 +69,7 @@ struct ConvParams {
     bf16 *U;
     int B, D, N;             // N = P * D
     int w_out_major;
+    int32_t *status;
 };
 
 // launchers: enqueue on `st`, add the number of kernels launched to *launches,
