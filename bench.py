@@ -303,87 +303,89 @@ def run_gpu(args, cfg) -> None:
     tokens_total = pd.reduce_sum(cfg.tokens_per_step * K)
     value = tokens_total / sec_max
 
-    # dominant kernel in place: eager steps with events around the coarse attention launches
-    n_ev = min(K, 256)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
-    for a, b in evs:
-        a.record(); b.record()                    # creates the underlying CUDA events
-    torch.cuda.synchronize()
-    ev_args = []
-    for i in range(n_ev):
-        t = reps[i % R]
-        ev_args.append(ph.make_step_args(t["kv"], k_new, v_new, q, t["out"], scale, t["w"], layout,
-                                         t["U"], cfg.B, chunks=t["ckv"], q_chunk=qc, out_chunk=t["oc"],
-                                         Nc=cfg.Nc, scale_chunk=scale, ev_attn_begin=evs[i][0],
-                                         ev_attn_end=evs[i][1]))
-    lens.copy_(lens0)
-    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    ee0.record()
-    for i in range(n_ev):
-        step(i, ev_args[i])
-    ee1.record()
-    torch.cuda.synchronize()
-    lens.copy_(lens0)
-    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
-    eager_ms_per_step = ee0.elapsed_time(ee1) / n_ev
-
+    # per-kernel times: a CUDA graph of back-to-back calls of one part, rotating over the replicas
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except OSError:
         pass
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
-    qo_bytes = 2 * cfg.B * cfg.Hq * cfg.dh * 2
-    attn_alg_bytes = coarse_bytes + qo_bytes
-    traffic = None
-    try:
-        traffic = json.load(open(os.path.join(ROOT, "profiles", "roofline_traffic.json"))).get(
-            f"config{cfg.index}", {}).get("coarse_attn_dram_bytes_per_launch")
-    except OSError:
-        pass
-    achieved = attn_alg_bytes / (attn_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "coarse attention (split-K partial + merge launches)",
-                "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                "traffic": traffic, "algorithmic_bytes": attn_alg_bytes, "us_per_launch": attn_ms * 1e3,
-                "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback 6650 GB/s",
-                "frac_of_nominal_8TBs": achieved / 8000.0}
+    tensor_peak = float(peaks.get("bf16_tflops", 1590.0))
+    peak_src = "MEASURED_PEAKS.json, of measured" if peaks else "6650 GB/s / 1590 TFLOP/s, of fallback"
 
-    # per-part times (eager, events around a batch of calls rotating over the replicas)
-    parts = {}
-    if not args.no_parts:
-        def time_part(fn, n=64):
-            for i in range(8):
-                fn(reps[i % R])
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            a.record()
-            for i in range(n):
-                fn(reps[i % R])
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) * 1e3 / n
-        parts["coarse_attn_us"] = time_part(lambda t: ph.photon_coarse_attn(ctx, t["kv"], q, t["out"], None, scale))
-        parts["converter_us"] = time_part(lambda t: ph.photon_converter(ctx, t["out"].view(cfg.B, -1), t["w"], layout, None, t["U"]))
-        parts["chunk_attn_us"] = time_part(lambda t: ph.photon_chunk_attn(ctx, t["ckv"], qc, None, t["oc"], scale=scale))
-
-        def app(t):
-            ph.photon_kv_append(ctx, t["kv"], k_new, v_new)
-        lens.copy_(lens0)
+    def graph_time_us(fn, reset_lens=False, calls=None, replays=6):
+        calls = calls or R * max(1, 32 // R)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(calls):
+                    fn(reps[i % R])
+                    if reset_lens and i % R == R - 1:
+                        lens.copy_(lens0)
+        g.replay()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record()
-        for i in range(R):
-            app(reps[i])
+        for _ in range(replays):
+            g.replay()
         b.record()
         torch.cuda.synchronize()
-        lens.copy_(lens0)
-        parts["kv_append_us"] = a.elapsed_time(b) * 1e3 / R
-        parts["note"] = "eager back-to-back calls; launch-rate bound below ~3 us"
-        parts["converter_gbs_weights"] = w_bytes / (parts["converter_us"] * 1e-6) / 1e9
-        parts["converter_tflops"] = 2.0 * cfg.B * cfg.D * cfg.P * cfg.D / (parts["converter_us"] * 1e-6) / 1e12
-        parts["chunk_attn_gbs"] = (chunk_bytes + 2 * cfg.Nc * cfg.Hq * cfg.dh * 2) / (parts["chunk_attn_us"] * 1e-6) / 1e9
-        parts["coarse_attn_gbs"] = attn_alg_bytes / (parts["coarse_attn_us"] * 1e-6) / 1e9
+        return a.elapsed_time(b) * 1e3 / (replays * calls)
+
+    qo_coarse = 2 * cfg.B * cfg.Hq * cfg.dh * 2
+    qo_chunk = 2 * cfg.Nc * cfg.Hq * cfg.dh * 2
+    conv_flops = 2.0 * cfg.B * cfg.D * cfg.P * cfg.D
+    conv_bytes = w_bytes + cfg.B * cfg.D * 2 + cfg.B * cfg.P * cfg.D * 2
+    kernels = {
+        "coarse_attn": {"bytes": coarse_bytes + qo_coarse,
+                        "fn": lambda t: ph.photon_coarse_attn(ctx, t["kv"], q, t["out"], None, scale)},
+        "chunk_attn": {"bytes": chunk_bytes + qo_chunk,
+                       "fn": lambda t: ph.photon_chunk_attn(ctx, t["ckv"], qc, None, t["oc"], scale=scale)},
+        "converter": {"bytes": conv_bytes, "flops": conv_flops,
+                      "fn": lambda t: ph.photon_converter(ctx, t["out"].view(cfg.B, -1), t["w"], layout,
+                                                          None, t["U"])},
+        "kv_append": {"bytes": 2 * 2 * cfg.B * cfg.Hkv * cfg.dh * 2, "reset": True,
+                      "fn": lambda t: ph.photon_kv_append(ctx, t["kv"], k_new, v_new)},
+    }
+    parts = {}
+    lens.copy_(lens0)
+    for name, kd in kernels.items():
+        if args.no_parts and name not in ("coarse_attn", "chunk_attn"):
+            continue
+        us = graph_time_us(kd["fn"], reset_lens=kd.get("reset", False))
+        kd["us"] = us
+        parts[name] = {"us": us, "algorithmic_bytes": kd["bytes"], "GBps": kd["bytes"] / us * 1e-3,
+                       "frac_hbm": kd["bytes"] / us * 1e-3 / hbm_peak}
+        if "flops" in kd:
+            parts[name]["TFLOPs"] = kd["flops"] / us * 1e-6
+            t_roof = max(kd["bytes"] / (hbm_peak * 1e3), kd["flops"] / (tensor_peak * 1e6))
+            parts[name]["frac_of_own_roofline"] = t_roof / us
+    lens.copy_(lens0)
+    torch.cuda.synchronize()
+    parts["note"] = ("each part timed as a CUDA graph of back-to-back calls rotating over the replicas; "
+                     "kv_append's figure includes a %d-int length reset every %d calls" % (cfg.B * R, R))
+
+    # roofline of the dominant kernel = the attention part that takes the longest
+    dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
+    traffic, traffic_note = None, "no ncu capture on record for this kernel and workload"
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.txt"))).get(
+            f"config{cfg.index}", {}).get(dom)
+        if rec:
+            import hashlib
+            src = os.path.join(ROOT, "paper_2512_20687_b200", "csrc", rec["source"])
+            if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["source_sha256"]:
+                traffic, traffic_note = rec["dram_bytes_per_launch"], rec.get("how", "")
+            else:
+                traffic_note = "kernel source changed since the ncu counters were taken"
+    except (OSError, ValueError, KeyError):
+        pass
+    ach = kernels[dom]["bytes"] / kernels[dom]["us"] * 1e-3
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
+                "frac": ach / hbm_peak, "traffic": traffic, "traffic_note": traffic_note,
+                "algorithmic_bytes": kernels[dom]["bytes"], "us_per_launch": kernels[dom]["us"],
+                "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0}
+    step_bytes = sum(kernels[n]["bytes"] for n in kernels)
 
     # end to end through the public API with host buffers: H2D of the step's inputs, D2H of its results
     pin = lambda t: t.cpu().pin_memory()
@@ -433,7 +435,8 @@ def run_gpu(args, cfg) -> None:
         "gpu_launches": launches_per_step * K,
         "roofline": roofline,
         "us_per_step": sec_max * 1e6 / K,
-        "eager_us_per_step": eager_ms_per_step * 1e3,
+        "step_hbm": {"algorithmic_bytes": step_bytes, "GBps": step_bytes / (sec_max / K) * 1e-9,
+                     "frac": step_bytes / (sec_max / K) * 1e-9 / hbm_peak},
         "parts": parts,
         "kv_bytes_per_token": {
             "photon_coarse_per_step": coarse_bytes,
