@@ -63,7 +63,7 @@ enum {                                   /* storage order of the converter weigh
  * or 128, Hq/Hkv at most 16, D = d_model a multiple of 64, P + C at most 64.
  * max_queries: largest number of queries (sequences, branches or chunks) any
  * single attention call will carry; max_splits: upper bound on the number of
- * key ranges one query's keys are split into (0 = library default).  Both
+ * key ranges a shared prefix is split into (0 = library default).  Both
  * only size the workspace. */
 typedef struct {
   int32_t Hq, Hkv, dh, D, P, C;
@@ -78,7 +78,7 @@ typedef struct {
  *               and never influence a result.
  *   len         [n_units] device int32.
  *   max_len     host-side upper bound on every len[u] during the call
- *               (0 = cap); only steers how many key splits are launched.
+ *               (0 = cap); only steers how many CTAs are launched.
  * Optional shared prefixes (Section 1: long-context, multi-query serving; one
  * document, many query branches): unit u with shared_id[u] = s >= 0 attends
  * rows [0, shared_len[s]) of segment s followed by its own rows, exactly as
@@ -122,8 +122,11 @@ photon_status photon_kv_append(photon_ctx *ctx, photon_kv *cache, const photon_b
  * a caller appends first and then attends.  q, out: [n_units, Hq, dh] bf16;
  * lse: [n_units, Hq] float (log-sum-exp of the logits, natural log) or NULL.
  * No valid key: out row = 0, lse = -inf.  fp32 accumulation, one rounding to
- * bf16 at the output.  Keys are split into ranges whose partial results are
- * merged by log-sum-exp; a shared prefix is read once for all its branches. */
+ * bf16 at the output.  The keys of all units are dealt out evenly over a
+ * persistent grid; a cache cut by a grid boundary is merged by log-sum-exp in
+ * a fixed order, so a call is deterministic, while the last bits of a unit's
+ * result may depend on where in the batch it sits.  A shared prefix is read
+ * once for all its branches. */
 photon_status photon_coarse_attn(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
                                  photon_bf16 *out, float *lse, float scale, photon_stream stream);
 
@@ -182,6 +185,13 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, 
 /* Reads (and optionally clears) the device status word.  Synchronises the
  * whole device; the only call that does. */
 photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear);
+
+/* Caps the persistent grid of photon_coarse_attn / photon_flat_attn at n CTAs
+ * (0 or more than the device holds: the default, two per SM).  The keys of a
+ * call are dealt out evenly over the grid, so n also moves the points where a
+ * long cache is cut and merged by log-sum-exp; a smaller grid leaves SMs free
+ * for work on another stream.  Takes effect from the next call. */
+photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n);
 
 /* Number of kernels the library has launched through this context so far. */
 int64_t photon_launch_count(const photon_ctx *ctx);

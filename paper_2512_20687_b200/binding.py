@@ -88,6 +88,8 @@ def load() -> ctypes.CDLL:
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_device_status.restype = st
     lib.photon_device_status.argtypes = [c_void_p, POINTER(c_int32), c_int32]
+    lib.photon_set_attention_ctas.restype = st
+    lib.photon_set_attention_ctas.argtypes = [c_void_p, c_int32]
     lib.photon_launch_count.restype = c_int64
     lib.photon_launch_count.argtypes = [c_void_p]
     lib.photon_status_str.restype = c_char_p
@@ -214,6 +216,10 @@ def photon_device_status(ctx, clear=True) -> int:
     bits = c_int32(0)
     _check(load().photon_device_status(ctx, byref(bits), int(bool(clear))), "photon_device_status")
     return bits.value
+
+
+def photon_set_attention_ctas(ctx, n: int) -> None:
+    _check(load().photon_set_attention_ctas(ctx, int(n)), "photon_set_attention_ctas")
 
 
 def photon_launch_count(ctx) -> int:

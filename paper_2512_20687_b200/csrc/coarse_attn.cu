@@ -1,0 +1,613 @@
+// Decode attention of the coarsest stream (attention half of STEP, Eq. 12) and
+// of a token-level cache: one query position per unit over the valid rows of
+// its own KV cache.  HBM-bound: every valid K and V row is streamed once.
+//
+// Work is cut into tiles of 64 keys of one (unit, KV head) stream.  The tiles
+// of all streams, in stream order, form one sequence; a persistent grid (two
+// CTAs per SM) gives every CTA an equal contiguous share of it, whatever the
+// lengths of the individual caches, so there is one wave and no tail.  The
+// split points are found on the device from len[] by a block-wide prefix sum.
+//
+// Inside a CTA one thread drives a ring of TMA loads (128-byte-swizzled boxes of
+// 32 rows, so rows past the end of a cache are not fetched; the group's query
+// rows ride along with the first tile of each stream), four warps consume the
+// tiles, and a sixth warp finishes streams (everything that needs a round trip
+// to global memory) while the consumers are already on the next stream.
+// Each consumer warp takes 16 keys of every tile, evaluates S^T = K Q^T and
+// O^T += V^T P^T with mma.sync tiles whose M side is the keys / head features
+// and whose N side is the G <= 16 query heads of the group (so a 16-key block
+// costs 2 * dh/16 MMAs whatever G is), and keeps an fp32 online softmax in the
+// base-2 domain.  With G query rows per KV head the contraction has G flop per
+// byte, far below the tensor ridge: the tensor pipe only has to keep pace with
+// HBM, which is why this is not a tcgen05 kernel.
+//
+// A stream that lies inside one CTA is finished there.  A stream cut by a CTA
+// boundary leaves one unnormalised partial (acc, m, l) per CTA in a small
+// workspace; the CTA that arrives last on the stream's ticket (an atomic
+// counter, no waiting) merges the partials in CTA order by log-sum-exp, so the
+// result does not depend on arrival order.  Partials of a shared prefix, when
+// present, were produced by an earlier launch and are folded in at the same
+// point.
+#include <math_constants.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace {
+
+constexpr int NW = 4;                      // consumer warps per CTA
+constexpr int BN = 64;                     // keys per tile
+constexpr int BOX = 32;                    // rows per TMA box
+constexpr int THREADS = (NW + 2) * 32;     // + one producer warp + one finishing warp
+constexpr int STAGES = 3;
+constexpr int HALF_BYTES = BN * 128;       // 64 rows x 64 elements, swizzled
+constexpr int BOX_BYTES = BOX * 128;
+constexpr int CTAS_PER_SM = 2;
+
+template <int DH>
+struct Ring {
+    static constexpr int HALVES = DH / 64;
+    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;     // K (or V) tile
+    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+};
+
+__host__ __device__ inline int q_slot_bytes(int G, int dh) { return (G * dh * 2 + 127) / 128 * 128; }
+
+template <int DH>
+size_t smem_bytes(int G) {
+    return 1024 /*alignment slack*/ + size_t(STAGES) * (Ring<DH>::STAGE_BYTES + q_slot_bytes(G, DH)) +
+           size_t(NW) * G * (DH + 2) * sizeof(float) + 128 /*barriers*/ + 128 /*scalars*/;
+}
+
+__device__ __forceinline__ int clamp_len(int len, int cap) { return max(0, min(len, cap)); }
+__device__ __forceinline__ int tiles_of(int len) { return (len + BN - 1) / BN; }
+
+// Position in the sequence of tiles: tile j of the stream (unit u, KV head h).
+struct Walker {
+    int u, h, j, nt, len;
+    __device__ __forceinline__ void load(const AttnParams &p) {
+        len = clamp_len(p.len[u], p.cap);
+        nt = tiles_of(len);
+    }
+    __device__ __forceinline__ void next(const AttnParams &p) {
+        if (++j < nt) return;
+        j = 0;
+        if (++h < p.Hkv) return;
+        h = 0;
+        do {
+            if (++u >= p.n_units) { nt = 0; len = 0; return; }
+            load(p);
+        } while (nt == 0);
+    }
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+
+// Final value of one output element: own keys (acc, M, L in the base-2 domain,
+// unnormalised) combined with the partials of the unit's shared prefix.
+template <int DH>
+__device__ __forceinline__ void emit(const AttnParams &p, int u, int hq, int d, float acc, float M, float L) {
+    const size_t qh = (size_t)u * p.Hq + hq;
+    if (p.splits_sh > 0) {
+        const int s = p.sh_id[u];
+        if (s >= p.n_shared) {                       // bad shared id voids the query
+            if (d == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+            L = 0.f; acc = 0.f;
+        } else if (s >= 0) {
+            const float *sp = p.partials + qh * p.splits_sh * (DH + 2);
+            for (int j = 0; j < p.splits_sh; ++j) {
+                const float *pj = sp + (size_t)j * (DH + 2);
+                const float lj = __ldcg(pj + DH + 1);
+                if (!(lj > 0.f)) continue;
+                const float mj = __ldcg(pj + DH);
+                const float Mn = fmaxf(M, mj);
+                const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
+                acc = acc * f0 + __ldcg(pj + d) * f1;
+                L = L * f0 + lj * f1;
+                M = Mn;
+            }
+        }
+    }
+    p.out[qh * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+    if (d == 0 && p.lse) p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
+}
+
+// The finishing warp holds, per lane, V consecutive features [d0, d0 + V) of one query head
+// (acc unnormalised, M and L of that head).  Same combination as emit(), with every partial
+// fetched by independent loads (one round trip per partial).
+template <int DH, int MAXV>
+__device__ __forceinline__ void emit_row(const AttnParams &p, int u, int hq, int d0, int V, bool lead,
+                                         float (&acc)[MAXV], float M, float L) {
+    const size_t qh = (size_t)u * p.Hq + hq;
+    if (p.splits_sh > 0) {
+        const int s = p.sh_id[u];
+        if (s >= p.n_shared) {
+            if (lead) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+            L = 0.f;
+        } else if (s >= 0) {
+            const float *sp = p.partials + qh * p.splits_sh * (DH + 2);
+            for (int j = 0; j < p.splits_sh; ++j) {
+                const float *pj = sp + (size_t)j * (DH + 2);
+                const float lj = __ldcg(pj + DH + 1), mj = __ldcg(pj + DH);
+                float2 a[MAXV / 2];
+#pragma unroll
+                for (int i = 0; i < MAXV / 2; ++i)
+                    a[i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
+                if (!(lj > 0.f)) continue;
+                const float Mn = fmaxf(M, mj);
+                const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
+#pragma unroll
+                for (int i = 0; i < MAXV / 2; ++i) {
+                    acc[2 * i] = acc[2 * i] * f0 + a[i].x * f1;
+                    acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[i].y * f1;
+                }
+                L = L * f0 + lj * f1;
+                M = Mn;
+            }
+        }
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + qh * DH + d0);
+#pragma unroll
+    for (int i = 0; i < MAXV / 2; ++i)
+        if (2 * i < V) dst[i] = pack_bf16(acc[2 * i] * inv, acc[2 * i + 1] * inv);
+    if (lead && p.lse) p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
+}
+
+// One 16-key block of a tile for this warp.
+//   kt, vt   shared-memory addresses of the K and V tiles (swizzled boxes)
+//   kb       index of the 16-key block inside the tile;  valid: keys of it in range (1..16)
+//   qb       Q^T fragments: [n-tile of 8 heads][16-wide slice of dh][2]
+//   o        O^T accumulators: [n-tile][16-row slice of dh][4]
+//   m, l     running maximum and (per-thread partial) sum for heads 2c, 2c+1 of each n-tile
+template <int DH, int NT8>
+__device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, int valid,
+                                              const uint32_t (&qb)[NT8][DH / 16][2],
+                                              float (&o)[NT8][DH / 16][4], float (&m)[NT8][2],
+                                              float (&l)[NT8][2], float scale_log2, int lane) {
+    const int g = lane >> 2, c = lane & 3;
+    const int mi = lane >> 3, r8 = lane & 7;
+    float s[NT8][2][4];
+#pragma unroll
+    for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[nt][a][e] = 0.f;
+
+    // S^T = K Q^T : A fragments (keys x dh) straight from the swizzled K tile
+    {
+        const int row = kb * 16 + r8 + (mi & 1) * 8;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+            const int cfull = ks * 2 + (mi >> 1);                // 16-byte chunk along dh
+            const uint32_t addr = kt + (cfull >> 3) * HALF_BYTES + row * 128 + (((cfull & 7) ^ (row & 7)) << 4);
+            uint32_t a[4];
+            ptx::ldmatrix_x4(a, addr);
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt) ptx::mma_bf16_16816(s[nt][ks & 1], a, qb[nt][ks][0], qb[nt][ks][1]);
+        }
+    }
+    // online softmax over the keys (rows g and g+8 of the block), per head column
+    uint32_t pb[NT8][2];
+    bool rescale = false;
+    float corr[NT8][2];
+#pragma unroll
+    for (int nt = 0; nt < NT8; ++nt) {
+        float p_lo[2], p_hi[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float s_lo = (s[nt][0][j] + s[nt][1][j]) * scale_log2;            // key g
+            float s_hi = (s[nt][0][2 + j] + s[nt][1][2 + j]) * scale_log2;    // key g + 8
+            if (g >= valid) s_lo = -CUDART_INF_F;
+            if (g + 8 >= valid) s_hi = -CUDART_INF_F;
+            float mx = fmaxf(s_lo, s_hi);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float mn = fmaxf(m[nt][j], mx);                 // key 0 of a block is always in range
+            corr[nt][j] = exp2f(m[nt][j] - mn);
+            rescale |= (corr[nt][j] != 1.f);
+            p_lo[j] = exp2f(s_lo - mn);
+            p_hi[j] = exp2f(s_hi - mn);
+            l[nt][j] = l[nt][j] * corr[nt][j] + (p_lo[j] + p_hi[j]);
+            m[nt][j] = mn;
+        }
+        // P (keys x heads) -> P^T fragments (B operand: keys along k, head g of this thread)
+        pb[nt][0] = ptx::movmatrix_trans(pack_bf16(p_lo[0], p_lo[1]));
+        pb[nt][1] = ptx::movmatrix_trans(pack_bf16(p_hi[0], p_hi[1]));
+    }
+    // masks that clear V entries of keys past the end (they may hold anything)
+    uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
+    if (valid < 16) {
+        vm0 = (2 * c < valid ? 0x0000FFFFu : 0u) | (2 * c + 1 < valid ? 0xFFFF0000u : 0u);
+        vm1 = (2 * c + 8 < valid ? 0x0000FFFFu : 0u) | (2 * c + 9 < valid ? 0xFFFF0000u : 0u);
+    }
+    if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+        for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < DH / 16; ++mt) {
+                o[nt][mt][0] *= corr[nt][0]; o[nt][mt][1] *= corr[nt][1];
+                o[nt][mt][2] *= corr[nt][0]; o[nt][mt][3] *= corr[nt][1];
+            }
+    }
+    // O^T += V^T P^T : A fragments (dh x keys) through transposing loads of the V tile
+    {
+        const int row = kb * 16 + r8 + (mi >> 1) * 8;
+#pragma unroll
+        for (int mt = 0; mt < DH / 16; ++mt) {
+            const int cfull = mt * 2 + (mi & 1);
+            const uint32_t addr = vt + (cfull >> 3) * HALF_BYTES + row * 128 + (((cfull & 7) ^ (row & 7)) << 4);
+            uint32_t a[4];
+            ptx::ldmatrix_x4_trans(a, addr);
+            a[0] &= vm0; a[1] &= vm0; a[2] &= vm1; a[3] &= vm1;
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt) ptx::mma_bf16_16816(o[nt][mt], a, pb[nt][0], pb[nt][1]);
+        }
+    }
+}
+
+template <int DH, int NT8>
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
+coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v) {
+    using R = Ring<DH>;
+    extern __shared__ uint8_t smem_raw[];
+    const int G = p.Hq / p.Hkv;
+    const int QB = q_slot_bytes(G, DH);
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+    const uint32_t q_base = base + STAGES * R::STAGE_BYTES;
+    float *red = reinterpret_cast<float *>(gen + STAGES * (R::STAGE_BYTES + QB));      // [NW][G][DH + 2]
+    uint8_t *tail = reinterpret_cast<uint8_t *>(red) + (size_t)NW * G * (DH + 2) * sizeof(float);
+    const uint32_t bars = ptx::smem_u32(tail);                  // full[s] at +16s, empty[s] at +16s+8
+    const uint32_t red_full = bars + 16 * STAGES, red_empty = red_full + 8;
+    int *sc = reinterpret_cast<int *>(tail + 128);              // [0..5] warp sums, [8] u0, [9] rem, [11] dead,
+    volatile int *dead = sc + 11;                               // [16..23] description of the stream in `red`
+    volatile int *meta = sc + 16;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(bars + 16 * s, 1);
+            ptx::mbar_init(bars + 16 * s + 8, NW);
+        }
+        ptx::mbar_init(red_full, NW);
+        ptx::mbar_init(red_empty, 1);
+        sc[8] = -1; sc[9] = 0; sc[11] = 0;
+        ptx::mbar_fence_init();
+        ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
+    }
+
+    // ---- where this CTA's share of the tile sequence starts: block-wide prefix sum of tile counts
+    const int per = (p.n_units + THREADS - 1) / THREADS;
+    const int ub = min(p.n_units, (int)threadIdx.x * per), ue = min(p.n_units, ub + per);
+    int mine = 0;
+    for (int u = ub; u < ue; ++u) mine += tiles_of(clamp_len(p.len[u], p.cap));
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) sc[warp] = incl;
+    __syncthreads();
+    int before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w) {
+        if (w < warp) before += sc[w];
+        all += sc[w];
+    }
+    const long long T = (long long)all * p.Hkv;                  // tiles in the whole call
+    // every CTA that takes part owns at least one tile, so the CTAs holding a stream are consecutive
+    const int n_cta = (int)min((long long)gridDim.x, T);
+    const long long t0 = cta < n_cta ? T * cta / n_cta : 0, t1 = cta < n_cta ? T * (cta + 1) / n_cta : 0;
+    {
+        const long long lo = (long long)(before + incl - mine) * p.Hkv, hi = lo + (long long)mine * p.Hkv;
+        if (t0 < t1 && lo <= t0 && t0 < hi) {
+            long long pre = lo;
+            for (int u = ub; u < ue; ++u) {
+                const long long k = (long long)tiles_of(clamp_len(p.len[u], p.cap)) * p.Hkv;
+                if (t0 < pre + k) { sc[8] = u; sc[9] = (int)(t0 - pre); break; }
+                pre += k;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- units without own keys are visited by no tile: finish them here
+    for (int u = cta; u < p.n_units; u += gridDim.x) {
+        if (clamp_len(p.len[u], p.cap) != 0) continue;
+        for (int idx = threadIdx.x; idx < p.Hq * DH; idx += THREADS)
+            emit<DH>(p, u, idx / DH, idx % DH, 0.f, -CUDART_INF_F, 0.f);
+    }
+    if (t0 >= t1) return;
+
+    const int n_tiles = (int)(t1 - t0);
+
+    if (warp == NW + 1) {
+        // ======================= finishing warp =======================
+        // lane -> (query head r of the group, features [d0, d0 + V))
+        constexpr int MAXV = DH * 8 * NT8 / 32;
+        int Gp = 1;
+        while (Gp < G) Gp <<= 1;
+        const int lpr = 32 / Gp;                        // lanes per query head
+        const int r = lane / lpr, V = DH / lpr, d0 = (lane % lpr) * V;
+        const bool row_ok = r < G, lead = row_ok && (lane % lpr == 0);
+        for (int sidx = 0;; ++sidx) {
+            if (*dead || !ptx::mbar_wait(red_full, sidx & 1)) {
+                if (!*dead) { *dead = 1; if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT); }
+                break;
+            }
+            const int u = meta[0], h = meta[1], flags = meta[2], c_first = meta[3], c_last = meta[4];
+            const bool whole = flags & 1, final_seg = flags & 2;
+            float acc[MAXV], M = -CUDART_INF_F, L = 0.f;
+#pragma unroll
+            for (int i = 0; i < MAXV; ++i) acc[i] = 0.f;
+            if (row_ok) {
+#pragma unroll
+                for (int ww = 0; ww < NW; ++ww) {
+                    const float *src = red + ((size_t)ww * G + r) * (DH + 2);
+                    if (src[DH + 1] > 0.f) M = fmaxf(M, src[DH]);
+                }
+#pragma unroll
+                for (int ww = 0; ww < NW; ++ww) {
+                    const float *src = red + ((size_t)ww * G + r) * (DH + 2);
+                    const float lw = src[DH + 1];
+                    if (lw > 0.f) {
+                        const float f = exp2f(src[DH] - M);
+                        L += lw * f;
+#pragma unroll
+                        for (int i = 0; i < MAXV / 2; ++i)
+                            if (2 * i < V) {
+                                const float2 a = *reinterpret_cast<const float2 *>(src + d0 + 2 * i);
+                                acc[2 * i] += a.x * f; acc[2 * i + 1] += a.y * f;
+                            }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(red_empty);          // consumers may reuse `red`
+            if (whole) {
+                if (row_ok) emit_row<DH, MAXV>(p, u, h * G + r, d0, V, lead, acc, M, L);
+            } else {
+                // the stream is shared with neighbouring CTAs: leave a partial, whoever arrives last merges
+                if (row_ok) {
+                    float *dst = p.cta_partials + ((size_t)(2 * cta + (cta < c_last ? 1 : 0)) * G + r) * (DH + 2);
+#pragma unroll
+                    for (int i = 0; i < MAXV / 2; ++i)
+                        if (2 * i < V) *reinterpret_cast<float2 *>(dst + d0 + 2 * i) = make_float2(acc[2 * i], acc[2 * i + 1]);
+                    if (lead) { dst[DH] = M; dst[DH + 1] = L; }
+                }
+                __threadfence();
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) {
+                    int *ticket = p.tickets + (size_t)u * p.Hkv + h;
+                    last = (atomicAdd(ticket, 1) == c_last - c_first);
+                    if (last) *ticket = 0;                       // zero again for the next call
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    if (row_ok) {
+                        M = -CUDART_INF_F; L = 0.f;
+#pragma unroll
+                        for (int i = 0; i < MAXV; ++i) acc[i] = 0.f;
+                        for (int cc = c_first; cc <= c_last; cc += 2) {
+                            // two partials per trip: all their loads are in flight together
+                            float mj[2], lj[2];
+                            float2 a[2][MAXV / 2];
+#pragma unroll
+                            for (int t = 0; t < 2; ++t) {
+                                const int c2 = min(cc + t, c_last);
+                                const float *src = p.cta_partials +
+                                                   ((size_t)(2 * c2 + (c2 < c_last ? 1 : 0)) * G + r) * (DH + 2);
+                                lj[t] = __ldcg(src + DH + 1); mj[t] = __ldcg(src + DH);
+#pragma unroll
+                                for (int i = 0; i < MAXV / 2; ++i)
+                                    a[t][i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(src + d0) + i)
+                                                        : make_float2(0.f, 0.f);
+                            }
+                            if (cc + 1 > c_last) lj[1] = 0.f;
+#pragma unroll
+                            for (int t = 0; t < 2; ++t) {
+                                if (!(lj[t] > 0.f)) continue;
+                                const float Mn = fmaxf(M, mj[t]);
+                                const float f0 = exp2f(M - Mn), f1 = exp2f(mj[t] - Mn);   // M = -inf at first: f0 = 0
+#pragma unroll
+                                for (int i = 0; i < MAXV / 2; ++i) {
+                                    acc[2 * i] = acc[2 * i] * f0 + a[t][i].x * f1;
+                                    acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[t][i].y * f1;
+                                }
+                                L = L * f0 + lj[t] * f1;
+                                M = Mn;
+                            }
+                        }
+                        emit_row<DH, MAXV>(p, u, h * G + r, d0, V, lead, acc, M, L);
+                    }
+                }
+            }
+            if (final_seg) break;
+        }
+        return;
+    }
+
+    Walker w;
+    w.u = sc[8]; w.h = 0; w.j = 0;
+    w.load(p);
+    w.h = sc[9] / w.nt;
+    w.j = sc[9] % w.nt;
+
+    if (warp == NW) {
+        // ======================= producer: one thread feeds the ring =======================
+        if (lane == 0) {
+            int it = 0;
+            for (; it < n_tiles; ++it, w.next(p)) {
+                const int s = it % STAGES;
+                if (*dead) break;
+                if (!ptx::mbar_wait(bars + 16 * s + 8, ((it / STAGES) & 1) ^ 1)) {
+                    *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
+                }
+                const uint32_t full = bars + 16 * s;
+                const uint32_t kd = base + s * R::STAGE_BYTES, vd = kd + R::TILE_BYTES;
+                const int rows = min(BN, w.len - w.j * BN);
+                const int nbox = (rows + BOX - 1) / BOX;
+                const bool first = (it == 0 || w.j == 0);
+                ptx::mbar_arrive_expect_tx(full, nbox * R::HALVES * BOX_BYTES * 2 + (first ? G * DH * 2 : 0));
+                const int y = (w.u * p.Hkv + w.h) * p.cap + w.j * BN;
+                for (int b = 0; b < nbox; ++b)
+#pragma unroll
+                    for (int hh = 0; hh < R::HALVES; ++hh) {
+                        ptx::tma_load_2d(kd + hh * HALF_BYTES + b * BOX_BYTES, &tm_k, hh * 64, y + b * BOX, full);
+                        ptx::tma_load_2d(vd + hh * HALF_BYTES + b * BOX_BYTES, &tm_v, hh * 64, y + b * BOX, full);
+                    }
+                if (first)
+                    ptx::bulk_load(q_base + s * QB, p.q + ((size_t)w.u * p.Hq + (size_t)w.h * G) * DH, G * DH * 2, full);
+            }
+            if (*dead) {
+                // loads already issued still land in this CTA's shared memory: give them time to finish
+                for (int b = max(0, it - STAGES); b < it; ++b) ptx::mbar_wait(bars + 16 * (b % STAGES), (b / STAGES) & 1);
+            }
+        }
+        return;
+    }
+
+    // ======================= consumers =======================
+    const int g = lane >> 2, c = lane & 3;
+    uint32_t qb[NT8][DH / 16][2];
+    float o[NT8][DH / 16][4];
+    float m[NT8][2], l[NT8][2];
+    int seg_j0 = 0;                                    // first tile of the stream this CTA saw
+    long long seg_t = 0;                               // position of the stream's tile 0 in the sequence
+    int sidx = 0;                                      // streams handed to the finishing warp so far
+
+    for (int it = 0; it < n_tiles; ++it) {
+        const int s = it % STAGES;
+        if (!*dead && !ptx::mbar_wait(bars + 16 * s, (it / STAGES) & 1)) {
+            *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+        }
+        if (it == 0 || w.j == 0) {
+            // a new stream starts: fetch the group's query rows, clear the running state
+            seg_j0 = w.j;
+            seg_t = t0 + it - w.j;
+            const uint32_t qs = q_base + s * QB;
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const int head = nt * 8 + g;
+                    uint32_t v0 = 0u, v1 = 0u;
+                    if (head < G) {
+                        v0 = ptx::lds32(qs + (head * DH + ks * 16 + 2 * c) * 2);
+                        v1 = ptx::lds32(qs + (head * DH + ks * 16 + 8 + 2 * c) * 2);
+                    }
+                    qb[nt][ks][0] = v0; qb[nt][ks][1] = v1;
+                }
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt) {
+                m[nt][0] = m[nt][1] = -CUDART_INF_F;
+                l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < DH / 16; ++mt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) o[nt][mt][e] = 0.f;
+            }
+        }
+        {
+            const uint32_t kt = base + s * R::STAGE_BYTES, vt = kt + R::TILE_BYTES;
+            const int v = min(BN, w.len - w.j * BN) - 16 * warp;
+            if (v > 0) process_block<DH, NT8>(kt, vt, warp, min(v, 16), qb, o, m, l, p.scale_log2, lane);
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bars + 16 * s + 8);
+
+        const bool stream_end = (w.j == w.nt - 1);
+        if (stream_end || it == n_tiles - 1) {
+            // ---- hand this warp's state to the finishing warp through `red`
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    l[nt][j] += __shfl_xor_sync(0xffffffffu, l[nt][j], 4);
+                    l[nt][j] += __shfl_xor_sync(0xffffffffu, l[nt][j], 8);
+                    l[nt][j] += __shfl_xor_sync(0xffffffffu, l[nt][j], 16);
+                }
+            if (!*dead && !ptx::mbar_wait(red_empty, (sidx & 1) ^ 1)) {
+                *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT8; ++nt)
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int head = nt * 8 + 2 * c + j;
+                    if (head < G) {
+                        float *dst = red + ((size_t)warp * G + head) * (DH + 2);
+#pragma unroll
+                        for (int mt = 0; mt < DH / 16; ++mt) {
+                            dst[mt * 16 + g] = o[nt][mt][j];
+                            dst[mt * 16 + 8 + g] = o[nt][mt][2 + j];
+                        }
+                        if (g == 0) { dst[DH] = m[nt][j]; dst[DH + 1] = l[nt][j]; }
+                    }
+                }
+            if (warp == 0 && lane == 0) {
+                // CTAs that hold a piece of this stream: first and last
+                const long long te = seg_t + w.nt;
+                meta[0] = w.u; meta[1] = w.h;
+                meta[2] = ((stream_end && seg_j0 == 0) ? 1 : 0) | (it == n_tiles - 1 ? 2 : 0);
+                meta[3] = (int)(((seg_t + 1) * n_cta - 1) / T);
+                meta[4] = (int)((te * n_cta - 1) / T);
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(red_full);
+            ++sidx;
+        }
+        w.next(p);
+    }
+}
+
+template <int DH, int NT8>
+cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
+    const int G = p.Hq / p.Hkv;
+    const size_t smem = smem_bytes<DH>(G);
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(coarse_attn_kernel<DH, NT8>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        smem_set = smem;
+    }
+    const CUtensorMap *t;
+    CUtensorMap mk, mv;
+    if (!(t = ctx->tmaps.get(p.k, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BOX))) return cudaErrorInvalidValue;
+    mk = *t;
+    if (!(t = ctx->tmaps.get(p.v, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BOX))) return cudaErrorInvalidValue;
+    mv = *t;
+    const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
+    const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, ctx->max_ctas));
+    coarse_attn_kernel<DH, NT8><<<grid, THREADS, smem, st>>>(p, mk, mv);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int coarse_attn_ctas_per_sm() { return CTAS_PER_SM; }
+
+cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st, long long *launches) {
+    if (p.n_q == 0) return cudaSuccess;
+    if (p.splits_sh > 0) {
+        const cudaError_t e = launch_shared_prefix_attention(ctx, p, st, launches);
+        if (e != cudaSuccess) return e;
+    }
+    const int G = p.Hq / p.Hkv;
+    if (p.dh == 64) return G <= 8 ? run<64, 1>(ctx, p, st, launches) : run<64, 2>(ctx, p, st, launches);
+    return G <= 8 ? run<128, 1>(ctx, p, st, launches) : run<128, 2>(ctx, p, st, launches);
+}

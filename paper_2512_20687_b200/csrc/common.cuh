@@ -31,9 +31,11 @@ struct photon_ctx {
     int device;
     int sm_count;
     int max_splits;          // resolved upper bound on key ranges per query
-    float *partials;         // split-K workspace: [max_queries * Hq * max_splits * (dh + 2)] floats
+    float *partials;         // shared-prefix partials: [max_queries * Hq * max_splits * (dh + 2)] floats
     size_t partial_floats;
-    int32_t *tickets;        // one arrival counter per (query, kv head); zero between calls
+    float *cta_partials;     // partials of streams cut by a CTA boundary: [2 * max_ctas][16][dh + 2] floats
+    int max_ctas;            // grid of the persistent attention kernel
+    int32_t *tickets;        // one arrival counter per (unit, kv head); zero between calls
     size_t n_tickets;
     int32_t *status;         // device status word
     long long launches;
@@ -51,15 +53,17 @@ struct AttnParams {
     const bf16 *k, *v;
     const int32_t *len;
     int n_units, cap;
+    int max_len;             // host-side bound on len[] (sizes the grid)
     const bf16 *ks, *vs;
     const int32_t *sh_len, *sh_id;
     int n_shared, cap_sh;
     const int32_t *slot;
     int n_q, Hq, Hkv, dh;
-    int splits_own, splits_sh;
-    int ctas_own, upc;       // filled by the launcher: CTAs on own keys; units per CTA on shared keys
+    int splits_sh;           // key ranges of a shared prefix (0: no shared prefix in this call)
+    int upc;                 // filled by the launcher: units per CTA on shared keys
     float scale_log2;        // scale * log2(e): logits are kept in the base-2 domain
     float *partials;
+    float *cta_partials;
     int32_t *tickets;
     int32_t *status;
 };
@@ -79,6 +83,9 @@ cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hk
                              int n_rows, int32_t *status, cudaStream_t st, long long *launches);
 cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                              long long *launches);
+cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+                                           long long *launches);
+int coarse_attn_ctas_per_sm();
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,

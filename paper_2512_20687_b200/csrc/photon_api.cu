@@ -70,30 +70,25 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
     p.tickets = ctx->tickets;
     p.status = ctx->status;
 
-    const size_t per_part = size_t(n_q) * c.Hq * (c.dh + 2);
-    const int parts_allowed = (int)std::min<size_t>(ctx->partial_floats / per_part, 1 << 20);
-    const int streams = n_q * c.Hkv;
-    if (chunk) {
-        p.splits_own = 1; p.splits_sh = 0;
-    } else {
-        const int max_len = cache->max_len ? cache->max_len : cache->cap;
-        p.splits_own = choose_splits(ctx, streams, max_len, 128, ctx->max_splits);
-        p.splits_sh = 0;
+    p.cta_partials = ctx->cta_partials;
+    p.max_len = cache->max_len ? cache->max_len : cache->cap;
+    p.splits_sh = 0;
+    if (!chunk) {
+        if ((size_t)n_q * c.Hkv > ctx->n_tickets) return PHOTON_ERR_WORKSPACE;
         if (cache->k_shared) {
             p.ks = reinterpret_cast<const bf16 *>(cache->k_shared);
             p.vs = reinterpret_cast<const bf16 *>(cache->v_shared);
             p.sh_len = cache->shared_len; p.sh_id = cache->shared_id;
             p.n_shared = cache->n_shared; p.cap_sh = cache->cap_shared;
             const int ms = cache->max_shared_len ? cache->max_shared_len : cache->cap_shared;
-            p.splits_sh = choose_splits(ctx, streams, ms, 128, ctx->max_splits);
-        }
-        while (p.splits_own + p.splits_sh > std::min(parts_allowed, ctx->max_splits) &&
-               (p.splits_own > 1 || p.splits_sh > 1)) {
-            if (p.splits_own >= p.splits_sh && p.splits_own > 1) --p.splits_own;
-            else --p.splits_sh;
+            const size_t per_part = size_t(n_q) * c.Hq * (c.dh + 2);
+            const int allowed = (int)std::min<size_t>(ctx->partial_floats / per_part, (size_t)ctx->max_splits);
+            if (allowed < 1) return PHOTON_ERR_WORKSPACE;
+            const int G = c.Hq / c.Hkv;
+            const int groups = ceil_div(n_q, 4 * (16 / G));       // units are taken in groups by the prefix kernel
+            p.splits_sh = choose_splits(ctx, groups * c.Hkv, ms, 128, allowed);
         }
     }
-    if (p.splits_own + p.splits_sh > parts_allowed) return PHOTON_ERR_WORKSPACE;
     const cudaError_t e = chunk ? launch_chunk_attention(ctx, p, st, &ctx->launches)
                                 : launch_attention(ctx, p, st, &ctx->launches);
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
@@ -134,12 +129,14 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
     const size_t per_part = size_t(c.max_queries) * c.Hq * (c.dh + 2);
     ctx->partial_floats = std::max(per_part, std::min(per_part * ctx->max_splits, kMaxPartialFloats));
     ctx->n_tickets = size_t(c.max_queries) * c.Hkv;
+    ctx->max_ctas = ctx->sm_count * coarse_attn_ctas_per_sm();
     if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&ctx->cta_partials, size_t(2) * ctx->max_ctas * 16 * (c.dh + 2) * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->tickets, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
         cudaMalloc(&ctx->status, sizeof(int32_t)) != cudaSuccess ||
         cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
         cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) {
-        cudaFree(ctx->partials); cudaFree(ctx->tickets); cudaFree(ctx->status);
+        cudaFree(ctx->partials); cudaFree(ctx->cta_partials); cudaFree(ctx->tickets); cudaFree(ctx->status);
         cudaGetLastError();
         delete ctx;
         return PHOTON_ERR_CUDA;
@@ -151,6 +148,7 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
 photon_status photon_destroy(photon_ctx *ctx) {
     if (!ctx) return PHOTON_ERR_INVALID_ARG;
     cudaFree(ctx->partials);
+    cudaFree(ctx->cta_partials);
     cudaFree(ctx->tickets);
     cudaFree(ctx->status);
     delete ctx;
@@ -273,6 +271,13 @@ photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t c
 }
 
 int64_t photon_launch_count(const photon_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n) {
+    if (!ctx || n < 0) return PHOTON_ERR_INVALID_ARG;
+    const int full = ctx->sm_count * coarse_attn_ctas_per_sm();
+    ctx->max_ctas = (n == 0 || n > full) ? full : n;
+    return PHOTON_OK;
+}
 
 const char *photon_status_str(photon_status s) {
     switch (s) {

@@ -1,21 +1,15 @@
-// Decode attention of the coarsest stream (attention half of STEP, Eq. 12) and
-// of a token-level cache: one query position per unit over the valid rows of
-// its KV cache, optionally preceded by a shared prefix that is streamed once
-// for all the branches that use it.
+// Shared-prefix phase of the coarse decode attention (Section 1: long-context,
+// multi-query serving): many units (query branches) attend the same stored
+// prefix, which is therefore read once for a whole group of units.
 //
-// Keys are cut into ranges ("parts").  A CTA streams the K/V tiles of one part
-// through a TMA-fed, 128-byte-swizzled shared-memory ring and evaluates the
-// grouped-query QK^T and PV products on tensor cores with fp32 online softmax
-// in the base-2 domain.  Each part leaves an unnormalised partial (acc, m, l);
-// a merge pass combines the parts of a query head by log-sum-exp.
-//
-//   own part:    CTA = (unit, kv head, key range).  The M tile is the G query
-//                heads of the group; the four consumer warps take different
-//                16-key slices of every 64-key tile and merge at the end.
-//   shared part: CTA = (group of units, kv head, key range of the prefix).
-//                Each consumer warp owns 16 query rows (16/G units x G heads)
-//                and runs them against every key of the tile, so the prefix
-//                leaves HBM once and L2 feeds the other groups.
+// CTA = (group of units, KV head, key range of the prefix).  The K/V tiles of
+// the range stream through a TMA-fed, 128-byte-swizzled shared-memory ring; each
+// of the four consumer warps owns 16 query rows (16/G units x G heads) and runs
+// them against every key of a tile on tensor cores with an fp32 online softmax
+// in the base-2 domain, so the prefix leaves HBM once and L2 feeds the other
+// groups.  Every (query head, key range) leaves an unnormalised partial
+// (acc, m, l) at partials[(query head) * splits_sh + range]; the kernel that
+// streams the units' own keys folds these partials into its result.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -146,9 +140,8 @@ __device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, 
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 2)
-attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ks,
-                const __grid_constant__ CUtensorMap tm_vs) {
+shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_ks,
+                     const __grid_constant__ CUtensorMap tm_vs) {
     using T = Tile<DH>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -160,7 +153,7 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
     const int G = p.Hq / p.Hkv;
-    const int parts = p.splits_sh + p.splits_own;
+    const int parts = p.splits_sh;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < T::STAGES; ++s) {
@@ -169,34 +162,23 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         }
         *dead = 0;
         ptx::mbar_fence_init();
-        ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
+        ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
 
-    const bool own = (int)blockIdx.x < p.ctas_own;
-    int part, h, unit0;          // unit0: the unit (own) or the first unit of the group (shared)
-    if (own) {
-        part = blockIdx.x % p.splits_own;
-        h = (blockIdx.x / p.splits_own) % p.Hkv;
-        unit0 = blockIdx.x / (p.splits_own * p.Hkv);
-    } else {
-        const int b2 = blockIdx.x - p.ctas_own;
-        part = b2 % p.splits_sh;
-        h = (b2 / p.splits_sh) % p.Hkv;
-        unit0 = (b2 / (p.splits_sh * p.Hkv)) * p.upc;
-    }
-    const int upw = 16 / G;                 // units per warp in shared mode
+    const int part = blockIdx.x % p.splits_sh;
+    const int h = (blockIdx.x / p.splits_sh) % p.Hkv;
+    const int unit0 = (blockIdx.x / (p.splits_sh * p.Hkv)) * p.upc;      // first unit of the group
+    const int upw = 16 / G;                 // units per warp
 
-    if (!own) {
-        // shared-segment id of every unit of the group: >= 0 valid, -1 none / out of range / bad
-        for (int j = threadIdx.x; j < p.upc; j += THREADS) {
-            const int i = unit0 + j;
-            int s = -1;
-            if (i < p.n_q) {
-                s = p.sh_id[i];
-                if (s >= p.n_shared || s < 0) s = -1;
-            }
-            sid[j] = s;
+    // shared-segment id of every unit of the group: >= 0 valid, -1 none / out of range / bad
+    for (int j = threadIdx.x; j < p.upc; j += THREADS) {
+        const int i = unit0 + j;
+        int s = -1;
+        if (i < p.n_q) {
+            s = p.sh_id[i];
+            if (s >= p.n_shared || s < 0) s = -1;
         }
+        sid[j] = s;
     }
     __syncthreads();
 
@@ -204,16 +186,13 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     uint32_t qa[DH / 16][4];
     float o[DH / 8][4];
     float m[2] = {-CUDART_INF_F, -CUDART_INF_F}, l[2] = {0.f, 0.f};
-    bool hi_rows = own ? (G > 8) : true;
     int row_unit[2] = {-1, -1};             // query index of rows g and g+8 (-1: padding row)
     int row_head[2] = {0, 0};
     if (warp < NW) {
 #pragma unroll
         for (int rs = 0; rs < 2; ++rs) {
             const int r = g + 8 * rs;
-            if (own) {
-                if (r < G) { row_unit[rs] = unit0; row_head[rs] = h * G + r; }
-            } else if (r < upw * G) {
+            if (r < upw * G) {
                 const int i = unit0 + warp * upw + r / G;
                 if (i < p.n_q) { row_unit[rs] = i; row_head[rs] = h * G + r % G; }
             }
@@ -270,16 +249,9 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 }
                 const uint32_t kt = base + s * T::STAGE_BYTES, vt = kt + T::TILE_BYTES;
                 const int nvalid = min(BN, (r1 - r0) - t * BN);
-                if (own) {
-                    const int v = nvalid - 16 * warp;
-                    if (v > 0)
-                        process_block<DH>(kt, vt, warp, min(v, 16), qa, o, m, l, p.scale_log2, lane, act0,
-                                          act1, hi_rows);
-                } else {
-                    for (int kb = 0; kb * 16 < nvalid; ++kb)
-                        process_block<DH>(kt, vt, kb, min(16, nvalid - kb * 16), qa, o, m, l, p.scale_log2,
-                                          lane, act0, act1, true);
-                }
+                for (int kb = 0; kb * 16 < nvalid; ++kb)
+                    process_block<DH>(kt, vt, kb, min(16, nvalid - kb * 16), qa, o, m, l, p.scale_log2, lane,
+                                      act0, act1, true);
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bars + 16 * s + 8);
             }
@@ -287,69 +259,7 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         tg += ntiles;
     };
 
-    if (own) {
-        const int u = p.slot ? p.slot[unit0] : unit0;
-        bool bad = (u < 0 || u >= p.n_units);
-        if (!bad && p.sh_id && p.splits_sh > 0 && p.sh_id[u] >= p.n_shared) bad = true;
-        int r0 = 0, r1 = 0;
-        if (bad) {
-            if (threadIdx.x == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
-        } else {
-            part_range(max(0, min(p.len[u], p.cap)), p.splits_own, part, r0, r1);
-        }
-        run_pass(&tm_k, &tm_v, ((long long)(bad ? 0 : u) * p.Hkv + h) * p.cap, r0, r1, g < G, g + 8 < G);
-
-        // ---- merge the four warps' partial states through shared memory
-        __syncthreads();                        // every tile has landed and been consumed
-        float *red = reinterpret_cast<float *>(gen_base);          // [NW][16][DH + 2]
-        if (warp < NW) {
-#pragma unroll
-            for (int rs = 0; rs < 2; ++rs) {
-                l[rs] += __shfl_xor_sync(0xffffffffu, l[rs], 1);
-                l[rs] += __shfl_xor_sync(0xffffffffu, l[rs], 2);
-            }
-#pragma unroll
-            for (int rs = 0; rs < 2; ++rs) {
-                const int r = g + 8 * rs;
-                if (r < G) {
-                    float *dst = red + ((size_t)warp * 16 + r) * (DH + 2);
-#pragma unroll
-                    for (int nt = 0; nt < DH / 8; ++nt) {
-                        dst[nt * 8 + 2 * c] = o[nt][2 * rs];
-                        dst[nt * 8 + 2 * c + 1] = o[nt][2 * rs + 1];
-                    }
-                    if (c == 0) { dst[DH] = m[rs]; dst[DH + 1] = l[rs]; }
-                }
-            }
-        }
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < G * DH; idx += THREADS) {
-            const int r = idx / DH, d = idx % DH;
-            float M = -CUDART_INF_F;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) M = fmaxf(M, red[((size_t)w * 16 + r) * (DH + 2) + DH]);
-            float L = 0.f, acc = 0.f;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float *src = red + ((size_t)w * 16 + r) * (DH + 2);
-                if (src[DH + 1] > 0.f) {
-                    const float f = exp2f(src[DH] - M);
-                    L += src[DH + 1] * f;
-                    acc += src[d] * f;
-                }
-            }
-            const size_t qh = (size_t)unit0 * p.Hq + h * G + r;
-            if (parts == 1) {
-                p.out[qh * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-                if (d == 0 && p.lse)
-                    p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
-            } else {
-                float *dst = p.partials + (qh * parts + p.splits_sh + part) * (DH + 2);
-                dst[d] = acc;
-                if (d == 0) { dst[DH] = M; dst[DH + 1] = L; }
-            }
-        }
-    } else {
+    {
         // ---- shared prefix: one pass per distinct segment id present in the group
         int last = -1;
         for (;;) {
@@ -388,80 +298,33 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     }
 }
 
-// One warp per (query, query head): log-sum-exp combination of its parts.
-template <int DH>
-__global__ void __launch_bounds__(128)
-attn_merge_kernel(const AttnParams p) {
-    constexpr int E = DH / 32;
-    const int parts = p.splits_sh + p.splits_own;
-    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (wid >= (long long)p.n_q * p.Hq) return;
-    const int lane = threadIdx.x & 31;
-    const float *src = p.partials + (size_t)wid * parts * (DH + 2);
-    float M = -CUDART_INF_F;
-    for (int j = 0; j < parts; ++j)
-        if (src[(size_t)j * (DH + 2) + DH + 1] > 0.f) M = fmaxf(M, src[(size_t)j * (DH + 2) + DH]);
-    float L = 0.f, o[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) o[e] = 0.f;
-    for (int j = 0; j < parts; ++j) {
-        const float *pj = src + (size_t)j * (DH + 2);
-        const float lj = pj[DH + 1];
-        if (!(lj > 0.f)) continue;                  // empty part
-        const float w = exp2f(pj[DH] - M);
-        L += lj * w;
-#pragma unroll
-        for (int e = 0; e < E; ++e) o[e] += w * pj[lane * E + e];
-    }
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    bf16 *op = p.out + (size_t)wid * DH + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) op[e] = __float2bfloat16_rn(o[e] * inv);
-    if (p.lse && lane == 0)
-        p.lse[wid] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
-}
-
 template <int DH>
 cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
-    if (p.n_q == 0) return cudaSuccess;
     using T = Tile<DH>;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(shared_prefix_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              T::SMEM);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     const int G = p.Hq / p.Hkv;
     p.upc = NW * (16 / G);
-    p.ctas_own = p.n_q * p.Hkv * p.splits_own;
     const int groups = (p.n_q + p.upc - 1) / p.upc;
-    const int ctas_sh = p.splits_sh ? groups * p.Hkv * p.splits_sh : 0;
     const CUtensorMap *t;
-    CUtensorMap mk, mv, mks, mvs;
-    if (!(t = ctx->tmaps.get(p.k, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BN))) return cudaErrorInvalidValue;
-    mk = *t;
-    if (!(t = ctx->tmaps.get(p.v, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BN))) return cudaErrorInvalidValue;
-    mv = *t;
-    mks = mk; mvs = mv;
-    if (p.splits_sh) {
-        if (!(t = ctx->tmaps.get(p.ks, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
-        mks = *t;
-        if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
-        mvs = *t;
-    }
-    attn_mma_kernel<DH><<<p.ctas_own + ctas_sh, THREADS, T::SMEM, st>>>(p, mk, mv, mks, mvs);
+    CUtensorMap mks, mvs;
+    if (!(t = ctx->tmaps.get(p.ks, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
+    mks = *t;
+    if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
+    mvs = *t;
+    shared_prefix_kernel<DH><<<groups * p.Hkv * p.splits_sh, THREADS, T::SMEM, st>>>(p, mks, mvs);
     ++*launches;
-    if (p.splits_sh + p.splits_own > 1) {
-        const long long mw = (long long)p.n_q * p.Hq;
-        attn_merge_kernel<DH><<<(unsigned)((mw + 3) / 4), 128, 0, st>>>(p);
-        ++*launches;
-    }
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st, long long *launches) {
+cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
+                                           long long *launches) {
     return p.dh == 64 ? run<64>(ctx, p, st, launches) : run<128>(ctx, p, st, launches);
 }

@@ -84,10 +84,10 @@ def test_coarse_attention_matches_oracle_at_full_size(oracle, idx):
     assert np.abs(lse - want_lse).max() < 2e-3
 
 
-@pytest.mark.parametrize("max_splits", [1, 2, 3, 7, 32])
-def test_split_count_does_not_change_the_result(oracle, max_splits):
-    """Ragged lengths incl. 0 and 1, more splits than keys, and splits that
-    receive no keys at all."""
+@pytest.mark.parametrize("n_ctas", [1, 2, 3, 7, 37, 101, 0])
+def test_grid_size_and_cut_points_do_not_change_the_result(oracle, n_ctas):
+    """Ragged lengths incl. 0 and 1; the grid size moves the points where caches
+    are cut and merged (one CTA: no cut at all; many: most units cut, some CTAs idle)."""
     cfg = cfg_small(1, B=9, S=701)
     co = wl.coarse_inputs(cfg, poison=True)
     lens = np.array([700, 0, 1, 2, 127, 128, 129, 513, 699], np.int32)
@@ -97,13 +97,34 @@ def test_split_count_does_not_change_the_result(oracle, max_splits):
     co["len"] = lens
     scale = cfg.dh ** -0.5
     want, want_lse = oracle.attention(co["q"], co["k"], co["v"], lens, scale, n_threads=NT)
-    with Ctx(cfg, max_splits=max_splits) as c:
-        got, lse, _ = run_coarse(c, co, scale)
+    with Ctx(cfg) as c:
+        ph.photon_set_attention_ctas(c.h, n_ctas)
+        got, lse, bits1 = run_coarse(c, co, scale)
+        _, _, bits2 = run_coarse(c, co, scale)
         assert c.status() == 0
-    assert_close(got, want, f"splits<={max_splits}")
+    assert np.array_equal(bits1, bits2)           # tickets are back at zero, merge order is fixed
+    assert_close(got, want, f"ctas={n_ctas}")
     assert np.all(got[1] == 0) and np.all(np.isneginf(lse[1]))
     fin = np.isfinite(want_lse)
     assert np.abs(lse[fin] - want_lse[fin]).max() < 2e-3
+
+
+@pytest.mark.parametrize("G,dh", [(1, 64), (2, 64), (8, 128), (16, 64), (16, 128)])
+def test_coarse_attention_other_group_sizes(oracle, G, dh):
+    Hkv = 2
+    cfg = cfg_small(1, B=5, S=300, Hq=G * Hkv, Hkv=Hkv, dh=dh, D=G * Hkv * dh)
+    co = wl.coarse_inputs(cfg, poison=True)
+    co["len"] = np.array([299, 64, 65, 7, 200], np.int32)
+    for u, n in enumerate(co["len"]):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0x7FC1
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, f"G={G} dh={dh}")
+    assert np.abs(lse - want_lse).max() < 2e-3
 
 
 def test_shared_prefix_variants(oracle):
@@ -150,6 +171,9 @@ def test_bad_shared_id_is_flagged_and_zeroed(oracle):
 
 
 def test_attention_is_deterministic_and_batch_permutation_equivariant():
+    """Repeated calls are bit-identical.  Permuting the batch permutes the result; because the
+    points where a cache is cut depend on its place in the batch, equality is up to the rounding
+    of the merge (well inside one bf16 step of an O(1) value), not bit for bit."""
     cfg = cfg_small(1, B=24, S=333)
     co = wl.coarse_inputs(cfg)
     co["len"] = wl.uniform_int(5, "lens", cfg.B, 0, 333)
@@ -160,7 +184,9 @@ def test_attention_is_deterministic_and_batch_permutation_equivariant():
         _, _, b1 = run_coarse(c, co, scale)
         _, _, b2 = run_coarse(c, co, scale)
         _, _, b3 = run_coarse(c, cp, scale)
-    assert np.array_equal(b1, b2) and np.array_equal(b3, b1[perm])
+    assert np.array_equal(b1, b2)
+    d = np.abs(wl.bf16_bits_to_f64(b3) - wl.bf16_bits_to_f64(b1[perm]))
+    assert d.max() <= 2.0 ** -7 and (d > 0).mean() < 0.05
 
 
 def test_flat_attention_on_a_token_level_cache(oracle):
