@@ -47,11 +47,14 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parts", action="store_true")
     ap.add_argument("--max-splits", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0,
+                    help="shrink the workload to this many sequences (for profiler captures of a small case)")
     return ap.parse_args()
 
 
 def workload_desc(cfg) -> dict:
-    d = {"workload": f"config {cfg.index} ({cfg.name}): batch {cfg.B}, context {cfg.context} tokens -> "
+    full = wl.CONFIGS[cfg.index].B
+    d = {"workload": f"config {cfg.index} ({cfg.name}{'' if cfg.B == full else f', REDUCED from batch {full}'}): batch {cfg.B}, context {cfg.context} tokens -> "
                      f"{cfg.S} coarse latents, {cfg.Hq}q/{cfg.Hkv}kv heads x {cfg.dh}, d_model {cfg.D}, "
                      f"converter {cfg.D}->{cfg.P}x{cfg.D}, chunk attention P={cfg.P} C={cfg.C}, "
                      f"{cfg.chunks_per_seq} in-flight chunks per sequence",
@@ -457,6 +460,8 @@ def run_gpu(args, cfg) -> None:
 def main():
     args = parse()
     cfg = wl.CONFIGS[args.config]
+    if args.batch and args.batch < cfg.B:
+        cfg = wl.scaled(cfg, B=args.batch, tokens_per_step=cfg.tokens_per_step * args.batch // cfg.B)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
