@@ -186,6 +186,30 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, 
  * whole device; the only call that does. */
 photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear);
 
+/* The paper has no counterpart to this call: it exists for hosts that must not
+ * allocate device memory (a serving process whose memory pool owns the whole
+ * device, a thread that may not take the allocator's locks or its implicit
+ * synchronisation, a process that has promised a fixed footprint), where
+ * photon_create is unusable.  It computes what photon_coarse_attn computes,
+ * for a cache without shared prefixes, and needs no context: the kernel's
+ * workspace is an array inside the library image (about 5.4 MB per GPU that
+ * loads the library, held until the process exits).  Nothing here calls
+ * cudaMalloc, cudaFree or an allocating library routine.
+ *   cfg         only Hq, Hkv and dh are read.
+ *   cache, q, out, lse, scale, stream   as for photon_coarse_attn.
+ *   dev_status  device int32 the kernel ORs PHOTON_DEV_* bits into, or NULL
+ *               (then they go to a word inside the array that nobody reads).
+ * Limit: n_units * Hkv <= PHOTON_NOALLOC_MAX_STREAMS, else
+ * PHOTON_ERR_WORKSPACE and nothing is launched; a shared prefix gives
+ * PHOTON_ERR_UNSUPPORTED.  The first call on a device looks up the array's
+ * device address; make that call before capturing a stream.  All calls on a
+ * device share the array and the call clears the part that must start at
+ * zero, so calls that overlap on one GPU race: keep them in stream order. */
+#define PHOTON_NOALLOC_MAX_STREAMS 16384
+photon_status photon_coarse_attn_noalloc(const photon_config *cfg, const photon_kv *cache,
+                                         const photon_bf16 *q, photon_bf16 *out, float *lse, float scale,
+                                         int32_t *dev_status, photon_stream stream);
+
 /* Caps the persistent grid of photon_coarse_attn / photon_flat_attn at n CTAs
  * (0 or more than the device holds: the default, two per SM).  The keys of a
  * call are dealt out evenly over the grid, so n also moves the points where a

@@ -78,6 +78,9 @@ def load() -> ctypes.CDLL:
         f = getattr(lib, name)
         f.restype = st
         f.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p, c_float, c_void_p]
+    lib.photon_coarse_attn_noalloc.restype = st
+    lib.photon_coarse_attn_noalloc.argtypes = [POINTER(photon_config), POINTER(photon_kv), c_void_p, c_void_p,
+                                               c_void_p, c_float, c_void_p, c_void_p]
     lib.photon_converter.restype = st
     lib.photon_converter.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
                                      c_int32, c_void_p]
@@ -166,6 +169,16 @@ def photon_kv_append(ctx, cache: photon_kv, k_new, v_new, unit_ids=None, n=None,
 def photon_coarse_attn(ctx, cache: photon_kv, q, out, lse=None, scale=1.0, stream=None) -> None:
     _check(load().photon_coarse_attn(ctx, byref(cache), _ptr(q), _ptr(out), _ptr(lse),
                                      c_float(scale), _stream(stream)), "photon_coarse_attn")
+
+
+def photon_coarse_attn_noalloc(Hq, Hkv, dh, cache: photon_kv, q, out, lse=None, scale=1.0, dev_status=None,
+                               stream=None) -> None:
+    """photon_coarse_attn without a context and without any device allocation (see photon.h);
+    dev_status: optional device int32 tensor that receives PHOTON_DEV_* bits."""
+    cfg = photon_config(Hq, Hkv, dh, Hq * dh, 1, 1, 1, 0)
+    _check(load().photon_coarse_attn_noalloc(byref(cfg), byref(cache), _ptr(q), _ptr(out), _ptr(lse),
+                                             c_float(scale), _ptr(dev_status), _stream(stream)),
+           "photon_coarse_attn_noalloc")
 
 
 def photon_flat_attn(ctx, cache: photon_kv, q, out, lse=None, scale=1.0, stream=None) -> None:
