@@ -73,6 +73,7 @@ struct ConvParams {
     bf16 *U;
     int B, D, N;             // N = P * D
     int w_out_major;
+    int x_rows;              // filled by the launcher: x rows fetched per K block (16, 32, 64 or 128)
     int32_t *status;
 };
 

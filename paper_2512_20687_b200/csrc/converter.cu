@@ -3,12 +3,16 @@
 //
 // A dense contraction on the 5th-generation tensor cores.  A CTA owns a
 // [128 batch rows x NT output columns] tile of U: the batch rows are the M
-// side (rows past the batch are zero-filled by TMA and cost no bandwidth), a
-// slab of NT weight columns is the N side, and the accumulator lives in TMEM.
-// One thread feeds a ring of TMA loads (x tile and weight tile per 64-wide K
-// block), one thread issues tcgen05.mma on the swizzled tiles, four warps read
-// the accumulator back with tcgen05.ld, add the bias, round once to bf16 and
-// store.  Every weight element leaves HBM exactly once; at small batch the
+// side, a slab of NT weight columns is the N side, and the accumulator lives
+// in TMEM.  Only as many x rows as the batch needs (rounded up to 16, 32, 64 or
+// 128) are fetched per K block; the MMA still spans 128 rows, and the rows it
+// reads beyond the fetched ones are whatever shared memory holds: they only
+// reach accumulator rows that are never read back.  A smaller x box makes a
+// stage smaller, so a small batch gets a deeper ring of weight tiles in flight.
+// One warp feeds a ring of TMA loads (x atoms and weight atoms for 128 K
+// elements per stage), one warp issues tcgen05.mma on the swizzled atoms (in both
+// an elected lane does the issuing), four warps read the accumulator back with
+// tcgen05.ld, add the bias, round once to bf16 and store.  Every weight element leaves HBM exactly once; at small batch the
 // kernel is bound by that stream, at large batch by the tensor pipe.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -16,18 +20,27 @@
 namespace {
 
 constexpr int BM = 128;                 // batch rows per CTA (UMMA M)
-constexpr int BK = 64;                  // K elements per stage (one 128-byte swizzle row)
+constexpr int BK = 64;                  // K elements per swizzle atom (one 128-byte row)
+constexpr int KA = 2;                   // atoms per stage: one barrier round trip per 128 K elements
 constexpr int CONV_THREADS = 192;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+
+constexpr int MAX_STAGES = 12;
+constexpr int RING_BYTES = 192 * 1024;
 
 template <int NT>
 struct ConvTile {
-    static constexpr int A_BYTES = BM * BK * 2;           // 16 KiB
-    static constexpr int B_BYTES = NT * BK * 2;           // 8 / 16 KiB
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = NT == 64 ? 8 : 6;       // 192 KiB of tiles either way
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 + 256;
+    static constexpr int B_BYTES = NT * BK * 2;           // weight atom: 8 / 16 KiB
+    // slack after the ring: the MMA reads 128 rows from every x atom, also past a short x box
+    static constexpr int SMEM = RING_BYTES + BM * BK * 2 + 1024 + 512;
 };
 
+__host__ __device__ inline int conv_stages(int a_bytes, int b_bytes) {
+    const int s = RING_BYTES / (KA * (a_bytes + b_bytes));
+    return s < MAX_STAGES ? s : MAX_STAGES;
+}
+
+// The loops of the TMA warp and of the MMA warp are run by the whole warp (so that their
+// address arithmetic stays warp-uniform); one elected lane issues the asynchronous operations.
 template <int NT, bool W_IN_MAJOR>
 __global__ void __launch_bounds__(CONV_THREADS, 1)
 converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
@@ -36,22 +49,25 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
-    const uint32_t bars = base + T::STAGES * T::STAGE_BYTES;     // full[s] +16s, empty[s] +16s+8
-    const uint32_t bar_acc = bars + 16 * T::STAGES;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen + T::STAGES * T::STAGE_BYTES + 16 * T::STAGES + 16);
-    volatile int *dead = reinterpret_cast<volatile int *>(gen + T::STAGES * T::STAGE_BYTES + 16 * T::STAGES + 32);
+    const int a_bytes = p.x_rows * BK * 2;                       // x atom of this launch
+    const int stage_bytes = KA * (a_bytes + T::B_BYTES);         // [x atoms][weight atoms]
+    const int n_stages = conv_stages(a_bytes, T::B_BYTES);
+    constexpr int TAIL = RING_BYTES + BM * BK * 2;
+    const uint32_t bars = base + TAIL;                           // full[s] +16s, empty[s] +16s+8
+    const uint32_t bar_acc = bars + 16 * MAX_STAGES;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen + TAIL + 16 * MAX_STAGES + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * NT, m0 = blockIdx.y * BM;
-    const int nkb = p.D / BK;
+    const int n_atoms = p.D / BK;
+    const int n_steps = (n_atoms + KA - 1) / KA;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < T::STAGES; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             ptx::mbar_init(bars + 16 * s, 1);
             ptx::mbar_init(bars + 16 * s + 8, 1);
         }
         ptx::mbar_init(bar_acc, 1);
-        *dead = 0;
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_x); ptx::prefetch_tmap(&tm_w);
     }
@@ -62,58 +78,73 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % T::STAGES;
-                if (*dead) break;
-                if (!ptx::mbar_wait(bars + 16 * s + 8, ((kb / T::STAGES) & 1) ^ 1)) {
-                    *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
-                }
-                const uint32_t full = bars + 16 * s;
-                const uint32_t a_dst = base + s * T::STAGE_BYTES, b_dst = a_dst + T::A_BYTES;
-                ptx::mbar_arrive_expect_tx(full, T::STAGE_BYTES);
-                ptx::tma_load_2d(a_dst, &tm_x, kb * BK, m0, full);               // x[m0.., k..]
-                if (!W_IN_MAJOR) {
-                    ptx::tma_load_2d(b_dst, &tm_w, kb * BK, n0, full);           // W[n0.., k..]  (K-major)
-                } else {
+        int s = 0;
+        uint32_t phase = 0;
+        for (int st = 0; st < n_steps; ++st) {
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(bars + 16 * s + 8, phase ^ 1))) {
+                if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+                break;
+            }
+            const int atoms = min(KA, n_atoms - st * KA);
+            const uint32_t full = bars + 16 * s;
+            const uint32_t a_dst = base + s * stage_bytes, b_dst = a_dst + KA * a_bytes;
+            if (ptx::elect_one()) {
+                ptx::mbar_arrive_expect_tx(full, atoms * (a_bytes + T::B_BYTES));
+                for (int j = 0; j < atoms; ++j) {
+                    const int k0 = (st * KA + j) * BK;
+                    ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, k0, m0, full);              // x[m0.., k0..]
+                    if (!W_IN_MAJOR) {
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);       // W[n0.., k0..]  (K-major)
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < NT / 64; ++j)                            // W[k.., n0+64j..] (N-major)
-                        ptx::tma_load_2d(b_dst + j * (BK * 128), &tm_w, n0 + 64 * j, kb * BK, full);
+                        for (int jj = 0; jj < NT / 64; ++jj)                                 // W[k0.., n0+64jj..] (N-major)
+                            ptx::tma_load_2d(b_dst + j * T::B_BYTES + jj * (BK * 128), &tm_w, n0 + 64 * jj, k0, full);
+                    }
                 }
             }
+            __syncwarp();
+            if (++s == n_stages) { s = 0; phase ^= 1; }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::umma_idesc_bf16(BM, NT, false, W_IN_MAJOR);
-            bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % T::STAGES;
-                if (*dead || !ptx::mbar_wait(bars + 16 * s, (kb / T::STAGES) & 1)) {
-                    if (!*dead) { *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); }
-                    ok = false; break;
-                }
-                ptx::tc_fence_after();
-                const uint32_t a_addr = base + s * T::STAGE_BYTES, b_addr = a_addr + T::A_BYTES;
-                const uint64_t adesc = ptx::umma_desc_sw128(a_addr, 0, 1024);
-                const uint64_t bdesc = W_IN_MAJOR ? ptx::umma_desc_sw128(b_addr, BK * 128, 1024)
-                                                  : ptx::umma_desc_sw128(b_addr, 0, 1024);
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16(BM, NT, false, W_IN_MAJOR);
+        int s = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int st = 0; st < n_steps; ++st) {
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(bars + 16 * s, phase))) {
+                if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after();
+            const int atoms = min(KA, n_atoms - st * KA);
+            const uint32_t a_addr = base + s * stage_bytes, b_addr = a_addr + KA * a_bytes;
+            if (ptx::elect_one()) {
+                for (int j = 0; j < atoms; ++j) {
+                    const uint64_t adesc = ptx::umma_desc_sw128(a_addr + j * a_bytes, 0, 1024);
+                    const uint64_t bdesc = W_IN_MAJOR ? ptx::umma_desc_sw128(b_addr + j * T::B_BYTES, BK * 128, 1024)
+                                                      : ptx::umma_desc_sw128(b_addr + j * T::B_BYTES, 0, 1024);
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k) {
-                    // advance 16 K elements: 32 bytes inside the swizzled row (K-major),
-                    // 16 rows of 128 bytes (N-major); the address field counts 16-byte units
-                    const uint64_t a_k = adesc + (uint64_t)(k * 2);
-                    const uint64_t b_k = bdesc + (uint64_t)(W_IN_MAJOR ? k * 128 : k * 2);
-                    ptx::umma_bf16(tmem, a_k, b_k, idesc, (kb | k) != 0);
+                    for (int k = 0; k < BK / 16; ++k) {
+                        // advance 16 K elements: 32 bytes inside the swizzled row (K-major),
+                        // 16 rows of 128 bytes (N-major); the address field counts 16-byte units
+                        const uint64_t a_k = adesc + (uint64_t)(k * 2);
+                        const uint64_t b_k = bdesc + (uint64_t)(W_IN_MAJOR ? k * 128 : k * 2);
+                        ptx::umma_bf16(tmem, a_k, b_k, idesc, (st | j | k) != 0);
+                    }
                 }
                 ptx::umma_commit(bars + 16 * s + 8);       // frees the stage once these MMAs have read it
+                if (st == n_steps - 1) ptx::umma_commit(bar_acc);     // accumulator complete
             }
-            ptx::umma_commit(bar_acc);                     // accumulator complete
+            __syncwarp();
+            if (++s == n_stages) { s = 0; phase ^= 1; }
         }
+        (void)ok;
     } else {
         // epilogue: warp w reads TMEM lanes [32*(w%4), +32) = batch rows m0 + that range
         const int quad = warp & 3;
         const int b = m0 + quad * 32 + lane;
-        bool ok = !*dead && ptx::mbar_wait(bar_acc, 0);
+        const bool ok = ptx::mbar_wait(bar_acc, 0);
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
 #pragma unroll 1
@@ -150,7 +181,8 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
 }
 
 template <int NT, bool IN_MAJOR>
-cudaError_t run(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
+cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches) {
+    p.x_rows = p.B > 64 ? 128 : p.B > 32 ? 64 : p.B > 16 ? 32 : 16;
     using T = ConvTile<NT>;
     static bool attr_set = false;
     if (!attr_set) {
@@ -161,7 +193,7 @@ cudaError_t run(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long
     }
     const CUtensorMap *t;
     CUtensorMap mx, mw;
-    if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, BM))) return cudaErrorInvalidValue;
+    if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, p.x_rows))) return cudaErrorInvalidValue;
     mx = *t;
     if (IN_MAJOR) t = ctx->tmaps.get(p.w, (uint64_t)p.D, (uint64_t)p.N, BK);        // [K, N], boxes of 64 k x 64 n
     else t = ctx->tmaps.get(p.w, (uint64_t)p.N, (uint64_t)p.D, NT);                 // [N, K], boxes of NT n x 64 k
