@@ -22,7 +22,11 @@ namespace {
 constexpr int BM = 128;                 // batch rows per CTA (UMMA M)
 constexpr int BK = 64;                  // K elements per swizzle atom (one 128-byte row)
 constexpr int KA = 2;                   // atoms per stage: one barrier round trip per 128 K elements
-constexpr int CONV_THREADS = 192;       // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int CONV_THREADS = 224;       // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue
+// With narrow weight slabs two warps issue MMAs: they take alternate stages and accumulate into
+// separate TMEM columns, because issuing a tcgen05.mma costs one thread more time than a narrow
+// MMA takes to run; the epilogue adds the accumulators.  Wide slabs gain nothing from it.
+template <int NT> __host__ __device__ constexpr int mma_warps() { return NT <= 64 ? 2 : 1; }
 
 constexpr int MAX_STAGES = 12;
 constexpr int RING_BYTES = 192 * 1024;
@@ -59,6 +63,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * NT, m0 = blockIdx.y * BM;
+    constexpr int MMA_WARPS = mma_warps<NT>();
     const int n_atoms = p.D / BK;
     const int n_steps = (n_atoms + KA - 1) / KA;
 
@@ -67,11 +72,11 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             ptx::mbar_init(bars + 16 * s, 1);
             ptx::mbar_init(bars + 16 * s + 8, 1);
         }
-        ptx::mbar_init(bar_acc, 1);
+        ptx::mbar_init(bar_acc, MMA_WARPS);
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_x); ptx::prefetch_tmap(&tm_w);
     }
-    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), NT);
+    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), MMA_WARPS * NT);
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
@@ -105,15 +110,22 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             __syncwarp();
             if (++s == n_stages) { s = 0; phase ^= 1; }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || (warp == 6 && MMA_WARPS == 2)) {
         constexpr uint32_t idesc = ptx::umma_idesc_bf16(BM, NT, false, W_IN_MAJOR);
+        const int me = warp == 1 ? 0 : 1;                  // which accumulator, and which stages
+        const uint32_t acc = tmem + me * NT;
+        const int last_mine = n_steps - 1 >= me ? n_steps - 1 - ((n_steps - 1 - me) % MMA_WARPS) : -1;
         int s = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool first = true;
+        if (last_mine < 0 && ptx::elect_one()) ptx::mbar_arrive(bar_acc);      // fewer steps than MMA warps
         for (int st = 0; st < n_steps; ++st) {
+            if (st % MMA_WARPS != me) {
+                if (++s == n_stages) { s = 0; phase ^= 1; }
+                continue;
+            }
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(bars + 16 * s, phase))) {
                 if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
-                ok = false;
                 break;
             }
             ptx::tc_fence_after();
@@ -130,17 +142,17 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
                         // 16 rows of 128 bytes (N-major); the address field counts 16-byte units
                         const uint64_t a_k = adesc + (uint64_t)(k * 2);
                         const uint64_t b_k = bdesc + (uint64_t)(W_IN_MAJOR ? k * 128 : k * 2);
-                        ptx::umma_bf16(tmem, a_k, b_k, idesc, (st | j | k) != 0);
+                        ptx::umma_bf16(acc, a_k, b_k, idesc, !first || (j | k) != 0);
                     }
                 }
                 ptx::umma_commit(bars + 16 * s + 8);       // frees the stage once these MMAs have read it
-                if (st == n_steps - 1) ptx::umma_commit(bar_acc);     // accumulator complete
+                if (st == last_mine) ptx::umma_commit(bar_acc);       // this warp's accumulator is complete
             }
+            first = false;
             __syncwarp();
             if (++s == n_stages) { s = 0; phase ^= 1; }
         }
-        (void)ok;
-    } else {
+    } else if (warp >= 2 && warp <= 5) {
         // epilogue: warp w reads TMEM lanes [32*(w%4), +32) = batch rows m0 + that range
         const int quad = warp & 3;
         const int b = m0 + quad * 32 + lane;
@@ -152,6 +164,13 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             uint32_t r[32];
             ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + c0, r);
             ptx::tmem_ld_wait();
+            if (MMA_WARPS == 2 && n_steps > 1) {           // second accumulator (untouched when there is one step)
+                uint32_t r2[32];
+                ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + NT + c0, r2);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) + __uint_as_float(r2[e]));
+            }
             if (ok && b < p.B) {
                 uint4 *dst = reinterpret_cast<uint4 *>(p.U + (size_t)b * p.N + n0 + c0);
 #pragma unroll
@@ -176,7 +195,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem, NT);
+        ptx::tmem_dealloc(tmem, MMA_WARPS * NT);
     }
 }
 
