@@ -87,6 +87,7 @@ cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t 
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                            long long *launches);
 int coarse_attn_ctas_per_sm();
+int shared_prefix_units_per_cta(int G);
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,

@@ -30,14 +30,6 @@ bool kv_ok(const photon_ctx *ctx, const photon_kv *c, bool allow_shared) {
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// Number of key ranges for a segment whose rows are bounded by max_rows:
-// enough CTAs to cover the SMs a few times over, but at least `min_rows` keys each.
-int choose_splits(const photon_ctx *ctx, int streams, int max_rows, int min_rows, int limit) {
-    if (max_rows <= 0 || streams <= 0) return 1;
-    const int want = ceil_div(ctx->sm_count * 4, streams);
-    const int by_rows = std::max(1, max_rows / min_rows);
-    return std::max(1, std::min(std::min(want, by_rows), limit));
-}
 
 photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
                                const int32_t *slot, int n_q, photon_bf16 *out, float *lse,
@@ -85,8 +77,10 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
             const int allowed = (int)std::min<size_t>(ctx->partial_floats / per_part, (size_t)ctx->max_splits);
             if (allowed < 1) return PHOTON_ERR_WORKSPACE;
             const int G = c.Hq / c.Hkv;
-            const int groups = ceil_div(n_q, 4 * (16 / G));       // units are taken in groups by the prefix kernel
-            p.splits_sh = choose_splits(ctx, groups * c.Hkv, ms, 128, allowed);
+            const int groups = ceil_div(n_q, shared_prefix_units_per_cta(G));     // tiles of 128 query rows
+            // one wave of CTAs: (row tiles x KV heads x key ranges) close to the number of SMs
+            const int want = std::max(1, ctx->sm_count / std::max(1, groups * c.Hkv));
+            p.splits_sh = std::max(1, std::min(std::min(want, std::max(1, ms / 128)), allowed));
         }
     }
     const cudaError_t e = chunk ? launch_chunk_attention(ctx, p, st, &ctx->launches)

@@ -1,15 +1,26 @@
 // Shared-prefix phase of the coarse decode attention (Section 1: long-context,
 // multi-query serving): many units (query branches) attend the same stored
-// prefix, which is therefore read once for a whole group of units.
+// prefix.  With hundreds of query rows per KV head this is a dense contraction,
+// so it runs on the 5th-generation tensor cores, and the prefix is read once per
+// group of 128 query rows instead of once per unit.
 //
-// CTA = (group of units, KV head, key range of the prefix).  The K/V tiles of
-// the range stream through a TMA-fed, 128-byte-swizzled shared-memory ring; each
-// of the four consumer warps owns 16 query rows (16/G units x G heads) and runs
-// them against every key of a tile on tensor cores with an fp32 online softmax
-// in the base-2 domain, so the prefix leaves HBM once and L2 feeds the other
-// groups.  Every (query head, key range) leaves an unnormalised partial
-// (acc, m, l) at partials[(query head) * splits_sh + range]; the kernel that
-// streams the units' own keys folds these partials into its result.
+// CTA = (tile of 128 query rows = 128/G units x G heads, KV head, key range of
+// the prefix).  Per 128-key tile:  S = Q K^T (tcgen05.mma, both operands
+// K-major from 128B-swizzled shared memory, S in TMEM);  four softmax warps read
+// their rows of S with tcgen05.ld (one thread = one query row), turn them into
+// probabilities in the base-2 domain and store them as bf16 into a swizzled
+// shared-memory tile P;  O += P V (tcgen05.mma, V as the N-major operand
+// straight from its TMA tile, O in TMEM across all tiles).  S is double
+// buffered, so the tensor pipe computes the next S while the warps work on this
+// one.  The reference maximum of a row is only raised when a tile exceeds it by
+// more than 2^8; then the row's O (and its running sum) is rescaled in TMEM
+// (tcgen05.ld / tcgen05.st).  Otherwise P simply carries factors up to 2^8.
+//
+// Every (query head, key range) leaves an unnormalised partial (acc, m, l) at
+// partials[(query head) * splits_sh + range]; the kernel that streams the
+// units' own keys folds these partials into its result.  Units of a tile that
+// name different prefixes are served in one pass per distinct prefix; a row
+// takes part only in the pass of its own prefix.
 #include <math_constants.h>
 
 #include "common.cuh"
@@ -17,24 +28,29 @@
 
 namespace {
 
-constexpr int NW = 4;                      // consumer warps per CTA
-constexpr int BN = 64;                     // keys per tile
-constexpr int THREADS = (NW + 1) * 32;     // + one producer warp
-constexpr int HALF_BYTES = BN * 128;       // one 64-row x 64-element swizzled box
+constexpr int BM = 128;                    // query rows per CTA (UMMA M; one TMEM lane each)
+constexpr int BN = 128;                    // keys per tile
+constexpr int KV_STAGES = 2;
+constexpr int SP_THREADS = 192;            // warps 0-3: softmax (TMEM lane quadrant = warp), 4: TMA, 5: MMA + TMEM owner
+constexpr float RESCALE_GAP = 8.f;         // log2 of the largest factor P may carry
 
 template <int DH>
-struct Tile {
+struct SpTile {
     static constexpr int HALVES = DH / 64;
-    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;     // K (or V) tile
-    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
-    static constexpr int STAGES = DH == 128 ? 3 : 4;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers, flags*/ +
-                                64 * 4 /*shared ids*/;
+    static constexpr int Q_BYTES = HALVES * BM * 128;
+    static constexpr int P_BYTES = (BN / 64) * BM * 128;
+    static constexpr int KV_BYTES = HALVES * BN * 128;          // K (or V) tile
+    static constexpr int OFF_P = Q_BYTES;
+    static constexpr int OFF_K = OFF_P + P_BYTES;
+    static constexpr int OFF_V = OFF_K + KV_STAGES * KV_BYTES;
+    static constexpr int OFF_TAIL = OFF_V + KV_STAGES * KV_BYTES;
+    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 /*barriers*/ + 64 /*scalars*/ + BM * 4 /*ids*/;
+    static constexpr int TMEM_COLS = 512;                       // S0, S1 (128 each), O (DH): next power of two
+    static constexpr int COL_O = 2 * BN;
 };
 
 __device__ __forceinline__ void part_range(int L, int n_splits, int p, int &r0, int &r1) {
-    // ranges start on tile boundaries so that TMA rows stay aligned to the key tiles
-    const int per = ((L + n_splits - 1) / n_splits + BN - 1) / BN * BN;
+    const int per = ((L + n_splits - 1) / n_splits + BN - 1) / BN * BN;      // whole tiles per range
     r0 = min(L, p * per);
     r1 = min(L, r0 + per);
 }
@@ -44,263 +60,298 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&t);
 }
 
-// One 16-key block of a tile against the warp's 16 query rows.
-//   kt, vt   shared-memory addresses of the K and V tiles (swizzled boxes)
-//   kb       index of the 16-key block inside the tile
-//   valid    number of valid keys in the block (1..16)
-//   act0/1   whether this thread's rows g and g+8 take part
 template <int DH>
-__device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, int valid,
-                                              const uint32_t (&qa)[DH / 16][4], float (&o)[DH / 8][4],
-                                              float (&m)[2], float (&l)[2], float scale_log2, int lane,
-                                              bool act0, bool act1, bool hi_rows) {
-    const int c = lane & 3;
-    float s[2][4];
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) s[j][e] = 0.f;
-
-    // S = Q K^T : B fragments straight from the swizzled K tile
-    {
-        const int mi = lane >> 3, r8 = lane & 7;
-#pragma unroll
-        for (int ks2 = 0; ks2 < DH / 32; ++ks2) {
-            const int cfull = ks2 * 4 + mi;                      // 16-byte chunk along dh
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int row = kb * 16 + j * 8 + r8;
-                const uint32_t addr = kt + (cfull >> 3) * HALF_BYTES + row * 128 +
-                                      ((((cfull & 7) ^ (row & 7))) << 4);
-                uint32_t b[4];
-                ptx::ldmatrix_x4(b, addr);
-                ptx::mma_bf16_16816(s[j], qa[ks2 * 2], b[0], b[1]);
-                ptx::mma_bf16_16816(s[j], qa[ks2 * 2 + 1], b[2], b[3]);
-            }
-        }
-    }
-    // scale, mask the tail keys
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int key = j * 8 + 2 * c + (e & 1);
-            s[j][e] = key < valid ? s[j][e] * scale_log2 : -CUDART_INF_F;
-        }
-    // online softmax, rows g (slot 0) and g+8 (slot 1)
-    float corr[2] = {1.f, 1.f};
-    uint32_t pa[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int rs = 0; rs < 2; ++rs) {
-        if (rs == 1 && !hi_rows) break;
-        const bool act = rs ? act1 : act0;
-        float mx = fmaxf(fmaxf(s[0][2 * rs], s[0][2 * rs + 1]), fmaxf(s[1][2 * rs], s[1][2 * rs + 1]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float mn = fmaxf(m[rs], mx);
-        const float cr = exp2f(m[rs] - mn);
-        float p0 = exp2f(s[0][2 * rs] - mn), p1 = exp2f(s[0][2 * rs + 1] - mn);
-        float p2 = exp2f(s[1][2 * rs] - mn), p3 = exp2f(s[1][2 * rs + 1] - mn);
-        if (act) {
-            corr[rs] = cr;
-            m[rs] = mn;
-            l[rs] = l[rs] * cr + ((p0 + p1) + (p2 + p3));
-            pa[rs] = pack_bf16(p0, p1);           // keys 2c, 2c+1
-            pa[rs + 2] = pack_bf16(p2, p3);       // keys 2c+8, 2c+9
-        }
-    }
-    // masks that clear V entries of keys past the end (they may hold anything)
-    uint32_t vm0 = 0xFFFFFFFFu, vm1 = 0xFFFFFFFFu;
-    if (valid < 16) {
-        vm0 = (2 * c < valid ? 0x0000FFFFu : 0u) | (2 * c + 1 < valid ? 0xFFFF0000u : 0u);
-        vm1 = (2 * c + 8 < valid ? 0x0000FFFFu : 0u) | (2 * c + 9 < valid ? 0xFFFF0000u : 0u);
-    }
-    // O = O * corr + P V : B fragments through transposing loads of the V tile
-    {
-        const int mi = lane >> 3, r8 = lane & 7;
-        const int row = kb * 16 + (mi & 1) * 8 + r8;
-#pragma unroll
-        for (int n2 = 0; n2 < DH / 16; ++n2) {
-            const int cfull = n2 * 2 + (mi >> 1);
-            const uint32_t addr = vt + (cfull >> 3) * HALF_BYTES + row * 128 +
-                                  ((((cfull & 7) ^ (row & 7))) << 4);
-            uint32_t b[4];
-            ptx::ldmatrix_x4_trans(b, addr);
-            b[0] &= vm0; b[1] &= vm1; b[2] &= vm0; b[3] &= vm1;
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                float(&acc)[4] = o[n2 * 2 + t];
-                acc[0] *= corr[0]; acc[1] *= corr[0];
-                if (hi_rows) { acc[2] *= corr[1]; acc[3] *= corr[1]; }
-                ptx::mma_bf16_16816(acc, pa, b[2 * t], b[2 * t + 1]);
-            }
-        }
-    }
-}
-
-template <int DH>
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(SP_THREADS, 1)
 shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_ks,
                      const __grid_constant__ CUtensorMap tm_vs) {
-    using T = Tile<DH>;
+    using T = SpTile<DH>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gen_base = smem_raw + (base - ptx::smem_u32(smem_raw));
-    const uint32_t bars = base + T::STAGES * T::STAGE_BYTES;        // full[s] at +16s, empty[s] at +16s+8
-    volatile int *dead = reinterpret_cast<volatile int *>(gen_base + T::STAGES * T::STAGE_BYTES + 128);
-    int *sid = reinterpret_cast<int *>(gen_base + T::STAGES * T::STAGE_BYTES + 256);
+    uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+    const uint32_t sQ = base, sP = base + T::OFF_P, sK = base + T::OFF_K, sV = base + T::OFF_V;
+    const uint32_t bars = base + T::OFF_TAIL;
+    // barriers (8 bytes each)
+    const uint32_t k_full = bars, v_full = bars + 16, kv_empty = bars + 32;      // [KV_STAGES]
+    const uint32_t s_ready = bars + 48, s_free = bars + 64;                      // [2]
+    const uint32_t p_ready = bars + 80, p_free = bars + 88;
+    int *sc = reinterpret_cast<int *>(gen + T::OFF_TAIL + 256);                  // [0] tmem base, [1..2] rescale flags
+    int *sid = sc + 16;                                                          // [BM] prefix id per query row's unit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, c = lane & 3;
     const int G = p.Hq / p.Hkv;
-    const int parts = p.splits_sh;
+    const int upt = BM / G;                                                      // units per tile
+    const int part = blockIdx.x % p.splits_sh;
+    const int h = (blockIdx.x / p.splits_sh) % p.Hkv;
+    const int unit0 = (blockIdx.x / (p.splits_sh * p.Hkv)) * upt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < T::STAGES; ++s) {
-            ptx::mbar_init(bars + 16 * s, 1);
-            ptx::mbar_init(bars + 16 * s + 8, NW);
+        for (int s = 0; s < KV_STAGES; ++s) {
+            ptx::mbar_init(k_full + 8 * s, 1);
+            ptx::mbar_init(v_full + 8 * s, 1);
+            ptx::mbar_init(kv_empty + 8 * s, 1);
         }
-        *dead = 0;
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(s_ready + 8 * b, 1);
+            ptx::mbar_init(s_free + 8 * b, 4);
+        }
+        ptx::mbar_init(p_ready, 4);
+        ptx::mbar_init(p_free, 1);
+        sc[1] = 0; sc[2] = 0;
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
+    if (warp == 5) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
 
-    const int part = blockIdx.x % p.splits_sh;
-    const int h = (blockIdx.x / p.splits_sh) % p.Hkv;
-    const int unit0 = (blockIdx.x / (p.splits_sh * p.Hkv)) * p.upc;      // first unit of the group
-    const int upw = 16 / G;                 // units per warp
-
-    // shared-segment id of every unit of the group: >= 0 valid, -1 none / out of range / bad
-    for (int j = threadIdx.x; j < p.upc; j += THREADS) {
-        const int i = unit0 + j;
+    // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch), and the Q tile:
+    // row r = (unit - unit0) * G + g, stored K-major with the 128-byte swizzle TMA would use
+    for (int r = threadIdx.x; r < BM; r += SP_THREADS) {
+        const int i = unit0 + r / G;
         int s = -1;
-        if (i < p.n_q) {
+        if (r < upt * G && i < p.n_q) {
             s = p.sh_id[i];
             if (s >= p.n_shared || s < 0) s = -1;
         }
-        sid[j] = s;
+        sid[r] = s;
     }
+    for (int idx = threadIdx.x; idx < BM * (DH / 8); idx += SP_THREADS) {
+        const int r = idx / (DH / 8), ch = idx % (DH / 8);                       // 16-byte chunk ch of row r
+        const int i = unit0 + r / G;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < upt * G && i < p.n_q)
+            v = *reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8);
+        ptx::sts128(sQ + (ch >> 3) * (BM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4), v);
+    }
+    ptx::fence_proxy_async();                  // generic-proxy writes of Q before the tensor core reads them
+    ptx::tc_fence_before();
     __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sc);
 
-    // ---- per-thread state of the consumer warps
-    uint32_t qa[DH / 16][4];
-    float o[DH / 8][4];
-    float m[2] = {-CUDART_INF_F, -CUDART_INF_F}, l[2] = {0.f, 0.f};
-    int row_unit[2] = {-1, -1};             // query index of rows g and g+8 (-1: padding row)
-    int row_head[2] = {0, 0};
-    if (warp < NW) {
-#pragma unroll
-        for (int rs = 0; rs < 2; ++rs) {
-            const int r = g + 8 * rs;
-            if (r < upw * G) {
-                const int i = unit0 + warp * upw + r / G;
-                if (i < p.n_q) { row_unit[rs] = i; row_head[rs] = h * G + r % G; }
-            }
+    // Every role walks the same list of tiles: for each distinct prefix id of the tile's units
+    // (ascending), the 128-key tiles of this CTA's key range of that prefix.
+    auto next_sid = [&](int last) {
+        int cur = 0x7FFFFFFF;
+        for (int r = 0; r < BM; r += G) {
+            const int s = sid[r];
+            if (s > last && s < cur) cur = s;
         }
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int rs = e & 1;                         // a0,a2: row g ; a1,a3: row g+8
-                const int col = ks * 16 + 2 * c + (e >> 1) * 8;
-                uint32_t v = 0u;
-                if (row_unit[rs] >= 0)
-                    v = *reinterpret_cast<const uint32_t *>(
-                        p.q + ((size_t)row_unit[rs] * p.Hq + row_head[rs]) * DH + col);
-                qa[ks][e] = v;
-            }
-#pragma unroll
-        for (int nt = 0; nt < DH / 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
-    }
-
-    int tg = 0;                               // tiles issued / consumed so far (ring position)
-
-    // One pass streams rows [r0, r1) of one (segment, kv head) through the ring.
-    auto run_pass = [&](const CUtensorMap *mk, const CUtensorMap *mv, long long row_base, int r0, int r1,
-                        bool act0, bool act1) {
-        const int ntiles = (r1 - r0 + BN - 1) / BN;
-        if (warp == NW) {
-            if (lane == 0) {
-                for (int t = 0; t < ntiles; ++t) {
-                    const int it = tg + t, s = it % T::STAGES;
-                    if (*dead) break;
-                    if (!ptx::mbar_wait(bars + 16 * s + 8, ((it / T::STAGES) & 1) ^ 1)) {
-                        *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
-                    }
-                    const uint32_t full = bars + 16 * s;
-                    const uint32_t kd = base + s * T::STAGE_BYTES, vd = kd + T::TILE_BYTES;
-                    const int y = (int)(row_base + r0 + (long long)t * BN);
-                    ptx::mbar_arrive_expect_tx(full, T::STAGE_BYTES);
-#pragma unroll
-                    for (int hh = 0; hh < T::HALVES; ++hh) {
-                        ptx::tma_load_2d(kd + hh * HALF_BYTES, mk, hh * 64, y, full);
-                        ptx::tma_load_2d(vd + hh * HALF_BYTES, mv, hh * 64, y, full);
-                    }
-                }
-            }
-        } else {
-            for (int t = 0; t < ntiles; ++t) {
-                const int it = tg + t, s = it % T::STAGES;
-                if (*dead) break;
-                if (!ptx::mbar_wait(bars + 16 * s, (it / T::STAGES) & 1)) {
-                    *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
-                }
-                const uint32_t kt = base + s * T::STAGE_BYTES, vt = kt + T::TILE_BYTES;
-                const int nvalid = min(BN, (r1 - r0) - t * BN);
-                for (int kb = 0; kb * 16 < nvalid; ++kb)
-                    process_block<DH>(kt, vt, kb, min(16, nvalid - kb * 16), qa, o, m, l, p.scale_log2, lane,
-                                      act0, act1, true);
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bars + 16 * s + 8);
-            }
-        }
-        tg += ntiles;
+        return cur;
     };
 
-    {
-        // ---- shared prefix: one pass per distinct segment id present in the group
-        int last = -1;
-        for (;;) {
-            int cur = 0x7FFFFFFF;
-            for (int j = 0; j < p.upc; ++j) {
-                const int s = sid[j];
-                if (s > last && s < cur) cur = s;
-            }
-            if (cur == 0x7FFFFFFF) break;
-            last = cur;
+    if (warp == 4) {
+        // ======================= TMA warp =======================
+        int it = 0;
+        bool ok = true;
+        for (int cur = next_sid(-1); cur != 0x7FFFFFFF && ok; cur = next_sid(cur)) {
             int r0, r1;
             part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
-            bool a0 = false, a1 = false;
-            if (warp < NW) {
-                const int j0 = warp * upw + g / G, j1 = warp * upw + (g + 8) / G;
-                a0 = row_unit[0] >= 0 && sid[j0] == cur;
-                a1 = row_unit[1] >= 0 && sid[j1] == cur;
-            }
-            run_pass(&tm_ks, &tm_vs, ((long long)cur * p.Hkv + h) * p.cap_sh, r0, r1, a0, a1);
-        }
-        if (warp < NW) {
+            const int row_base = (cur * p.Hkv + h) * p.cap_sh;
+            for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
+                const int s = it % KV_STAGES;
+                if (!__all_sync(0xffffffffu, ptx::mbar_wait(kv_empty + 8 * s, ((it / KV_STAGES) & 1) ^ 1))) {
+                    if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+                    ok = false;
+                    break;                     // stop loading; the other warps run out on their own bounded waits
+                }
+                if (ptx::elect_one()) {
+                    ptx::mbar_arrive_expect_tx(k_full + 8 * s, T::KV_BYTES);
 #pragma unroll
-            for (int rs = 0; rs < 2; ++rs) {
-                l[rs] += __shfl_xor_sync(0xffffffffu, l[rs], 1);
-                l[rs] += __shfl_xor_sync(0xffffffffu, l[rs], 2);
-                if (row_unit[rs] < 0) continue;
-                const size_t qh = (size_t)row_unit[rs] * p.Hq + row_head[rs];
-                float *dst = p.partials + (qh * parts + part) * (DH + 2);
+                    for (int hh = 0; hh < T::HALVES; ++hh)
+                        ptx::tma_load_2d(sK + s * T::KV_BYTES + hh * (BN * 128), &tm_ks, hh * 64, row_base + k0, k_full + 8 * s);
+                    ptx::mbar_arrive_expect_tx(v_full + 8 * s, T::KV_BYTES);
 #pragma unroll
-                for (int nt = 0; nt < DH / 8; ++nt)
-                    *reinterpret_cast<float2 *>(dst + nt * 8 + 2 * c) =
-                        make_float2(o[nt][2 * rs], o[nt][2 * rs + 1]);
-                if (c == 0) { dst[DH] = m[rs]; dst[DH + 1] = l[rs]; }
+                    for (int hh = 0; hh < T::HALVES; ++hh)
+                        ptx::tma_load_2d(sV + s * T::KV_BYTES + hh * (BN * 128), &tm_vs, hh * 64, row_base + k0, v_full + 8 * s);
+                }
+                __syncwarp();
             }
         }
+    } else if (warp == 5) {
+        // ======================= MMA warp =======================
+        constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(BM, BN, false, false);
+        constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(BM, DH, false, true);
+        int n_tiles = 0;
+        for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
+            int r0, r1;
+            part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
+            n_tiles += (r1 - r0 + BN - 1) / BN;
+        }
+        bool ok = true;
+        auto issue_qk = [&](int i) {           // S[i % 2] = Q K_i^T
+            const int s = i % KV_STAGES, b = i & 1;
+            bool good = ptx::mbar_wait(k_full + 8 * s, (i / KV_STAGES) & 1);
+            if (good && i >= 2) good = ptx::mbar_wait(s_free + 8 * b, ((i - 2) >> 1) & 1);
+            if (!__all_sync(0xffffffffu, good)) return false;
+            ptx::tc_fence_after();
+            if (ptx::elect_one()) {
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint64_t a = ptx::umma_desc_sw128(sQ + (ks >> 2) * (BM * 128) + (ks & 3) * 32, 0, 1024);
+                    const uint64_t bdesc = ptx::umma_desc_sw128(sK + s * T::KV_BYTES + (ks >> 2) * (BN * 128) + (ks & 3) * 32, 0, 1024);
+                    ptx::umma_bf16(tmem + b * BN, a, bdesc, idesc_qk, ks != 0);
+                }
+                ptx::umma_commit(s_ready + 8 * b);
+            }
+            __syncwarp();
+            return true;
+        };
+        if (n_tiles > 0) ok = issue_qk(0);
+        for (int i = 0; i < n_tiles && ok; ++i) {
+            if (i + 1 < n_tiles) ok = issue_qk(i + 1);
+            if (!ok) break;
+            const int s = i % KV_STAGES;
+            bool good = ptx::mbar_wait(p_ready, i & 1);
+            if (good) good = ptx::mbar_wait(v_full + 8 * s, (i / KV_STAGES) & 1);
+            if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
+            ptx::tc_fence_after();
+            if (ptx::elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {     // 16 keys per MMA
+                    const uint64_t a = ptx::umma_desc_sw128(sP + (kk >> 2) * (BM * 128) + (kk & 3) * 32, 0, 1024);
+                    // V tile: rows = keys (the K index), 128 bytes = 64 features (the N index): N-major operand
+                    const uint64_t bdesc = ptx::umma_desc_sw128(sV + s * T::KV_BYTES + kk * (16 * 128), BN * 128, 1024);
+                    ptx::umma_bf16(tmem + T::COL_O, a, bdesc, idesc_pv, (i | kk) != 0);
+                }
+                ptx::umma_commit(kv_empty + 8 * s);
+                ptx::umma_commit(p_free);
+            }
+            __syncwarp();
+        }
+        if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+    } else {
+        // ======================= softmax warps: thread = query row =======================
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const int my_sid = sid[row];
+        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        int it = 0;
+        bool ok = true;
+        // After a wait has run out (ok = false) the loop goes on without waiting, so that the four
+        // warps keep meeting at the named barrier; the results are then void and the status says so.
+        for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
+            int r0, r1;
+            part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
+            const bool active = (my_sid == cur);
+            for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
+                const int b = it & 1, st = it % KV_STAGES;
+                const int nvalid = min(BN, r1 - k0);
+                if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(s_ready + 8 * b, (it >> 1) & 1))) ok = false;
+                ptx::tc_fence_after();
+                uint32_t sr[BN];
+#pragma unroll
+                for (int c0 = 0; c0 < BN; c0 += 32)
+                    ptx::tmem_ld_32x32(tmem + lane_base + b * BN + c0, *reinterpret_cast<uint32_t(*)[32]>(&sr[c0]));
+                ptx::tmem_ld_wait();
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(s_free + 8 * b);          // the tensor pipe may overwrite this S
+
+                float mx = -CUDART_INF_F;
+#pragma unroll
+                for (int c = 0; c < BN; ++c) {
+                    const float v = c < nvalid ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
+                    sr[c] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+                float corr = 1.f;
+                bool need = false;
+                if (active) {
+                    if (m_ref == -CUDART_INF_F) {
+                        m_ref = mx;                                        // nothing accumulated for this row yet
+                    } else if (mx > m_ref + RESCALE_GAP) {
+                        corr = exp2f(m_ref - mx);
+                        m_ref = mx;
+                        need = true;
+                    }
+                }
+                // does any row of the CTA have to rescale its accumulator?
+                if (need) sc[1 + b] = 1;
+                ptx::named_bar_sync(1, 128);
+                const bool rescale = sc[1 + b] != 0;
+                // the previous P V must be done before P is overwritten (and before O is touched)
+                if (ok && it > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1))) ok = false;
+                if (rescale) {
+                    ptx::tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = 0; c0 < DH; c0 += 32) {
+                        uint32_t orow[32];
+                        ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * corr);
+                        ptx::tmem_st_32x32(tmem + lane_base + T::COL_O + c0, orow);
+                    }
+                    ptx::tmem_st_wait();
+                    l_sum *= corr;
+                    ptx::named_bar_sync(1, 128);                           // every reader of the flag is past it
+                    if (threadIdx.x == 0) sc[1 + b] = 0;
+                }
+                // rows of V past the end of the range may hold anything: clear them (P is 0 there, 0 * NaN is not)
+                if (nvalid < BN) {
+                    if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
+                    for (int idx = threadIdx.x; idx < (BN - nvalid) * T::HALVES * 8; idx += 128) {
+                        const int r = nvalid + idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
+                        ptx::sts128(sV + st * T::KV_BYTES + (c16 >> 3) * (BN * 128) + r * 128 + ((c16 & 7) << 4),
+                                    make_uint4(0u, 0u, 0u, 0u));
+                    }
+                }
+                // probabilities of this row, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
+                float ls = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < BN / 8; ++ch) {
+                    float e[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        e[j] = active ? exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref) : 0.f;
+                        ls += e[j];
+                    }
+                    const uint4 v = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]),
+                                               pack_bf16(e[6], e[7]));
+                    ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4), v);
+                }
+                l_sum += ls;
+                ptx::fence_proxy_async();
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(p_ready);
+            }
+        }
+        // ---- the partial of this row: accumulator relative to m_ref, m_ref, running sum
+        if (ok && it > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1));
+        if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+        ptx::tc_fence_after();
+        const int i = unit0 + row / G;
+        const bool row_ok = row < upt * G && i < p.n_q;
+        float *dst = nullptr;
+        if (row_ok) dst = p.partials + (((size_t)i * p.Hq + (size_t)h * G + row % G) * p.splits_sh + part) * (DH + 2);
+        const bool have = ok && it > 0 && l_sum > 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+            uint32_t orow[32];
+            if (it > 0) {                                                   // O was written by at least one P V
+                ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
+                ptx::tmem_ld_wait();
+            }
+            if (row_ok) {
+#pragma unroll
+                for (int e = 0; e < 32; e += 2)
+                    *reinterpret_cast<float2 *>(dst + c0 + e) =
+                        have ? make_float2(__uint_as_float(orow[e]), __uint_as_float(orow[e + 1])) : make_float2(0.f, 0.f);
+            }
+        }
+        if (row_ok) { dst[DH] = have ? m_ref : -CUDART_INF_F; dst[DH + 1] = have ? l_sum : 0.f; }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, T::TMEM_COLS);
     }
 }
 
 template <int DH>
 cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
-    using T = Tile<DH>;
+    using T = SpTile<DH>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(shared_prefix_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -309,20 +360,22 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
         attr_set = true;
     }
     const int G = p.Hq / p.Hkv;
-    p.upc = NW * (16 / G);
-    const int groups = (p.n_q + p.upc - 1) / p.upc;
+    const int upt = BM / G;
+    const int groups = (p.n_q + upt - 1) / upt;
     const CUtensorMap *t;
     CUtensorMap mks, mvs;
     if (!(t = ctx->tmaps.get(p.ks, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mks = *t;
     if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mvs = *t;
-    shared_prefix_kernel<DH><<<groups * p.Hkv * p.splits_sh, THREADS, T::SMEM, st>>>(p, mks, mvs);
+    shared_prefix_kernel<DH><<<groups * p.Hkv * p.splits_sh, SP_THREADS, T::SMEM, st>>>(p, mks, mvs);
     ++*launches;
     return cudaGetLastError();
 }
 
 }  // namespace
+
+int shared_prefix_units_per_cta(int G) { return BM / G; }
 
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                            long long *launches) {

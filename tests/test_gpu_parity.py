@@ -155,6 +155,30 @@ def test_shared_prefix_variants(oracle):
     assert np.abs(lse[fin] - want_lse[fin]).max() < 2e-3
 
 
+@pytest.mark.parametrize("max_splits", [1, 0])
+def test_shared_prefix_with_logits_that_grow_along_the_prefix(oracle, max_splits):
+    """Keys of later tiles score far higher than earlier ones for some query heads, so the reference
+    maximum of those rows has to be raised, and their accumulator rescaled, in the middle of a key range."""
+    cfg = cfg_small(3, B=40, S=8, shared_S=640)
+    co = wl.coarse_inputs(cfg)
+    co["len"][:] = 8
+    qf = wl.bf16_bits_to_f64(co["q"])                               # [B, Hq, dh]
+    ks = wl.bf16_bits_to_f64(co["k_shared"])                        # [1, Hkv, 640, dh]
+    for kvh in range(cfg.Hkv):
+        hq = kvh * cfg.G                                            # first query head of the group, unit 3
+        for t in range(1, 5):                                       # one boosted key per 128-key tile, growing
+            ks[0, kvh, 128 * t + 5] = qf[3, hq] * (0.6 * t)
+    co["k_shared"] = wl.f32_to_bf16_bits(ks.astype(np.float32))
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, shared=shared_of(co),
+                                      n_threads=NT)
+    with Ctx(cfg, max_splits=max_splits) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, "growing logits")
+    assert np.abs(lse - want_lse).max() < 2e-3 * max(1.0, np.abs(want_lse).max() / 10)
+
+
 def test_bad_shared_id_is_flagged_and_zeroed(oracle):
     cfg = cfg_small(3, B=6, S=20, shared_S=50)
     co = wl.coarse_inputs(cfg)
