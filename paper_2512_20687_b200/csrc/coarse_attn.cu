@@ -6,7 +6,9 @@
 // of all streams, in stream order, form one sequence; a persistent grid (two
 // CTAs per SM) gives every CTA an equal contiguous share of it, whatever the
 // lengths of the individual caches, so there is one wave and no tail.  The
-// split points are found on the device from len[] by a block-wide prefix sum.
+// split points are found on the device from len[] by a block-wide prefix sum;
+// a split point that falls inside a short stream moves to the nearer end of it
+// (a cut costs more than a few tiles of imbalance), long streams are cut.
 //
 // Inside a CTA one thread drives a ring of TMA loads (128-byte-swizzled boxes of
 // 32 rows, so rows past the end of a cache are not fetched; the group's query
@@ -43,6 +45,7 @@ constexpr int STAGES = 3;
 constexpr int HALF_BYTES = BN * 128;       // 64 rows x 64 elements, swizzled
 constexpr int BOX_BYTES = BOX * 128;
 constexpr int CTAS_PER_SM = 2;
+constexpr int SNAP = 8;                    // streams of at most this many tiles are never cut
 
 template <int DH>
 struct Ring {
@@ -129,23 +132,31 @@ __device__ __forceinline__ void emit_row(const AttnParams &p, int u, int hq, int
             L = 0.f;
         } else if (s >= 0) {
             const float *sp = p.partials + qh * p.splits_sh * (DH + 2);
-            for (int j = 0; j < p.splits_sh; ++j) {
-                const float *pj = sp + (size_t)j * (DH + 2);
-                const float lj = __ldcg(pj + DH + 1), mj = __ldcg(pj + DH);
-                float2 a[MAXV / 2];
+            constexpr int PB = MAXV <= 32 ? 2 : 1;           // partials fetched per trip: all their loads in flight together
+            for (int j0 = 0; j0 < p.splits_sh; j0 += PB) {
+                float lj[PB], mj[PB];
+                float2 a[PB][MAXV / 2];
 #pragma unroll
-                for (int i = 0; i < MAXV / 2; ++i)
-                    a[i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
-                if (!(lj > 0.f)) continue;
-                const float Mn = fmaxf(M, mj);
-                const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
+                for (int t = 0; t < PB; ++t) {
+                    const float *pj = sp + (size_t)min(j0 + t, p.splits_sh - 1) * (DH + 2);
+                    lj[t] = __ldcg(pj + DH + 1); mj[t] = __ldcg(pj + DH);
 #pragma unroll
-                for (int i = 0; i < MAXV / 2; ++i) {
-                    acc[2 * i] = acc[2 * i] * f0 + a[i].x * f1;
-                    acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[i].y * f1;
+                    for (int i = 0; i < MAXV / 2; ++i)
+                        a[t][i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
                 }
-                L = L * f0 + lj * f1;
-                M = Mn;
+#pragma unroll
+                for (int t = 0; t < PB; ++t) {
+                    if (j0 + t >= p.splits_sh || !(lj[t] > 0.f)) continue;
+                    const float Mn = fmaxf(M, mj[t]);
+                    const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj[t] - Mn);
+#pragma unroll
+                    for (int i = 0; i < MAXV / 2; ++i) {
+                        acc[2 * i] = acc[2 * i] * f0 + a[t][i].x * f1;
+                        acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[t][i].y * f1;
+                    }
+                    L = L * f0 + lj[t] * f1;
+                    M = Mn;
+                }
             }
         }
     }
@@ -266,7 +277,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     uint8_t *tail = reinterpret_cast<uint8_t *>(red) + (size_t)NW * G * (DH + 2) * sizeof(float);
     const uint32_t bars = ptx::smem_u32(tail);                  // full[s] at +16s, empty[s] at +16s+8
     const uint32_t red_full = bars + 16 * STAGES, red_empty = red_full + 8;
-    int *sc = reinterpret_cast<int *>(tail + 128);              // [0..5] warp sums, [8] u0, [9] rem, [11] dead,
+    int *sc = reinterpret_cast<int *>(tail + 128);              // [0..5] warp sums, [8] u0, [9] rem, [10] len(u0), [11] dead, [12] t0, [14] t1,
     volatile int *dead = sc + 11;                               // [16..23] description of the stream in `red`
     volatile int *meta = sc + 16;
 
@@ -280,7 +291,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         }
         ptx::mbar_init(red_full, NW);
         ptx::mbar_init(red_empty, 1);
-        sc[8] = -1; sc[9] = 0; sc[11] = 0;
+        sc[8] = -1; sc[9] = 0; sc[10] = 0; sc[11] = 0; sc[12] = 0; sc[14] = -1;
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
     }
@@ -305,21 +316,48 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         all += sc[w];
     }
     const long long T = (long long)all * p.Hkv;                  // tiles in the whole call
-    // every CTA that takes part owns at least one tile, so the CTAs holding a stream are consecutive
+    // every CTA that takes part owns at least one tile of the even deal, so the CTAs holding a cut stream
+    // are consecutive
     const int n_cta = (int)min((long long)gridDim.x, T);
-    const long long t0 = cta < n_cta ? T * cta / n_cta : 0, t1 = cta < n_cta ? T * (cta + 1) / n_cta : 0;
+    // Boundary c of the even deal is tile T*c/n_cta.  Where it falls inside a short stream (<= SNAP
+    // tiles) it moves to the nearer end of that stream: finishing a cut stream costs several round trips
+    // to global memory at the end of a CTA, more than a few tiles of imbalance.  Long streams are cut.
     {
         const long long lo = (long long)(before + incl - mine) * p.Hkv, hi = lo + (long long)mine * p.Hkv;
-        if (t0 < t1 && lo <= t0 && t0 < hi) {
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            const int c = cta + which;
+            if (cta >= n_cta || c >= n_cta) continue;
+            const long long x = T * c / n_cta;
+            if (!(lo <= x && x < hi)) continue;
             long long pre = lo;
             for (int u = ub; u < ue; ++u) {
-                const long long k = (long long)tiles_of(clamp_len(p.len[u], p.cap)) * p.Hkv;
-                if (t0 < pre + k) { sc[8] = u; sc[9] = (int)(t0 - pre); break; }
+                const int len = clamp_len(p.len[u], p.cap);
+                const int nt = tiles_of(len);
+                const long long k = (long long)nt * p.Hkv;
+                if (x < pre + k) {
+                    int rem = (int)(x - pre), uu = u, ll = len;
+                    const int j = rem % nt;
+                    long long bx = x;
+                    if (nt <= SNAP && j != 0) {
+                        if (2 * j <= nt) { bx = x - j; rem -= j; }
+                        else { bx = x + (nt - j); rem += nt - j; }
+                    }
+                    if (rem == nt * p.Hkv) {                      // moved to the start of the next stream's unit
+                        rem = 0;
+                        do { ++uu; ll = uu < p.n_units ? clamp_len(p.len[uu], p.cap) : 0; } while (uu < p.n_units && ll == 0);
+                    }
+                    if (which == 0) { sc[8] = uu; sc[9] = rem; sc[10] = ll; sc[12] = (int)bx; }
+                    else sc[14] = (int)bx;
+                    break;
+                }
                 pre += k;
             }
         }
     }
     __syncthreads();
+    const long long t0 = cta < n_cta ? sc[12] : 0;
+    const long long t1 = cta < n_cta ? (sc[14] >= 0 ? sc[14] : T) : 0;
 
     // ---- units without own keys are visited by no tile: finish them here
     for (int u = cta; u < p.n_units; u += gridDim.x) {
@@ -440,8 +478,9 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     }
 
     Walker w;
-    w.u = sc[8]; w.h = 0; w.j = 0;
-    w.load(p);
+    w.u = sc[8];
+    w.len = sc[10];
+    w.nt = tiles_of(w.len);
     w.h = sc[9] / w.nt;
     w.j = sc[9] % w.nt;
 

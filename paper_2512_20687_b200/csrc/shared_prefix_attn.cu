@@ -100,10 +100,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
-    if (warp == 5) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
-
-    // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch), and the Q tile:
-    // row r = (unit - unit0) * G + g, stored K-major with the 128-byte swizzle TMA would use
+    // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch); row r = (unit - unit0) * G + g
     for (int r = threadIdx.x; r < BM; r += SP_THREADS) {
         const int i = unit0 + r / G;
         int s = -1;
@@ -113,19 +110,39 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         sid[r] = s;
     }
-    for (int idx = threadIdx.x; idx < BM * (DH / 8); idx += SP_THREADS) {
-        const int r = idx / (DH / 8), ch = idx % (DH / 8);                       // 16-byte chunk ch of row r
-        const int i = unit0 + r / G;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (r < upt * G && i < p.n_q)
-            v = *reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8);
-        ptx::sts128(sQ + (ch >> 3) * (BM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4), v);
+    __syncthreads();                           // barriers and ids are ready: the TMA warp starts loading at once
+
+    uint32_t tmem = 0;
+    if (warp != 4) {
+        if (warp == 5) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
+        // the Q tile, stored K-major with the 128-byte swizzle TMA would use; all of a thread's loads are
+        // issued before its first store: one round trip to memory, not one per chunk
+        constexpr int NQT = SP_THREADS - 32;
+        constexpr int QV = (BM * (DH / 8) + NQT - 1) / NQT;
+        const int tq = threadIdx.x < 128 ? threadIdx.x : threadIdx.x - 32;
+        uint4 qv[QV];
+#pragma unroll
+        for (int t = 0; t < QV; ++t) {
+            const int idx = tq + t * NQT;
+            const int r = idx / (DH / 8), ch = idx % (DH / 8);                   // 16-byte chunk ch of row r
+            const int i = unit0 + r / G;
+            qv[t] = make_uint4(0u, 0u, 0u, 0u);
+            if (idx < BM * (DH / 8) && r < upt * G && i < p.n_q)
+                qv[t] = __ldg(reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8));
+        }
+#pragma unroll
+        for (int t = 0; t < QV; ++t) {
+            const int idx = tq + t * NQT;
+            const int r = idx / (DH / 8), ch = idx % (DH / 8);
+            if (idx < BM * (DH / 8))
+                ptx::sts128(sQ + (ch >> 3) * (BM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4), qv[t]);
+        }
+        ptx::fence_proxy_async();              // generic-proxy writes of Q before the tensor core reads them
+        ptx::tc_fence_before();
+        ptx::named_bar_sync(2, NQT);
+        ptx::tc_fence_after();
+        tmem = *reinterpret_cast<volatile uint32_t *>(sc);
     }
-    ptx::fence_proxy_async();                  // generic-proxy writes of Q before the tensor core reads them
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sc);
 
     // Every role walks the same list of tiles: for each distinct prefix id of the tile's units
     // (ascending), the 128-key tiles of this CTA's key range of that prefix.
@@ -247,11 +264,20 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 if (lane == 0) ptx::mbar_arrive(s_free + 8 * b);          // the tensor pipe may overwrite this S
 
                 float mx = -CUDART_INF_F;
+                if (nvalid == BN) {
 #pragma unroll
-                for (int c = 0; c < BN; ++c) {
-                    const float v = c < nvalid ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
-                    sr[c] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
+                    for (int c = 0; c < BN; ++c) {
+                        const float v = __uint_as_float(sr[c]) * p.scale_log2;
+                        sr[c] = __float_as_uint(v);
+                        mx = fmaxf(mx, v);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < BN; ++c) {
+                        const float v = c < nvalid ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
+                        sr[c] = __float_as_uint(v);
+                        mx = fmaxf(mx, v);
+                    }
                 }
                 float corr = 1.f;
                 bool need = false;
@@ -297,17 +323,24 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 }
                 // probabilities of this row, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
                 float ls = 0.f;
+                if (active) {
 #pragma unroll
-                for (int ch = 0; ch < BN / 8; ++ch) {
-                    float e[8];
+                    for (int ch = 0; ch < BN / 8; ++ch) {
+                        float e[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        e[j] = active ? exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref) : 0.f;
-                        ls += e[j];
+                        for (int j = 0; j < 8; ++j) {
+                            e[j] = exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref);
+                            ls += e[j];
+                        }
+                        const uint4 v = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]),
+                                                   pack_bf16(e[6], e[7]));
+                        ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4), v);
                     }
-                    const uint4 v = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]),
-                                               pack_bf16(e[6], e[7]));
-                    ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4), v);
+                } else {
+#pragma unroll
+                    for (int ch = 0; ch < BN / 8; ++ch)
+                        ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4),
+                                    make_uint4(0u, 0u, 0u, 0u));
                 }
                 l_sum += ls;
                 ptx::fence_proxy_async();
@@ -320,10 +353,10 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         if (ok && it > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1));
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
-        const int i = unit0 + row / G;
-        const bool row_ok = row < upt * G && i < p.n_q;
-        float *dst = nullptr;
-        if (row_ok) dst = p.partials + (((size_t)i * p.Hq + (size_t)h * G + row % G) * p.splits_sh + part) * (DH + 2);
+        // every MMA and every load of this CTA is done, so the tile buffers can serve as a staging area:
+        // rows go to shared memory (odd stride: no bank conflicts), then whole rows go out coalesced
+        constexpr int SROW = DH + 1;
+        float *stage = reinterpret_cast<float *>(gen);                            // [BM][SROW], then m[BM], l[BM]
         const bool have = ok && it > 0 && l_sum > 0.f;
 #pragma unroll 1
         for (int c0 = 0; c0 < DH; c0 += 32) {
@@ -332,14 +365,20 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
                 ptx::tmem_ld_wait();
             }
-            if (row_ok) {
 #pragma unroll
-                for (int e = 0; e < 32; e += 2)
-                    *reinterpret_cast<float2 *>(dst + c0 + e) =
-                        have ? make_float2(__uint_as_float(orow[e]), __uint_as_float(orow[e + 1])) : make_float2(0.f, 0.f);
-            }
+            for (int e = 0; e < 32; ++e) stage[row * SROW + c0 + e] = have ? __uint_as_float(orow[e]) : 0.f;
         }
-        if (row_ok) { dst[DH] = have ? m_ref : -CUDART_INF_F; dst[DH + 1] = have ? l_sum : 0.f; }
+        stage[BM * SROW + row] = have ? m_ref : -CUDART_INF_F;
+        stage[BM * SROW + BM + row] = have ? l_sum : 0.f;
+        ptx::named_bar_sync(1, 128);
+        for (int rr = warp; rr < BM; rr += 4) {
+            const int i = unit0 + rr / G;
+            if (rr >= upt * G || i >= p.n_q) continue;
+            float *dst = p.partials + (((size_t)i * p.Hq + (size_t)h * G + rr % G) * p.splits_sh + part) * (DH + 2);
+            for (int x = lane; x < DH / 2; x += 32)
+                *reinterpret_cast<float2 *>(dst + 2 * x) = make_float2(stage[rr * SROW + 2 * x], stage[rr * SROW + 2 * x + 1]);
+            if (lane == 0) { dst[DH] = stage[BM * SROW + rr]; dst[DH + 1] = stage[BM * SROW + BM + rr]; }
+        }
     }
     ptx::tc_fence_before();
     __syncthreads();
