@@ -63,8 +63,8 @@ enum {                                   /* storage order of the converter weigh
  * or 128, Hq/Hkv at most 16, D = d_model a multiple of 64, P + C at most 64.
  * max_queries: largest number of queries (sequences, branches or chunks) any
  * single attention call will carry; max_splits: upper bound on the number of
- * key ranges a shared prefix is split into (0 = library default).  Both
- * only size the workspace. */
+ * key ranges a shared prefix is split into (0 = library default; at most 8
+ * are used).  max_queries sizes the workspace. */
 typedef struct {
   int32_t Hq, Hkv, dh, D, P, C;
   int32_t max_queries;

@@ -100,11 +100,9 @@ __device__ __forceinline__ void emit(const AttnParams &p, int u, int hq, int d, 
             if (d == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
             L = 0.f; acc = 0.f;
         } else if (s >= 0) {
-            const float *sp = p.partials + qh * p.splits_sh * (DH + 2);
-            for (int j = 0; j < p.splits_sh; ++j) {
-                const float *pj = sp + (size_t)j * (DH + 2);
-                const float lj = __ldcg(pj + DH + 1);
-                if (!(lj > 0.f)) continue;
+            const float *pj = p.partials + qh * (DH + 2);
+            const float lj = __ldcg(pj + DH + 1);
+            if (lj > 0.f) {
                 const float mj = __ldcg(pj + DH);
                 const float Mn = fmaxf(M, mj);
                 const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
@@ -131,32 +129,22 @@ __device__ __forceinline__ void emit_row(const AttnParams &p, int u, int hq, int
             if (lead) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
             L = 0.f;
         } else if (s >= 0) {
-            const float *sp = p.partials + qh * p.splits_sh * (DH + 2);
-            constexpr int PB = MAXV <= 32 ? 2 : 1;           // partials fetched per trip: all their loads in flight together
-            for (int j0 = 0; j0 < p.splits_sh; j0 += PB) {
-                float lj[PB], mj[PB];
-                float2 a[PB][MAXV / 2];
+            const float *pj = p.partials + qh * (DH + 2);
+            const float lj = __ldcg(pj + DH + 1), mj = __ldcg(pj + DH);
+            float2 a[MAXV / 2];
 #pragma unroll
-                for (int t = 0; t < PB; ++t) {
-                    const float *pj = sp + (size_t)min(j0 + t, p.splits_sh - 1) * (DH + 2);
-                    lj[t] = __ldcg(pj + DH + 1); mj[t] = __ldcg(pj + DH);
+            for (int i = 0; i < MAXV / 2; ++i)
+                a[i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
+            if (lj > 0.f) {
+                const float Mn = fmaxf(M, mj);
+                const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
 #pragma unroll
-                    for (int i = 0; i < MAXV / 2; ++i)
-                        a[t][i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
+                for (int i = 0; i < MAXV / 2; ++i) {
+                    acc[2 * i] = acc[2 * i] * f0 + a[i].x * f1;
+                    acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[i].y * f1;
                 }
-#pragma unroll
-                for (int t = 0; t < PB; ++t) {
-                    if (j0 + t >= p.splits_sh || !(lj[t] > 0.f)) continue;
-                    const float Mn = fmaxf(M, mj[t]);
-                    const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj[t] - Mn);
-#pragma unroll
-                    for (int i = 0; i < MAXV / 2; ++i) {
-                        acc[2 * i] = acc[2 * i] * f0 + a[t][i].x * f1;
-                        acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[t][i].y * f1;
-                    }
-                    L = L * f0 + lj[t] * f1;
-                    M = Mn;
-                }
+                L = L * f0 + lj * f1;
+                M = Mn;
             }
         }
     }

@@ -31,7 +31,7 @@ struct photon_ctx {
     int device;
     int sm_count;
     int max_splits;          // resolved upper bound on key ranges per query
-    float *partials;         // shared-prefix partials: [max_queries * Hq * max_splits * (dh + 2)] floats
+    float *partials;         // shared-prefix partials: [max_queries * Hq][dh + 2] floats (acc, m, l)
     size_t partial_floats;
     float *cta_partials;     // partials of streams cut by a CTA boundary: [2 * max_ctas][16][dh + 2] floats
     int max_ctas;            // grid of the persistent attention kernel
@@ -59,7 +59,7 @@ struct AttnParams {
     int n_shared, cap_sh;
     const int32_t *slot;
     int n_q, Hq, Hkv, dh;
-    int splits_sh;           // key ranges of a shared prefix (0: no shared prefix in this call)
+    int splits_sh;           // key ranges of a shared prefix = cluster size of its kernel (0: no shared prefix)
     int upc;                 // filled by the launcher: units per CTA on shared keys
     float scale_log2;        // scale * log2(e): logits are kept in the base-2 domain
     float *partials;

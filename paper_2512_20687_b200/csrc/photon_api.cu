@@ -8,7 +8,6 @@
 namespace {
 
 constexpr int kDefaultMaxSplits = 32;
-constexpr size_t kMaxPartialFloats = size_t(64) << 20;     // 256 MiB ceiling on the split-K workspace
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -73,14 +72,14 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
             p.sh_len = cache->shared_len; p.sh_id = cache->shared_id;
             p.n_shared = cache->n_shared; p.cap_sh = cache->cap_shared;
             const int ms = cache->max_shared_len ? cache->max_shared_len : cache->cap_shared;
-            const size_t per_part = size_t(n_q) * c.Hq * (c.dh + 2);
-            const int allowed = (int)std::min<size_t>(ctx->partial_floats / per_part, (size_t)ctx->max_splits);
-            if (allowed < 1) return PHOTON_ERR_WORKSPACE;
+            if (size_t(n_q) * c.Hq * (c.dh + 2) > ctx->partial_floats) return PHOTON_ERR_WORKSPACE;
             const int G = c.Hq / c.Hkv;
             const int groups = ceil_div(n_q, shared_prefix_units_per_cta(G));     // tiles of 128 query rows
-            // one wave of CTAs: (row tiles x KV heads x key ranges) close to the number of SMs
+            // key ranges per row tile = cluster size: a power of two up to 8, about one wave of CTAs in all
             const int want = std::max(1, ctx->sm_count / std::max(1, groups * c.Hkv));
-            p.splits_sh = std::max(1, std::min(std::min(want, std::max(1, ms / 128)), allowed));
+            const int cap = std::min(std::min(want, std::max(1, ms / 128)), std::min(8, ctx->max_splits));
+            p.splits_sh = 1;
+            while (p.splits_sh * 2 <= cap) p.splits_sh *= 2;
         }
     }
     const cudaError_t e = chunk ? launch_chunk_attention(ctx, p, st, &ctx->launches)
@@ -120,8 +119,7 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
         return PHOTON_ERR_UNSUPPORTED;
     }
     ctx->sm_count = prop.multiProcessorCount;
-    const size_t per_part = size_t(c.max_queries) * c.Hq * (c.dh + 2);
-    ctx->partial_floats = std::max(per_part, std::min(per_part * ctx->max_splits, kMaxPartialFloats));
+    ctx->partial_floats = size_t(c.max_queries) * c.Hq * (c.dh + 2);      // one shared-prefix partial per query head
     ctx->n_tickets = size_t(c.max_queries) * c.Hkv;
     ctx->max_ctas = ctx->sm_count * coarse_attn_ctas_per_sm();
     if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||

@@ -16,9 +16,12 @@
 // more than 2^8; then the row's O (and its running sum) is rescaled in TMEM
 // (tcgen05.ld / tcgen05.st).  Otherwise P simply carries factors up to 2^8.
 //
-// Every (query head, key range) leaves an unnormalised partial (acc, m, l) at
-// partials[(query head) * splits_sh + range]; the kernel that streams the
-// units' own keys folds these partials into its result.  Units of a tile that
+// The key ranges of one row tile (1, 2, 4 or 8 of them) are the CTAs of one
+// thread-block cluster: at the end they merge their results by log-sum-exp
+// through distributed shared memory, each CTA taking a share of the rows, and
+// leave ONE unnormalised partial (acc, m, l) per query head at
+// partials[query head]; the kernel that streams the units' own keys folds it
+// into its result.  Units of a tile that
 // name different prefixes are served in one pass per distinct prefix; a row
 // takes part only in the pass of its own prefix.
 #include <math_constants.h>
@@ -370,18 +373,40 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         stage[BM * SROW + row] = have ? m_ref : -CUDART_INF_F;
         stage[BM * SROW + BM + row] = have ? l_sum : 0.f;
-        ptx::named_bar_sync(1, 128);
-        for (int rr = warp; rr < BM; rr += 4) {
+    }
+
+    // ---- the key ranges of one row tile are the CTAs of one cluster: every CTA merges a share of the
+    // rows across all of them through distributed shared memory and writes one partial per query head
+    ptx::tc_fence_before();
+    ptx::cluster_sync();                                           // every CTA of the cluster has staged its rows
+    {
+        constexpr int SROW = DH + 1;
+        const int C = p.splits_sh, rows_per = BM / C;
+        const uint32_t st_rows = base, st_m = base + BM * SROW * 4, st_l = st_m + BM * 4;
+        for (int rr = part * rows_per + warp; rr < (part + 1) * rows_per; rr += SP_THREADS / 32) {
             const int i = unit0 + rr / G;
             if (rr >= upt * G || i >= p.n_q) continue;
-            float *dst = p.partials + (((size_t)i * p.Hq + (size_t)h * G + rr % G) * p.splits_sh + part) * (DH + 2);
-            for (int x = lane; x < DH / 2; x += 32)
-                *reinterpret_cast<float2 *>(dst + 2 * x) = make_float2(stage[rr * SROW + 2 * x], stage[rr * SROW + 2 * x + 1]);
-            if (lane == 0) { dst[DH] = stage[BM * SROW + rr]; dst[DH + 1] = stage[BM * SROW + BM + rr]; }
+            float M = -CUDART_INF_F;
+            for (int r = 0; r < C; ++r)
+                if (ptx::ld_cluster_f32(st_l + rr * 4, r) > 0.f) M = fmaxf(M, ptx::ld_cluster_f32(st_m + rr * 4, r));
+            float L = 0.f, acc[DH / 32];
+#pragma unroll
+            for (int k = 0; k < DH / 32; ++k) acc[k] = 0.f;
+            for (int r = 0; r < C; ++r) {
+                const float lr = ptx::ld_cluster_f32(st_l + rr * 4, r);
+                if (!(lr > 0.f)) continue;
+                const float f = exp2f(ptx::ld_cluster_f32(st_m + rr * 4, r) - M);
+                L += lr * f;
+#pragma unroll
+                for (int k = 0; k < DH / 32; ++k) acc[k] += f * ptx::ld_cluster_f32(st_rows + (rr * SROW + lane + 32 * k) * 4, r);
+            }
+            float *dst = p.partials + ((size_t)i * p.Hq + (size_t)h * G + rr % G) * (DH + 2);
+#pragma unroll
+            for (int k = 0; k < DH / 32; ++k) dst[lane + 32 * k] = acc[k];
+            if (lane == 0) { dst[DH] = M; dst[DH + 1] = L; }
         }
     }
-    ptx::tc_fence_before();
-    __syncthreads();
+    ptx::cluster_sync();                                           // nobody reads this CTA's shared memory any more
     if (warp == 5) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, T::TMEM_COLS);
@@ -407,9 +432,21 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     mks = *t;
     if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mvs = *t;
-    shared_prefix_kernel<DH><<<groups * p.Hkv * p.splits_sh, SP_THREADS, T::SMEM, st>>>(p, mks, mvs);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(groups * p.Hkv * p.splits_sh);
+    cfg.blockDim = dim3(SP_THREADS);
+    cfg.dynamicSmemBytes = T::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;          // the key ranges of a row tile form a cluster
+    attr[0].val.clusterDim.x = p.splits_sh;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, shared_prefix_kernel<DH>, p, mks, mvs);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
