@@ -116,43 +116,54 @@ __device__ __forceinline__ void emit(const AttnParams &p, int u, int hq, int d, 
     if (d == 0 && p.lse) p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
 }
 
-// The finishing warp holds, per lane, V consecutive features [d0, d0 + V) of one query head
-// (acc unnormalised, M and L of that head).  Same combination as emit(), with every partial
-// fetched by independent loads (one round trip per partial).
+// The shared-prefix partial of one query head as the finishing warp holds it: fetched before the own keys
+// of the stream are done, so that its latency hides behind the consumers' work.
+template <int MAXV>
+struct SharedPart {
+    int sid;                 // prefix id of the unit (< 0: none)
+    float l, m;
+    float2 a[MAXV / 2];
+};
+
 template <int DH, int MAXV>
-__device__ __forceinline__ void emit_row(const AttnParams &p, int u, int hq, int d0, int V, bool lead,
-                                         float (&acc)[MAXV], float M, float L) {
+__device__ __forceinline__ void fetch_shared(const AttnParams &p, int u, int hq, int d0, SharedPart<MAXV> &sp) {
+    sp.sid = -1;
+    if (p.splits_sh <= 0) return;
+    sp.sid = p.sh_id[u];
+    if (sp.sid < 0 || sp.sid >= p.n_shared) return;
+    const float *pj = p.partials + ((size_t)u * p.Hq + hq) * (DH + 2);
+    sp.l = __ldcg(pj + DH + 1);
+    sp.m = __ldcg(pj + DH);
+#pragma unroll
+    for (int i = 0; i < MAXV / 2; ++i) sp.a[i] = __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i);
+}
+
+// The finishing warp holds, per lane, MAXV consecutive features [d0, d0 + MAXV) of one query head
+// (acc unnormalised, M and L of that head).  Same combination as emit().
+template <int DH, int MAXV>
+__device__ __forceinline__ void emit_row(const AttnParams &p, int u, int hq, int d0, bool lead,
+                                         float (&acc)[MAXV], float M, float L, const SharedPart<MAXV> &sp) {
     const size_t qh = (size_t)u * p.Hq + hq;
     if (p.splits_sh > 0) {
-        const int s = p.sh_id[u];
-        if (s >= p.n_shared) {
+        if (sp.sid >= p.n_shared) {                  // bad shared id voids the query
             if (lead) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
             L = 0.f;
-        } else if (s >= 0) {
-            const float *pj = p.partials + qh * (DH + 2);
-            const float lj = __ldcg(pj + DH + 1), mj = __ldcg(pj + DH);
-            float2 a[MAXV / 2];
+        } else if (sp.sid >= 0 && sp.l > 0.f) {
+            const float Mn = fmaxf(M, sp.m);
+            const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(sp.m - Mn);
 #pragma unroll
-            for (int i = 0; i < MAXV / 2; ++i)
-                a[i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(pj + d0) + i) : make_float2(0.f, 0.f);
-            if (lj > 0.f) {
-                const float Mn = fmaxf(M, mj);
-                const float f0 = L > 0.f ? exp2f(M - Mn) : 0.f, f1 = exp2f(mj - Mn);
-#pragma unroll
-                for (int i = 0; i < MAXV / 2; ++i) {
-                    acc[2 * i] = acc[2 * i] * f0 + a[i].x * f1;
-                    acc[2 * i + 1] = acc[2 * i + 1] * f0 + a[i].y * f1;
-                }
-                L = L * f0 + lj * f1;
-                M = Mn;
+            for (int i = 0; i < MAXV / 2; ++i) {
+                acc[2 * i] = acc[2 * i] * f0 + sp.a[i].x * f1;
+                acc[2 * i + 1] = acc[2 * i + 1] * f0 + sp.a[i].y * f1;
             }
+            L = L * f0 + sp.l * f1;
+            M = Mn;
         }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     uint32_t *dst = reinterpret_cast<uint32_t *>(p.out + qh * DH + d0);
 #pragma unroll
-    for (int i = 0; i < MAXV / 2; ++i)
-        if (2 * i < V) dst[i] = pack_bf16(acc[2 * i] * inv, acc[2 * i + 1] * inv);
+    for (int i = 0; i < MAXV / 2; ++i) dst[i] = pack_bf16(acc[2 * i] * inv, acc[2 * i + 1] * inv);
     if (lead && p.lse) p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
 }
 
@@ -250,11 +261,14 @@ __device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, 
     }
 }
 
-template <int DH, int NT8>
+// GP: the group size G rounded up to a power of two (1 .. 16); it fixes how the finishing warp's lanes
+// map to (query head, features) and how many n-tiles of 8 heads the MMAs span.
+template <int DH, int GP>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
 coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v) {
     using R = Ring<DH>;
+    constexpr int NT8 = GP > 8 ? 2 : 1;
     extern __shared__ uint8_t smem_raw[];
     const int G = p.Hq / p.Hkv;
     const int QB = q_slot_bytes(G, DH);
@@ -360,13 +374,18 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     if (warp == NW + 1) {
         // ======================= finishing warp =======================
         // lane -> (query head r of the group, features [d0, d0 + V))
-        constexpr int MAXV = DH * 8 * NT8 / 32;
-        int Gp = 1;
-        while (Gp < G) Gp <<= 1;
-        const int lpr = 32 / Gp;                        // lanes per query head
-        const int r = lane / lpr, V = DH / lpr, d0 = (lane % lpr) * V;
+        constexpr int MAXV = DH * GP / 32;
+        constexpr int lpr = 32 / GP;                    // lanes per query head
+        const int r = lane / lpr, d0 = (lane % lpr) * MAXV;
         const bool row_ok = r < G, lead = row_ok && (lane % lpr == 0);
+        // it walks the streams of this CTA in the consumers' order, one step ahead of them
+        Walker fw;
+        fw.u = sc[8]; fw.len = sc[10]; fw.nt = tiles_of(fw.len);
+        fw.h = sc[9] / fw.nt; fw.j = sc[9] % fw.nt;
         for (int sidx = 0;; ++sidx) {
+            SharedPart<MAXV> sp;
+            sp.sid = -1;
+            if (row_ok && fw.u < p.n_units) fetch_shared<DH, MAXV>(p, fw.u, fw.h * G + r, d0, sp);
             if (*dead || !ptx::mbar_wait(red_full, sidx & 1)) {
                 if (!*dead) { *dead = 1; if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT); }
                 break;
@@ -390,25 +409,24 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         const float f = exp2f(src[DH] - M);
                         L += lw * f;
 #pragma unroll
-                        for (int i = 0; i < MAXV / 2; ++i)
-                            if (2 * i < V) {
-                                const float2 a = *reinterpret_cast<const float2 *>(src + d0 + 2 * i);
-                                acc[2 * i] += a.x * f; acc[2 * i + 1] += a.y * f;
-                            }
+                        for (int i = 0; i < MAXV / 2; ++i) {
+                            const float2 a = *reinterpret_cast<const float2 *>(src + d0 + 2 * i);
+                            acc[2 * i] += a.x * f; acc[2 * i + 1] += a.y * f;
+                        }
                     }
                 }
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(red_empty);          // consumers may reuse `red`
             if (whole) {
-                if (row_ok) emit_row<DH, MAXV>(p, u, h * G + r, d0, V, lead, acc, M, L);
+                if (row_ok) emit_row<DH, MAXV>(p, u, h * G + r, d0, lead, acc, M, L, sp);
             } else {
                 // the stream is shared with neighbouring CTAs: leave a partial, whoever arrives last merges
                 if (row_ok) {
                     float *dst = p.cta_partials + ((size_t)(2 * cta + (cta < c_last ? 1 : 0)) * G + r) * (DH + 2);
 #pragma unroll
                     for (int i = 0; i < MAXV / 2; ++i)
-                        if (2 * i < V) *reinterpret_cast<float2 *>(dst + d0 + 2 * i) = make_float2(acc[2 * i], acc[2 * i + 1]);
+                        *reinterpret_cast<float2 *>(dst + d0 + 2 * i) = make_float2(acc[2 * i], acc[2 * i + 1]);
                     if (lead) { dst[DH] = M; dst[DH + 1] = L; }
                 }
                 __threadfence();
@@ -438,8 +456,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                 lj[t] = __ldcg(src + DH + 1); mj[t] = __ldcg(src + DH);
 #pragma unroll
                                 for (int i = 0; i < MAXV / 2; ++i)
-                                    a[t][i] = 2 * i < V ? __ldcg(reinterpret_cast<const float2 *>(src + d0) + i)
-                                                        : make_float2(0.f, 0.f);
+                                    a[t][i] = __ldcg(reinterpret_cast<const float2 *>(src + d0) + i);
                             }
                             if (cc + 1 > c_last) lj[1] = 0.f;
 #pragma unroll
@@ -456,11 +473,13 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                 M = Mn;
                             }
                         }
-                        emit_row<DH, MAXV>(p, u, h * G + r, d0, V, lead, acc, M, L);
+                        emit_row<DH, MAXV>(p, u, h * G + r, d0, lead, acc, M, L, sp);
                     }
                 }
             }
             if (final_seg) break;
+            fw.j = fw.nt - 1;                                   // on to the next stream
+            fw.next(p);
         }
         return;
     }
@@ -600,13 +619,13 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     }
 }
 
-template <int DH, int NT8>
+template <int DH, int GP>
 cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
     const int G = p.Hq / p.Hkv;
     const size_t smem = smem_bytes<DH>(G);
     static size_t smem_set = 0;
     if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(coarse_attn_kernel<DH, NT8>,
+        cudaError_t e = cudaFuncSetAttribute(coarse_attn_kernel<DH, GP>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
@@ -619,7 +638,7 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     mv = *t;
     const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
     const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, ctx->max_ctas));
-    coarse_attn_kernel<DH, NT8><<<grid, THREADS, smem, st>>>(p, mk, mv);
+    coarse_attn_kernel<DH, GP><<<grid, THREADS, smem, st>>>(p, mk, mv);
     ++*launches;
     return cudaGetLastError();
 }
@@ -635,6 +654,13 @@ cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t 
         if (e != cudaSuccess) return e;
     }
     const int G = p.Hq / p.Hkv;
-    if (p.dh == 64) return G <= 8 ? run<64, 1>(ctx, p, st, launches) : run<64, 2>(ctx, p, st, launches);
-    return G <= 8 ? run<128, 1>(ctx, p, st, launches) : run<128, 2>(ctx, p, st, launches);
+    int gp = 1;
+    while (gp < G) gp <<= 1;
+#define PHOTON_COARSE_CASE(D, GPV) if (p.dh == D && gp == GPV) return run<D, GPV>(ctx, p, st, launches);
+    PHOTON_COARSE_CASE(128, 1) PHOTON_COARSE_CASE(128, 2) PHOTON_COARSE_CASE(128, 4) PHOTON_COARSE_CASE(128, 8)
+    PHOTON_COARSE_CASE(128, 16)
+    PHOTON_COARSE_CASE(64, 1) PHOTON_COARSE_CASE(64, 2) PHOTON_COARSE_CASE(64, 4) PHOTON_COARSE_CASE(64, 8)
+    PHOTON_COARSE_CASE(64, 16)
+#undef PHOTON_COARSE_CASE
+    return cudaErrorInvalidValue;
 }

@@ -17,9 +17,9 @@
 // (tcgen05.ld / tcgen05.st).  Otherwise P simply carries factors up to 2^8.
 //
 // The key ranges of one row tile (1, 2, 4 or 8 of them) are the CTAs of one
-// thread-block cluster: at the end they merge their results by log-sum-exp
-// through distributed shared memory, each CTA taking a share of the rows, and
-// leave ONE unnormalised partial (acc, m, l) per query head at
+// thread-block cluster: at the end every CTA sends its rows to the CTA that owns
+// them (bulk copies into the peer's shared memory), each CTA merges the rows it owns
+// by log-sum-exp, and the cluster leaves ONE unnormalised partial (acc, m, l) per query head at
 // partials[query head]; the kernel that streams the units' own keys folds it
 // into its result.  Units of a tile that
 // name different prefixes are served in one pass per distinct prefix; a row
@@ -76,7 +76,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     // barriers (8 bytes each)
     const uint32_t k_full = bars, v_full = bars + 16, kv_empty = bars + 32;      // [KV_STAGES]
     const uint32_t s_ready = bars + 48, s_free = bars + 64;                      // [2]
-    const uint32_t p_ready = bars + 80, p_free = bars + 88;
+    const uint32_t p_ready = bars + 80, p_free = bars + 88, recv_bar = bars + 96;
     int *sc = reinterpret_cast<int *>(gen + T::OFF_TAIL + 256);                  // [0] tmem base, [1..2] rescale flags
     int *sid = sc + 16;                                                          // [BM] prefix id per query row's unit
 
@@ -99,8 +99,11 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         ptx::mbar_init(p_ready, 4);
         ptx::mbar_init(p_free, 1);
+        ptx::mbar_init(recv_bar, 1);
         sc[1] = 0; sc[2] = 0;
         ptx::mbar_fence_init();
+        // the rows this CTA owns arrive from every CTA of its cluster (itself included) at the very end
+        ptx::mbar_arrive_expect_tx(recv_bar, BM * (DH + 4) * 4);
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
     // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch); row r = (unit - unit0) * G + g
@@ -157,6 +160,10 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         return cur;
     };
+
+    // what a softmax thread carries out of the key loop for its row
+    float fin_m = -CUDART_INF_F, fin_l = 0.f;
+    bool fin_have = false, fin_any = false;
 
     if (warp == 4) {
         // ======================= TMA warp =======================
@@ -356,57 +363,102 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         if (ok && it > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1));
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
-        // every MMA and every load of this CTA is done, so the tile buffers can serve as a staging area:
-        // rows go to shared memory (odd stride: no bank conflicts), then whole rows go out coalesced
-        constexpr int SROW = DH + 1;
-        float *stage = reinterpret_cast<float *>(gen);                            // [BM][SROW], then m[BM], l[BM]
-        const bool have = ok && it > 0 && l_sum > 0.f;
+        fin_have = ok && it > 0 && l_sum > 0.f;
+        fin_any = it > 0;
+        fin_m = m_ref;
+        fin_l = l_sum;
+    }
+
+    // ---- the key ranges of one row tile are the CTAs of one cluster.  Each CTA stages its rows
+    // (acc, m, l) in its own shared memory; when every CTA of the cluster is done with its tile buffers,
+    // one bulk copy per owner moves the rows a peer owns into that peer's receive buffer (completion
+    // counted on the peer's mbarrier); every CTA then merges the rows it owns by log-sum-exp from its own
+    // shared memory and writes one partial per query head.
+    constexpr int RS = DH + 4;                                     // floats per staged row: 16-byte aligned rows
+    const int C = p.splits_sh, rows_per = BM / C;
+    const uint32_t stage_a = base, recv_a = base + BM * RS * 4;    // stage [BM][RS]; receive [C sources][rows_per][RS]
+    if (warp < 4) {
+        // every MMA and every load of this CTA is done, so its tile buffers can serve as the staging area
+        ptx::tc_fence_after();
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float *stage = reinterpret_cast<float *>(gen) + (size_t)row * RS;
 #pragma unroll 1
         for (int c0 = 0; c0 < DH; c0 += 32) {
             uint32_t orow[32];
-            if (it > 0) {                                                   // O was written by at least one P V
+            if (fin_any) {                                                  // O was written by at least one P V
                 ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
                 ptx::tmem_ld_wait();
             }
 #pragma unroll
-            for (int e = 0; e < 32; ++e) stage[row * SROW + c0 + e] = have ? __uint_as_float(orow[e]) : 0.f;
+            for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<float4 *>(stage + c0 + e) =
+                    fin_have ? make_float4(__uint_as_float(orow[e]), __uint_as_float(orow[e + 1]), __uint_as_float(orow[e + 2]),
+                                           __uint_as_float(orow[e + 3]))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        stage[BM * SROW + row] = have ? m_ref : -CUDART_INF_F;
-        stage[BM * SROW + BM + row] = have ? l_sum : 0.f;
+        *reinterpret_cast<float4 *>(stage + DH) =
+            make_float4(fin_have ? fin_m : -CUDART_INF_F, fin_have ? fin_l : 0.f, 0.f, 0.f);
+        ptx::fence_proxy_async();                                  // the bulk copies below read what was staged here
     }
-
-    // ---- the key ranges of one row tile are the CTAs of one cluster: every CTA merges a share of the
-    // rows across all of them through distributed shared memory and writes one partial per query head
     ptx::tc_fence_before();
-    ptx::cluster_sync();                                           // every CTA of the cluster has staged its rows
+    ptx::cluster_sync();                                           // staged everywhere; receive buffers are free
+    if (warp == 4 && ptx::elect_one()) {
+        const uint32_t bytes = rows_per * RS * 4;
+        for (int o = 0; o < C; ++o)
+            ptx::bulk_copy_to_peer(ptx::map_cluster(recv_a + part * bytes, o), stage_a + o * bytes, bytes,
+                                   ptx::map_cluster(recv_bar, o));
+    }
+    const bool got = ptx::mbar_wait(recv_bar, 0);                  // the rows this CTA owns are all here
+    if (!got && threadIdx.x == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
     {
-        constexpr int SROW = DH + 1;
-        const int C = p.splits_sh, rows_per = BM / C;
-        const uint32_t st_rows = base, st_m = base + BM * SROW * 4, st_l = st_m + BM * 4;
-        for (int rr = part * rows_per + warp; rr < (part + 1) * rows_per; rr += SP_THREADS / 32) {
+        const float *recv = reinterpret_cast<const float *>(gen) + BM * RS;
+        for (int rl = warp; rl < rows_per; rl += SP_THREADS / 32) {
+            const int rr = part * rows_per + rl;
             const int i = unit0 + rr / G;
             if (rr >= upt * G || i >= p.n_q) continue;
-            float M = -CUDART_INF_F;
-            for (int r = 0; r < C; ++r)
-                if (ptx::ld_cluster_f32(st_l + rr * 4, r) > 0.f) M = fmaxf(M, ptx::ld_cluster_f32(st_m + rr * 4, r));
-            float L = 0.f, acc[DH / 32];
+            float mr[8], lr[8];
 #pragma unroll
-            for (int k = 0; k < DH / 32; ++k) acc[k] = 0.f;
-            for (int r = 0; r < C; ++r) {
-                const float lr = ptx::ld_cluster_f32(st_l + rr * 4, r);
-                if (!(lr > 0.f)) continue;
-                const float f = exp2f(ptx::ld_cluster_f32(st_m + rr * 4, r) - M);
-                L += lr * f;
-#pragma unroll
-                for (int k = 0; k < DH / 32; ++k) acc[k] += f * ptx::ld_cluster_f32(st_rows + (rr * SROW + lane + 32 * k) * 4, r);
+            for (int r = 0; r < 8; ++r) {
+                mr[r] = -CUDART_INF_F; lr[r] = 0.f;
+                if (r < C) {
+                    const float2 ml = *reinterpret_cast<const float2 *>(recv + (size_t)(r * rows_per + rl) * RS + DH);
+                    mr[r] = ml.x; lr[r] = ml.y;
+                }
             }
-            float *dst = p.partials + ((size_t)i * p.Hq + (size_t)h * G + rr % G) * (DH + 2);
+            float M = -CUDART_INF_F;
 #pragma unroll
-            for (int k = 0; k < DH / 32; ++k) dst[lane + 32 * k] = acc[k];
-            if (lane == 0) { dst[DH] = M; dst[DH + 1] = L; }
+            for (int r = 0; r < 8; ++r)
+                if (lr[r] > 0.f) M = fmaxf(M, mr[r]);
+            float L = 0.f;
+            float4 acc[DH / 128 > 0 ? DH / 128 : 1];
+#pragma unroll
+            for (int k = 0; k < (DH + 127) / 128; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r >= C || !(lr[r] > 0.f)) continue;
+                const float f = exp2f(mr[r] - M);
+                L += lr[r] * f;
+#pragma unroll
+                for (int k = 0; k < (DH + 127) / 128; ++k) {
+                    if (4 * lane + 128 * k < DH) {
+                        const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(r * rows_per + rl) * RS + 4 * lane + 128 * k);
+                        acc[k].x += f * v.x; acc[k].y += f * v.y; acc[k].z += f * v.z; acc[k].w += f * v.w;
+                    }
+                }
+            }
+            float *out = p.partials + ((size_t)i * p.Hq + (size_t)h * G + rr % G) * (DH + 2);
+#pragma unroll
+            for (int k = 0; k < (DH + 127) / 128; ++k) {
+                if (4 * lane + 128 * k < DH) {
+                    *reinterpret_cast<float2 *>(out + 4 * lane + 128 * k) = make_float2(acc[k].x, acc[k].y);
+                    *reinterpret_cast<float2 *>(out + 4 * lane + 128 * k + 2) = make_float2(acc[k].z, acc[k].w);
+                }
+            }
+            if (lane == 0) { out[DH] = M; out[DH + 1] = L; }
         }
     }
-    ptx::cluster_sync();                                           // nobody reads this CTA's shared memory any more
+    ptx::cluster_sync();                                           // every copy out of this CTA's staging area has landed
     if (warp == 5) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, T::TMEM_COLS);
