@@ -168,6 +168,7 @@ chunk_attn_kernel(const AttnParams p) {
 template <int DH, int RP, int GT>
 cudaError_t launch(const AttnParams &p, cudaStream_t st, long long *launches) {
     const long long items = (long long)p.n_q * p.Hkv;
+    // a plain launch: with thousands of CTAs in many waves an early start only parks CTAs on the SMs
     chunk_attn_kernel<DH, RP, GT><<<(unsigned)((items + CH_WARPS - 1) / CH_WARPS), CH_WARPS * 32, 0, st>>>(p);
     ++*launches;
     return cudaGetLastError();

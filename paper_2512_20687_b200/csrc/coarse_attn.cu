@@ -298,11 +298,14 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
     }
 
+    ptx::grid_dep_wait();                   // lengths, caches and queries may come from the kernel before this one
+    ptx::grid_dep_launch();                 // one wave of CTAs, all resident: the next kernel may line up behind them
+
     // ---- where this CTA's share of the tile sequence starts: block-wide prefix sum of tile counts
     const int per = (p.n_units + THREADS - 1) / THREADS;
     const int ub = min(p.n_units, (int)threadIdx.x * per), ue = min(p.n_units, ub + per);
     int mine = 0;
-    for (int u = ub; u < ue; ++u) mine += tiles_of(clamp_len(p.len[u], p.cap));
+    for (int u = ub; u < ue; ++u) mine += tiles_of(clamp_len(__ldg(p.len + u), p.cap));
     int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -334,7 +337,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             if (!(lo <= x && x < hi)) continue;
             long long pre = lo;
             for (int u = ub; u < ue; ++u) {
-                const int len = clamp_len(p.len[u], p.cap);
+                const int len = clamp_len(__ldg(p.len + u), p.cap);
                 const int nt = tiles_of(len);
                 const long long k = (long long)nt * p.Hkv;
                 if (x < pre + k) {
@@ -361,13 +364,19 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const long long t0 = cta < n_cta ? sc[12] : 0;
     const long long t1 = cta < n_cta ? (sc[14] >= 0 ? sc[14] : T) : 0;
 
-    // ---- units without own keys are visited by no tile: finish them here
-    for (int u = cta; u < p.n_units; u += gridDim.x) {
-        if (clamp_len(p.len[u], p.cap) != 0) continue;
-        for (int idx = threadIdx.x; idx < p.Hq * DH; idx += THREADS)
-            emit<DH>(p, u, idx / DH, idx % DH, 0.f, -CUDART_INF_F, 0.f);
+    // ---- units without own keys are visited by no tile: they are finished by whoever has time for it
+    // (the whole CTA when it has no tiles, else the finishing warp before its first stream arrives)
+    auto finish_empty_units = [&](int tid, int nthreads) {
+        for (int u = cta; u < p.n_units; u += gridDim.x) {
+            if (clamp_len(__ldg(p.len + u), p.cap) != 0) continue;
+            for (int idx = tid; idx < p.Hq * DH; idx += nthreads)
+                emit<DH>(p, u, idx / DH, idx % DH, 0.f, -CUDART_INF_F, 0.f);
+        }
+    };
+    if (t0 >= t1) {
+        finish_empty_units(threadIdx.x, THREADS);
+        return;
     }
-    if (t0 >= t1) return;
 
     const int n_tiles = (int)(t1 - t0);
 
@@ -378,6 +387,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         constexpr int lpr = 32 / GP;                    // lanes per query head
         const int r = lane / lpr, d0 = (lane % lpr) * MAXV;
         const bool row_ok = r < G, lead = row_ok && (lane % lpr == 0);
+        finish_empty_units(lane, 32);
         // it walks the streams of this CTA in the consumers' order, one step ahead of them
         Walker fw;
         fw.u = sc[8]; fw.len = sc[10]; fw.nt = tiles_of(fw.len);
@@ -638,9 +648,9 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     mv = *t;
     const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
     const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, ctx->max_ctas));
-    coarse_attn_kernel<DH, GP><<<grid, THREADS, smem, st>>>(p, mk, mv);
+    const cudaError_t e = launch_dependent(coarse_attn_kernel<DH, GP>, dim3(grid), dim3(THREADS), smem, st, 0, p, mk, mv);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

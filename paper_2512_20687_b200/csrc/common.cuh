@@ -77,6 +77,33 @@ struct ConvParams {
     int32_t *status;
 };
 
+// Launch with programmatic stream serialization (and, optionally, a cluster width): the kernel's launch
+// latency and its set-up before grid_dep_wait() overlap the tail of the kernel before it in the stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    int cluster_x, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 0) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // launchers: enqueue on `st`, add the number of kernels launched to *launches,
 // return the launch error (cudaSuccess when fine)
 cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,

@@ -81,6 +81,8 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    ptx::grid_dep_wait();                   // x may be the output of the kernel before this one
+    ptx::grid_dep_launch();                 // at most one CTA per SM and one wave
 
     if (warp == 0) {
         int s = 0;
@@ -219,9 +221,9 @@ cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launc
     if (!t) return cudaErrorInvalidValue;
     mw = *t;
     dim3 grid(p.N / NT, (p.B + BM - 1) / BM);
-    converter_umma_kernel<NT, IN_MAJOR><<<grid, CONV_THREADS, T::SMEM, st>>>(p, mx, mw);
+    const cudaError_t e = launch_dependent(converter_umma_kernel<NT, IN_MAJOR>, grid, dim3(CONV_THREADS), T::SMEM, st, 0, p, mx, mw);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

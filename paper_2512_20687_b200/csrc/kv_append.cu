@@ -1,6 +1,7 @@
 // KV-cache append: the cache half of the streaming update STEP (Eq. 12, Eq. 13).
 // A bit copy of n_rows new rows per unit plus the length update.
 #include "common.cuh"
+#include "ptx.cuh"
 
 // One CTA per appended item.  Every thread reads len[u] before the CTA-wide
 // barrier and only thread 0 writes it after, and unit ids within a call are
@@ -11,6 +12,7 @@ kv_append_kernel(uint4 *__restrict__ k, uint4 *__restrict__ v, int32_t *__restri
                  const uint4 *__restrict__ v_new, const int32_t *__restrict__ unit_ids, int n_rows,
                  int32_t *__restrict__ status) {
     const int i = blockIdx.x;
+    ptx::grid_dep_wait();
     const int u = unit_ids ? unit_ids[i] : i;
     if (u < 0 || u >= n_units) {
         if (threadIdx.x == 0) atomicOr(status, PHOTON_DEV_BAD_INDEX);
@@ -39,9 +41,9 @@ cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hk
                              const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
                              int n_rows, int32_t *status, cudaStream_t st, long long *launches) {
     if (n == 0) return cudaSuccess;
-    kv_append_kernel<<<n, 128, 0, st>>>((uint4 *)k, (uint4 *)v, len, n_units, Hkv, cap, dh / 8,
+    const cudaError_t e = launch_dependent(kv_append_kernel, dim3(n), dim3(128), 0, st, 0, (uint4 *)k, (uint4 *)v, len, n_units, Hkv, cap, dh / 8,
                                         (const uint4 *)k_new, (const uint4 *)v_new, unit_ids, n_rows,
                                         status);
     ++*launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -116,6 +116,13 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---- programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor in the stream still runs.  grid_dep_wait() returns once the predecessor
+// has completed and its writes are visible (a no-op under a plain launch): every access to global memory
+// comes after it.  grid_dep_launch() lets the successor begin to launch.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- thread-block clusters: barrier over all threads of all CTAs, loads from a peer CTA's shared memory
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");

@@ -106,6 +106,8 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         ptx::mbar_arrive_expect_tx(recv_bar, BM * (DH + 4) * 4);
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
+    ptx::grid_dep_wait();                      // queries may come from the kernel before this one
+    ptx::grid_dep_launch();                    // one wave: the kernel for the units' own keys may line up
     // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch); row r = (unit - unit0) * G + g
     for (int r = threadIdx.x; r < BM; r += SP_THREADS) {
         const int i = unit0 + r / G;
@@ -484,19 +486,8 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     mks = *t;
     if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mvs = *t;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(groups * p.Hkv * p.splits_sh);
-    cfg.blockDim = dim3(SP_THREADS);
-    cfg.dynamicSmemBytes = T::SMEM;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;          // the key ranges of a row tile form a cluster
-    attr[0].val.clusterDim.x = p.splits_sh;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, shared_prefix_kernel<DH>, p, mks, mvs);
+    const cudaError_t e = launch_dependent(shared_prefix_kernel<DH>, dim3(groups * p.Hkv * p.splits_sh), dim3(SP_THREADS), T::SMEM, st,
+                                           p.splits_sh /* the key ranges of a row tile form a cluster */, p, mks, mvs);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
