@@ -160,7 +160,13 @@ photon_status photon_chunk_attn(photon_ctx *ctx, const photon_kv *chunks, const 
  * NULL, on out_coarse viewed as [B, Hq*dh] (requires Hq*dh == D and
  * B == coarse->n_units); chunk attention of q_chunk over `chunks`.
  * ev_attn_begin / ev_attn_end, when not NULL, are recorded on the stream
- * around the coarse attention launches (for timing that part in place). */
+ * around the coarse attention launches (for timing that part in place).
+ * For the caller everything is ordered on `stream`.  Inside, a small chunk
+ * workload runs beside the other parts on a low-priority stream of the
+ * context that forks from `stream` when the call starts and joins it before
+ * the call's work ends (it shares no data with them).  A context serves one
+ * stream at a time: its workspace, tickets and this side stream are not
+ * meant for concurrent calls. */
 typedef struct {
   photon_kv *coarse;
   const photon_bf16 *k_new, *v_new, *q_coarse;

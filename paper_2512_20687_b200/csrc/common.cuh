@@ -39,6 +39,8 @@ struct photon_ctx {
     size_t n_tickets;
     int32_t *status;         // device status word
     long long launches;
+    cudaStream_t side;       // lowest-priority stream for the chunk attention of a decode step
+    cudaEvent_t ev_fork, ev_join;
     TmapCache tmaps;
 };
 

@@ -133,6 +133,15 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
         delete ctx;
         return PHOTON_ERR_CUDA;
     }
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, lo) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        photon_destroy(ctx);
+        cudaGetLastError();
+        return PHOTON_ERR_CUDA;
+    }
     *out = ctx;
     return PHOTON_OK;
 }
@@ -143,6 +152,9 @@ photon_status photon_destroy(photon_ctx *ctx) {
     cudaFree(ctx->cta_partials);
     cudaFree(ctx->tickets);
     cudaFree(ctx->status);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
     return PHOTON_OK;
 }
@@ -234,22 +246,35 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, pho
             return PHOTON_ERR_INVALID_ARG;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    photon_status s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr,
-                                       a->coarse->n_units, 1, stream);
-    if (s != PHOTON_OK) return s;
-    if (a->ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_begin), st) != cudaSuccess)
-        return PHOTON_ERR_CUDA;
-    s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse,
-                           a->scale_coarse, stream);
-    if (s != PHOTON_OK) return s;
-    if (a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
-        return PHOTON_ERR_CUDA;
-    s = photon_converter(ctx, chain ? a->out_coarse : a->x, a->w, a->w_layout, a->bias, a->U, a->B,
-                         stream);
-    if (s != PHOTON_OK) return s;
-    if (a->Nc > 0)
-        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc,
-                              a->scale_chunk, stream);
+    // The chunk attention shares no data with the other parts (the decoders' projections, which are not
+    // built, sit between the converter's output and the chunk caches): it runs beside them on a
+    // low-priority stream that forks from `stream` here and joins it again before the call returns, so
+    // for the caller the whole step is still ordered on `stream`.  Large chunk workloads stay in line:
+    // two kernels that are both bound by HBM gain nothing from running side by side.
+    const bool beside = a->Nc > 0 &&
+                        (size_t)a->Nc * c.Hkv * a->chunks->cap * c.dh * 4 <= (size_t(32) << 20);
+    photon_status s = PHOTON_OK;
+    if (beside) {
+        if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+            return PHOTON_ERR_CUDA;
+        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, ctx->side);
+        if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return PHOTON_ERR_CUDA;
+        if (s != PHOTON_OK) { cudaStreamWaitEvent(st, ctx->ev_join, 0); return s; }
+    }
+    s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr, a->coarse->n_units, 1, stream);
+    if (s == PHOTON_OK && a->ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_begin), st) != cudaSuccess)
+        s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK)
+        s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse, a->scale_coarse, stream);
+    if (s == PHOTON_OK && a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
+        s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK)
+        s = photon_converter(ctx, chain ? a->out_coarse : a->x, a->w, a->w_layout, a->bias, a->U, a->B, stream);
+    if (beside) {
+        if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess && s == PHOTON_OK) s = PHOTON_ERR_CUDA;
+    } else if (s == PHOTON_OK && a->Nc > 0) {
+        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, stream);
+    }
     return s;
 }
 
