@@ -6,10 +6,10 @@
 //
 // CTA = (tile of 128 query rows = 128/G units x G heads, KV head, key range of
 // the prefix).  Per 128-key tile:  S = Q K^T (tcgen05.mma, both operands
-// K-major from 128B-swizzled shared memory, S in TMEM);  four softmax warps read
-// their rows of S with tcgen05.ld (one thread = one query row), turn them into
-// probabilities in the base-2 domain and store them as bf16 into a swizzled
-// shared-memory tile P;  O += P V (tcgen05.mma, V as the N-major operand
+// K-major from 128B-swizzled shared memory, S in TMEM);  eight softmax warps read
+// S with tcgen05.ld (two threads share a query row, 64 keys each, and exchange
+// their maxima through shared memory), turn it into probabilities in the base-2
+// domain and store them as bf16 into a swizzled shared-memory tile P;  O += P V (tcgen05.mma, V as the N-major operand
 // straight from its TMA tile, O in TMEM across all tiles).  S is double
 // buffered, so the tensor pipe computes the next S while the warps work on this
 // one.  The reference maximum of a row is only raised when a tile exceeds it by
@@ -34,7 +34,8 @@ namespace {
 constexpr int BM = 128;                    // query rows per CTA (UMMA M; one TMEM lane each)
 constexpr int BN = 128;                    // keys per tile
 constexpr int KV_STAGES = 2;
-constexpr int SP_THREADS = 192;            // warps 0-3: softmax (TMEM lane quadrant = warp), 4: TMA, 5: MMA + TMEM owner
+constexpr int SW = 8;                      // softmax warps: warp w works on TMEM lanes 32*(w%4).., keys 64*(w/4)..
+constexpr int SP_THREADS = (SW + 2) * 32;  // + TMA warp (8) + MMA warp and TMEM owner (9)
 constexpr float RESCALE_GAP = 8.f;         // log2 of the largest factor P may carry
 
 template <int DH>
@@ -47,7 +48,9 @@ struct SpTile {
     static constexpr int OFF_K = OFF_P + P_BYTES;
     static constexpr int OFF_V = OFF_K + KV_STAGES * KV_BYTES;
     static constexpr int OFF_TAIL = OFF_V + KV_STAGES * KV_BYTES;
-    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 /*barriers*/ + 64 /*scalars*/ + BM * 4 /*ids*/;
+    // after the tiles: barriers (256), scalars (64), prefix ids (BM ints), maxima exchange (2 x 2 x BM floats),
+    // sums exchange (2 x BM floats)
+    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 + 64 + BM * 4 + 4 * BM * 4 + 2 * BM * 4;
     static constexpr int TMEM_COLS = 512;                       // S0, S1 (128 each), O (DH): next power of two
     static constexpr int COL_O = 2 * BN;
 };
@@ -79,13 +82,17 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     const uint32_t p_ready = bars + 80, p_free = bars + 88, recv_bar = bars + 96;
     int *sc = reinterpret_cast<int *>(gen + T::OFF_TAIL + 256);                  // [0] tmem base, [1..2] rescale flags
     int *sid = sc + 16;                                                          // [BM] prefix id per query row's unit
+    float *xch_m = reinterpret_cast<float *>(sid + BM);                          // [2 tiles in flight][2 halves][BM]
+    float *xch_l = xch_m + 4 * BM;                                               // [2 halves][BM]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = p.Hq / p.Hkv;
     const int upt = BM / G;                                                      // units per tile
-    const int part = blockIdx.x % p.splits_sh;
+    const int part = blockIdx.x % p.splits_sh;                                   // = rank in the cluster
     const int h = (blockIdx.x / p.splits_sh) % p.Hkv;
     const int unit0 = (blockIdx.x / (p.splits_sh * p.Hkv)) * upt;
+    constexpr int RS = DH + 4;                                                   // floats per staged row (16-byte aligned)
+    const int C = p.splits_sh, rows_per = BM / C;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < KV_STAGES; ++s) {
@@ -95,15 +102,16 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(s_ready + 8 * b, 1);
-            ptx::mbar_init(s_free + 8 * b, 4);
+            ptx::mbar_init(s_free + 8 * b, SW);
         }
-        ptx::mbar_init(p_ready, 4);
+        ptx::mbar_init(p_ready, SW);
         ptx::mbar_init(p_free, 1);
         ptx::mbar_init(recv_bar, 1);
         sc[1] = 0; sc[2] = 0;
         ptx::mbar_fence_init();
-        // the rows this CTA owns arrive from every CTA of its cluster (itself included) at the very end
-        ptx::mbar_arrive_expect_tx(recv_bar, BM * (DH + 4) * 4);
+        // the rows this CTA owns arrive from the other CTAs of its cluster at the very end
+        if (C > 1) ptx::mbar_arrive_expect_tx(recv_bar, (C - 1) * rows_per * RS * 4);
+        else ptx::mbar_arrive(recv_bar);
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
     ptx::grid_dep_wait();                      // queries may come from the kernel before this one
@@ -121,13 +129,13 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     __syncthreads();                           // barriers and ids are ready: the TMA warp starts loading at once
 
     uint32_t tmem = 0;
-    if (warp != 4) {
-        if (warp == 5) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
+    if (warp != SW) {
+        if (warp == SW + 1) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
         // the Q tile, stored K-major with the 128-byte swizzle TMA would use; all of a thread's loads are
         // issued before its first store: one round trip to memory, not one per chunk
         constexpr int NQT = SP_THREADS - 32;
         constexpr int QV = (BM * (DH / 8) + NQT - 1) / NQT;
-        const int tq = threadIdx.x < 128 ? threadIdx.x : threadIdx.x - 32;
+        const int tq = threadIdx.x < SW * 32 ? threadIdx.x : threadIdx.x - 32;
         uint4 qv[QV];
 #pragma unroll
         for (int t = 0; t < QV; ++t) {
@@ -167,7 +175,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     float fin_m = -CUDART_INF_F, fin_l = 0.f;
     bool fin_have = false, fin_any = false;
 
-    if (warp == 4) {
+    if (warp == SW) {
         // ======================= TMA warp =======================
         int it = 0;
         bool ok = true;
@@ -195,7 +203,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 __syncwarp();
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == SW + 1) {
         // ======================= MMA warp =======================
         constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(BM, BN, false, false);
         constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(BM, DH, false, true);
@@ -248,120 +256,125 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
     } else {
-        // ======================= softmax warps: thread = query row =======================
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // ======================= softmax warps: two threads per query row =======================
+        const int quad = warp & 3, hf = warp >> 2;                 // TMEM lane quadrant; which 64 keys of a tile
+        const int row = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const int my_sid = sid[row];
-        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        constexpr int CH = BN / 2;                                 // keys per thread and tile
+        float m_ref = -CUDART_INF_F, l_half = 0.f;                 // m_ref is kept identical in both threads of a row
         int it = 0;
         bool ok = true;
-        // After a wait has run out (ok = false) the loop goes on without waiting, so that the four
-        // warps keep meeting at the named barrier; the results are then void and the status says so.
+        // After a wait has run out (ok = false) the loop goes on without waiting, so that the warps
+        // keep meeting at the named barrier; the results are then void and the status says so.
         for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
             int r0, r1;
             part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
             const bool active = (my_sid == cur);
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int b = it & 1, st = it % KV_STAGES;
-                const int nvalid = min(BN, r1 - k0);
+                const int nvalid = min(BN, r1 - k0) - hf * CH;     // keys of my half that are in range (may be <= 0)
                 if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(s_ready + 8 * b, (it >> 1) & 1))) ok = false;
                 ptx::tc_fence_after();
-                uint32_t sr[BN];
+                uint32_t sr[CH];
 #pragma unroll
-                for (int c0 = 0; c0 < BN; c0 += 32)
-                    ptx::tmem_ld_32x32(tmem + lane_base + b * BN + c0, *reinterpret_cast<uint32_t(*)[32]>(&sr[c0]));
+                for (int c0 = 0; c0 < CH; c0 += 32)
+                    ptx::tmem_ld_32x32(tmem + lane_base + b * BN + hf * CH + c0, *reinterpret_cast<uint32_t(*)[32]>(&sr[c0]));
                 ptx::tmem_ld_wait();
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(s_free + 8 * b);          // the tensor pipe may overwrite this S
 
                 float mx = -CUDART_INF_F;
-                if (nvalid == BN) {
+                if (nvalid >= CH) {
 #pragma unroll
-                    for (int c = 0; c < BN; ++c) {
+                    for (int c = 0; c < CH; ++c) {
                         const float v = __uint_as_float(sr[c]) * p.scale_log2;
                         sr[c] = __float_as_uint(v);
                         mx = fmaxf(mx, v);
                     }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < BN; ++c) {
+                    for (int c = 0; c < CH; ++c) {
                         const float v = c < nvalid ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
                         sr[c] = __float_as_uint(v);
                         mx = fmaxf(mx, v);
                     }
                 }
+                // the two threads of a row exchange their maxima; a row whose maximum outgrows its reference
+                // by more than the gap makes the whole CTA rescale its accumulators
+                xch_m[(b * 2 + hf) * BM + row] = mx;
+                if (active && m_ref != -CUDART_INF_F && mx > m_ref + RESCALE_GAP) sc[1 + b] = 1;
+                ptx::named_bar_sync(1, SW * 32);
+                mx = fmaxf(mx, xch_m[(b * 2 + (hf ^ 1)) * BM + row]);
+                const bool rescale = sc[1 + b] != 0;
                 float corr = 1.f;
-                bool need = false;
                 if (active) {
                     if (m_ref == -CUDART_INF_F) {
                         m_ref = mx;                                        // nothing accumulated for this row yet
                     } else if (mx > m_ref + RESCALE_GAP) {
                         corr = exp2f(m_ref - mx);
                         m_ref = mx;
-                        need = true;
                     }
                 }
-                // does any row of the CTA have to rescale its accumulator?
-                if (need) sc[1 + b] = 1;
-                ptx::named_bar_sync(1, 128);
-                const bool rescale = sc[1 + b] != 0;
                 // the previous P V must be done before P is overwritten (and before O is touched)
                 if (ok && it > 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1))) ok = false;
                 if (rescale) {
                     ptx::tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < DH; c0 += 32) {
+                    for (int c0 = 0; c0 < DH / 2; c0 += 32) {              // my half of the row's accumulator
                         uint32_t orow[32];
-                        ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
+                        ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + hf * (DH / 2) + c0, orow);
                         ptx::tmem_ld_wait();
 #pragma unroll
                         for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * corr);
-                        ptx::tmem_st_32x32(tmem + lane_base + T::COL_O + c0, orow);
+                        ptx::tmem_st_32x32(tmem + lane_base + T::COL_O + hf * (DH / 2) + c0, orow);
                     }
                     ptx::tmem_st_wait();
-                    l_sum *= corr;
-                    ptx::named_bar_sync(1, 128);                           // every reader of the flag is past it
+                    l_half *= corr;
+                    ptx::named_bar_sync(1, SW * 32);                       // every reader of the flag is past it
                     if (threadIdx.x == 0) sc[1 + b] = 0;
                 }
                 // rows of V past the end of the range may hold anything: clear them (P is 0 there, 0 * NaN is not)
-                if (nvalid < BN) {
+                const int tile_valid = min(BN, r1 - k0);
+                if (tile_valid < BN) {
                     if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
-                    for (int idx = threadIdx.x; idx < (BN - nvalid) * T::HALVES * 8; idx += 128) {
-                        const int r = nvalid + idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
+                    for (int idx = threadIdx.x; idx < (BN - tile_valid) * T::HALVES * 8; idx += SW * 32) {
+                        const int r = tile_valid + idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
                         ptx::sts128(sV + st * T::KV_BYTES + (c16 >> 3) * (BN * 128) + r * 128 + ((c16 & 7) << 4),
                                     make_uint4(0u, 0u, 0u, 0u));
                     }
                 }
-                // probabilities of this row, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
+                // probabilities of my 64 keys, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
                 float ls = 0.f;
+                const uint32_t prow = sP + hf * (BM * 128) + row * 128;
                 if (active) {
 #pragma unroll
-                    for (int ch = 0; ch < BN / 8; ++ch) {
+                    for (int ch = 0; ch < CH / 8; ++ch) {
                         float e[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             e[j] = exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref);
                             ls += e[j];
                         }
-                        const uint4 v = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]),
-                                                   pack_bf16(e[6], e[7]));
-                        ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4), v);
+                        ptx::sts128(prow + ((ch ^ (row & 7)) << 4),
+                                    make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])));
                     }
                 } else {
 #pragma unroll
-                    for (int ch = 0; ch < BN / 8; ++ch)
-                        ptx::sts128(sP + (ch >> 3) * (BM * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4),
-                                    make_uint4(0u, 0u, 0u, 0u));
+                    for (int ch = 0; ch < CH / 8; ++ch) ptx::sts128(prow + ((ch ^ (row & 7)) << 4), make_uint4(0u, 0u, 0u, 0u));
                 }
-                l_sum += ls;
+                l_half += ls;
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(p_ready);
             }
         }
-        // ---- the partial of this row: accumulator relative to m_ref, m_ref, running sum
+        // ---- what the row carries out: reference maximum and the sum over both halves
+        xch_l[hf * BM + row] = l_half;
+        ptx::named_bar_sync(1, SW * 32);
+        const float l_sum = l_half + xch_l[(hf ^ 1) * BM + row];
         if (ok && it > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1));
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
@@ -373,20 +386,18 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
 
     // ---- the key ranges of one row tile are the CTAs of one cluster.  Each CTA stages its rows
     // (acc, m, l) in its own shared memory; when every CTA of the cluster is done with its tile buffers,
-    // one bulk copy per owner moves the rows a peer owns into that peer's receive buffer (completion
-    // counted on the peer's mbarrier); every CTA then merges the rows it owns by log-sum-exp from its own
-    // shared memory and writes one partial per query head.
-    constexpr int RS = DH + 4;                                     // floats per staged row: 16-byte aligned rows
-    const int C = p.splits_sh, rows_per = BM / C;
+    // one bulk copy per peer moves the rows that peer owns into its receive buffer (completion counted on
+    // the peer's mbarrier); every CTA then merges the rows it owns by log-sum-exp from its own shared
+    // memory and writes one partial per query head.
     const uint32_t stage_a = base, recv_a = base + BM * RS * 4;    // stage [BM][RS]; receive [C sources][rows_per][RS]
-    if (warp < 4) {
+    if (warp < SW) {
         // every MMA and every load of this CTA is done, so its tile buffers can serve as the staging area
-        ptx::tc_fence_after();
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const int quad = warp & 3, hf = warp >> 2;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float *stage = reinterpret_cast<float *>(gen) + (size_t)row * RS;
 #pragma unroll 1
-        for (int c0 = 0; c0 < DH; c0 += 32) {
+        for (int c0 = hf * (DH / 2); c0 < (hf + 1) * (DH / 2); c0 += 32) {
             uint32_t orow[32];
             if (fin_any) {                                                  // O was written by at least one P V
                 ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
@@ -399,59 +410,69 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                                            __uint_as_float(orow[e + 3]))
                              : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        *reinterpret_cast<float4 *>(stage + DH) =
-            make_float4(fin_have ? fin_m : -CUDART_INF_F, fin_have ? fin_l : 0.f, 0.f, 0.f);
+        if (hf == 0)
+            *reinterpret_cast<float4 *>(stage + DH) =
+                make_float4(fin_have ? fin_m : -CUDART_INF_F, fin_have ? fin_l : 0.f, 0.f, 0.f);
         ptx::fence_proxy_async();                                  // the bulk copies below read what was staged here
     }
     ptx::tc_fence_before();
     ptx::cluster_sync();                                           // staged everywhere; receive buffers are free
-    if (warp == 4 && ptx::elect_one()) {
+    if (warp == SW && ptx::elect_one()) {
         const uint32_t bytes = rows_per * RS * 4;
         for (int o = 0; o < C; ++o)
-            ptx::bulk_copy_to_peer(ptx::map_cluster(recv_a + part * bytes, o), stage_a + o * bytes, bytes,
-                                   ptx::map_cluster(recv_bar, o));
+            if (o != part)
+                ptx::bulk_copy_to_peer(ptx::map_cluster(recv_a + part * bytes, o), stage_a + o * bytes, bytes,
+                                       ptx::map_cluster(recv_bar, o));
     }
     const bool got = ptx::mbar_wait(recv_bar, 0);                  // the rows this CTA owns are all here
     if (!got && threadIdx.x == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
     {
-        const float *recv = reinterpret_cast<const float *>(gen) + BM * RS;
+        const float *stage = reinterpret_cast<const float *>(gen);
+        const float *recv = stage + BM * RS;
         for (int rl = warp; rl < rows_per; rl += SP_THREADS / 32) {
             const int rr = part * rows_per + rl;
             const int i = unit0 + rr / G;
             if (rr >= upt * G || i >= p.n_q) continue;
-            float mr[8], lr[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                mr[r] = -CUDART_INF_F; lr[r] = 0.f;
-                if (r < C) {
-                    const float2 ml = *reinterpret_cast<const float2 *>(recv + (size_t)(r * rows_per + rl) * RS + DH);
-                    mr[r] = ml.x; lr[r] = ml.y;
-                }
-            }
+            const float *src[8];
+            float f[8];
             float M = -CUDART_INF_F;
 #pragma unroll
-            for (int r = 0; r < 8; ++r)
-                if (lr[r] > 0.f) M = fmaxf(M, mr[r]);
+            for (int r = 0; r < 8; ++r) {
+                src[r] = r == part ? stage + (size_t)rr * RS : recv + (size_t)(r * rows_per + rl) * RS;
+                f[r] = -CUDART_INF_F;
+                if (r < C) {
+                    const float2 ml = *reinterpret_cast<const float2 *>(src[r] + DH);
+                    if (ml.y > 0.f) { f[r] = ml.x; M = fmaxf(M, ml.x); }
+                }
+            }
             float L = 0.f;
-            float4 acc[DH / 128 > 0 ? DH / 128 : 1];
-#pragma unroll
-            for (int k = 0; k < (DH + 127) / 128; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
-                if (r >= C || !(lr[r] > 0.f)) continue;
-                const float f = exp2f(mr[r] - M);
-                L += lr[r] * f;
+                const float l = r < C ? src[r][DH + 1] : 0.f;
+                f[r] = f[r] > -CUDART_INF_F ? exp2f(f[r] - M) : 0.f;      // weight of source r (0: nothing there)
+                L += l * f[r];
+            }
+            constexpr int NK = (DH + 127) / 128;
+            float4 acc[NK];
 #pragma unroll
-                for (int k = 0; k < (DH + 127) / 128; ++k) {
-                    if (4 * lane + 128 * k < DH) {
-                        const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(r * rows_per + rl) * RS + 4 * lane + 128 * k);
-                        acc[k].x += f * v.x; acc[k].y += f * v.y; acc[k].z += f * v.z; acc[k].w += f * v.w;
+            for (int k = 0; k < NK; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            const bool mine = 4 * lane < DH || NK > 1;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r < C) {
+#pragma unroll
+                    for (int k = 0; k < NK; ++k) {
+                        if (4 * lane + 128 * k < DH) {
+                            const float4 v = *reinterpret_cast<const float4 *>(src[r] + 4 * lane + 128 * k);
+                            acc[k].x += f[r] * v.x; acc[k].y += f[r] * v.y; acc[k].z += f[r] * v.z; acc[k].w += f[r] * v.w;
+                        }
                     }
                 }
             }
+            (void)mine;
             float *out = p.partials + ((size_t)i * p.Hq + (size_t)h * G + rr % G) * (DH + 2);
 #pragma unroll
-            for (int k = 0; k < (DH + 127) / 128; ++k) {
+            for (int k = 0; k < NK; ++k) {
                 if (4 * lane + 128 * k < DH) {
                     *reinterpret_cast<float2 *>(out + 4 * lane + 128 * k) = make_float2(acc[k].x, acc[k].y);
                     *reinterpret_cast<float2 *>(out + 4 * lane + 128 * k + 2) = make_float2(acc[k].z, acc[k].w);
@@ -461,7 +482,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         }
     }
     ptx::cluster_sync();                                           // every copy out of this CTA's staging area has landed
-    if (warp == 5) {
+    if (warp == SW + 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, T::TMEM_COLS);
     }
