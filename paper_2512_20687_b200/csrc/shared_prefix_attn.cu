@@ -35,7 +35,7 @@ constexpr int BM = 128;                    // query rows per CTA (UMMA M; one TM
 constexpr int BN = 128;                    // keys per tile
 constexpr int KV_STAGES = 2;
 constexpr int SW = 8;                      // softmax warps: warp w works on TMEM lanes 32*(w%4).., keys 64*(w/4)..
-constexpr int SP_THREADS = (SW + 2) * 32;  // + TMA warp (8) + MMA warp and TMEM owner (9)
+constexpr int SP_THREADS = (SW + 3) * 32;  // + K loader (8) + MMA warp and TMEM owner (9) + V loader (10)
 constexpr float RESCALE_GAP = 8.f;         // log2 of the largest factor P may carry
 
 template <int DH>
@@ -77,7 +77,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     const uint32_t sQ = base, sP = base + T::OFF_P, sK = base + T::OFF_K, sV = base + T::OFF_V;
     const uint32_t bars = base + T::OFF_TAIL;
     // barriers (8 bytes each)
-    const uint32_t k_full = bars, v_full = bars + 16, kv_empty = bars + 32;      // [KV_STAGES]
+    const uint32_t k_full = bars, v_full = bars + 16, k_empty = bars + 32, v_empty = bars + 112;   // [KV_STAGES]
     const uint32_t s_ready = bars + 48, s_free = bars + 64;                      // [2]
     const uint32_t p_ready = bars + 80, p_free = bars + 88, recv_bar = bars + 96;
     int *sc = reinterpret_cast<int *>(gen + T::OFF_TAIL + 256);                  // [0] tmem base, [1..2] rescale flags
@@ -98,7 +98,8 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         for (int s = 0; s < KV_STAGES; ++s) {
             ptx::mbar_init(k_full + 8 * s, 1);
             ptx::mbar_init(v_full + 8 * s, 1);
-            ptx::mbar_init(kv_empty + 8 * s, 1);
+            ptx::mbar_init(k_empty + 8 * s, 1);
+            ptx::mbar_init(v_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(s_ready + 8 * b, 1);
@@ -129,11 +130,11 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     __syncthreads();                           // barriers and ids are ready: the TMA warp starts loading at once
 
     uint32_t tmem = 0;
-    if (warp != SW) {
+    if (warp != SW && warp != SW + 2) {
         if (warp == SW + 1) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
         // the Q tile, stored K-major with the 128-byte swizzle TMA would use; all of a thread's loads are
         // issued before its first store: one round trip to memory, not one per chunk
-        constexpr int NQT = SP_THREADS - 32;
+        constexpr int NQT = SP_THREADS - 64;
         constexpr int QV = (BM * (DH / 8) + NQT - 1) / NQT;
         const int tq = threadIdx.x < SW * 32 ? threadIdx.x : threadIdx.x - 32;
         uint4 qv[QV];
@@ -175,8 +176,13 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     float fin_m = -CUDART_INF_F, fin_l = 0.f;
     bool fin_have = false, fin_any = false;
 
-    if (warp == SW) {
-        // ======================= TMA warp =======================
+    if (warp == SW || warp == SW + 2) {
+        // ======================= the two loader warps: one for K tiles, one for V tiles =======================
+        // (separate rings: a K slot is free again as soon as its Q K^T is done, long before the V slot of
+        // the same tile, so the next K tile can be on its way a whole tile earlier)
+        const bool is_k = warp == SW;
+        const uint32_t full0 = is_k ? k_full : v_full, empty0 = is_k ? k_empty : v_empty, dst0 = is_k ? sK : sV;
+        const CUtensorMap *tm = is_k ? &tm_ks : &tm_vs;
         int it = 0;
         bool ok = true;
         for (int cur = next_sid(-1); cur != 0x7FFFFFFF && ok; cur = next_sid(cur)) {
@@ -185,20 +191,16 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
             const int row_base = (cur * p.Hkv + h) * p.cap_sh;
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int s = it % KV_STAGES;
-                if (!__all_sync(0xffffffffu, ptx::mbar_wait(kv_empty + 8 * s, ((it / KV_STAGES) & 1) ^ 1))) {
+                if (!__all_sync(0xffffffffu, ptx::mbar_wait(empty0 + 8 * s, ((it / KV_STAGES) & 1) ^ 1))) {
                     if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
                     ok = false;
                     break;                     // stop loading; the other warps run out on their own bounded waits
                 }
                 if (ptx::elect_one()) {
-                    ptx::mbar_arrive_expect_tx(k_full + 8 * s, T::KV_BYTES);
+                    ptx::mbar_arrive_expect_tx(full0 + 8 * s, T::KV_BYTES);
 #pragma unroll
                     for (int hh = 0; hh < T::HALVES; ++hh)
-                        ptx::tma_load_2d(sK + s * T::KV_BYTES + hh * (BN * 128), &tm_ks, hh * 64, row_base + k0, k_full + 8 * s);
-                    ptx::mbar_arrive_expect_tx(v_full + 8 * s, T::KV_BYTES);
-#pragma unroll
-                    for (int hh = 0; hh < T::HALVES; ++hh)
-                        ptx::tma_load_2d(sV + s * T::KV_BYTES + hh * (BN * 128), &tm_vs, hh * 64, row_base + k0, v_full + 8 * s);
+                        ptx::tma_load_2d(dst0 + s * T::KV_BYTES + hh * (BN * 128), tm, hh * 64, row_base + k0, full0 + 8 * s);
                 }
                 __syncwarp();
             }
@@ -228,6 +230,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                     ptx::umma_bf16(tmem + b * BN, a, bdesc, idesc_qk, ks != 0);
                 }
                 ptx::umma_commit(s_ready + 8 * b);
+                ptx::umma_commit(k_empty + 8 * s);             // this K tile has been read
             }
             __syncwarp();
             return true;
@@ -249,7 +252,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                     const uint64_t bdesc = ptx::umma_desc_sw128(sV + s * T::KV_BYTES + kk * (16 * 128), BN * 128, 1024);
                     ptx::umma_bf16(tmem + T::COL_O, a, bdesc, idesc_pv, (i | kk) != 0);
                 }
-                ptx::umma_commit(kv_empty + 8 * s);
+                ptx::umma_commit(v_empty + 8 * s);
                 ptx::umma_commit(p_free);
             }
             __syncwarp();
