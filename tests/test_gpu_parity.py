@@ -315,6 +315,30 @@ def test_chunk_attention_strict_positions_gather_and_bad_slots(oracle):
     assert_close(got, want, "chunk gather")
 
 
+@pytest.mark.parametrize("idx,B", [(1, 2048), (0, 1024)])
+def test_chunk_attention_large_batches_with_gather(oracle, idx, B):
+    """Thousands of chunks, grouped query heads, a gather through `slot` with one bad entry,
+    strict (prefix-only) positions and poisoned rows."""
+    cfg = cfg_small(idx, B=B)
+    ch = wl.chunk_inputs(cfg, poison=True, strict_paper=True)
+    scale = cfg.dh ** -0.5
+    slot = np.random.default_rng(idx).permutation(cfg.Nc).astype(np.int32)
+    slot[123] = -5
+    pick = np.sort(np.random.default_rng(9).choice(cfg.Nc, 400, replace=False))
+    pick[0] = 123
+    pick.sort()
+    want, _, flags = oracle.attention(ch["q"][pick], ch["kc"], ch["vc"], ch["len"], scale,
+                                      slot=slot[pick], n_threads=NT, want_flags=True)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        out = torch.full_like(d["q"], 3.0)
+        ph.photon_chunk_attn(c.h, d["kv"], d["q"], dev_i32(slot), out, scale=scale)
+        assert c.status() == flags == ph.PHOTON_DEV_BAD_INDEX
+    got = host_f64(out)
+    assert np.all(got[123] == 0)
+    assert_close(got[pick], want, "chunk gather, large batch")
+
+
 def test_chunk_attention_ignores_other_chunks_bit_exactly():
     cfg = cfg_small(4, B=2)
     ch = wl.chunk_inputs(cfg)
