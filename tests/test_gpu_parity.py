@@ -339,6 +339,49 @@ def test_chunk_attention_large_batches_with_gather(oracle, idx, B):
     assert_close(got[pick], want, "chunk gather, large batch")
 
 
+@pytest.mark.parametrize("dh,Hq,Hkv", [(128, 8, 2), (64, 6, 2), (64, 3, 3)])
+def test_chunk_attention_at_the_largest_window(oracle, dh, Hq, Hkv):
+    """P + C = 64, the widest window a context accepts (several passes over the rows), every length
+    from 0 to 64, group sizes 4, 3 and 1, poisoned rows past the end."""
+    cfg = cfg_small(4, B=5, chunks_per_seq=13, P=16, C=48, Hq=Hq, Hkv=Hkv, dh=dh, D=Hq * dh)
+    ch = wl.chunk_inputs(cfg, poison=True)
+    lens = (np.arange(cfg.Nc) % 65).astype(np.int32)
+    cap = cfg.P + cfg.C
+    bad = np.arange(cap)[None, :] >= lens[:, None]
+    ch["kc"][np.broadcast_to(bad[:, None, :, None], ch["kc"].shape)] = 0x7FC1
+    ch["vc"][np.broadcast_to(bad[:, None, :, None], ch["vc"].shape)] = 0xFFC1
+    # rows that are valid now but were poisoned by the generator: give them values again
+    fresh_k = wl.normal_bf16(11, "k", ch["kc"].shape)
+    fresh_v = wl.normal_bf16(12, "v", ch["vc"].shape)
+    ok = np.broadcast_to(~bad[:, None, :, None], ch["kc"].shape)
+    ch["kc"][ok] = fresh_k[ok]
+    ch["vc"][ok] = fresh_v[ok]
+    ch["len"] = lens
+    scale = cfg.dh ** -0.5
+    want, _ = oracle.chunk_attention(ch["q"], ch["kc"], ch["vc"], lens, scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        out = torch.full_like(d["q"], 5.0)
+        ph.photon_chunk_attn(c.h, d["kv"], d["q"], None, out, scale=scale)
+        assert c.status() == 0
+    got = host_f64(out)
+    assert np.all(got[lens == 0] == 0)
+    assert_close(got, want, f"chunk cap 64 dh={dh} G={Hq // Hkv}")
+
+
+def test_calls_larger_than_the_context_was_made_for_are_refused():
+    cfg = cfg_small(1, B=8, S=70)
+    co = wl.coarse_inputs(cfg)
+    with Ctx(cfg, max_queries=4) as c:
+        d = coarse_to_dev(co)
+        out = torch.empty_like(d["q"])
+        n0 = ph.photon_launch_count(c.h)
+        with pytest.raises(ph.PhotonError) as e:
+            ph.photon_coarse_attn(c.h, d["kv"], d["q"], out, None, 1.0)
+        assert e.value.code == ph.PHOTON_ERR_WORKSPACE
+        assert ph.photon_launch_count(c.h) == n0 and c.status() == 0
+
+
 def test_chunk_attention_ignores_other_chunks_bit_exactly():
     cfg = cfg_small(4, B=2)
     ch = wl.chunk_inputs(cfg)
