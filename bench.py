@@ -375,6 +375,41 @@ def run_gpu(args, cfg) -> None:
     parts["note"] = ("each part timed as a CUDA graph of back-to-back calls rotating over the replicas; "
                      "kv_append's figure includes a %d-int length reset every %d calls" % (cfg.B * R, R))
 
+    # what a flat Transformer and hierarchical generation (every level keeps a global cache) would read
+    # for the same context, measured with the same attention kernel: a token-level cache (context rows per
+    # sequence) through photon_flat_attn, and a level-1 cache (context / C1 rows) through photon_coarse_attn.
+    # These caches only feed a timing, so they are filled on the device from a fixed torch seed.
+    kv_measured = {}
+    if not args.no_parts and cfg.compress == 16:
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1234 + cfg.seed)
+        c1 = 4                                                   # C1 of the two-level hierarchy
+        for name, rows, fn in (("flat_token_level", cfg.context + cfg.shared_context, ph.photon_flat_attn),
+                               ("level1_global", (cfg.context + cfg.shared_context) // c1, ph.photon_coarse_attn)):
+            nbytes = cfg.B * cfg.Hkv * rows * cfg.dh * 2 * 2
+            if nbytes > (24 << 30):
+                continue
+            kk = torch.empty(cfg.B, cfg.Hkv, rows, cfg.dh, dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+            vv = torch.empty_like(kk).normal_(generator=gen)
+            ln = torch.full((cfg.B,), rows, dtype=torch.int32, device=dev)
+            kvf = ph.make_kv(kk, vv, ln, max_len=rows)
+            o2 = torch.empty_like(q)
+            for _ in range(2):
+                fn(ctx, kvf, q, o2, None, scale)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_rep = 5
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(n_rep):
+                fn(ctx, kvf, q, o2, None, scale)
+            b.record()
+            torch.cuda.synchronize()
+            us = a.elapsed_time(b) * 1e3 / n_rep
+            kv_measured[name] = {"rows_per_sequence": rows, "kv_bytes_per_step": nbytes, "us": us,
+                             "GBps": nbytes / us * 1e-3}
+            del kk, vv, kvf
+        torch.cuda.empty_cache()
+
     # roofline of the dominant kernel = the attention part that takes the longest
     dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
     traffic, traffic_note = None, "no ncu capture on record for this kernel and workload"
@@ -474,7 +509,14 @@ def run_gpu(args, cfg) -> None:
             "photon_coarse_per_step": coarse_bytes,
             "photon_per_token": coarse_bytes / cfg.compress / cfg.B + (chunk_bytes / cfg.Nc),
             "flat_per_token": wl.flat_kv_bytes(cfg) / cfg.B,
-            "note": "per sequence and layer; coarse step amortised over %d tokens" % cfg.compress},
+            "note": "per sequence and layer; coarse step amortised over %d tokens" % cfg.compress,
+            "measured": dict(kv_measured,
+                             recursive_top_level={"rows_per_sequence": cfg.S + cfg.shared_S, "kv_bytes_per_step": coarse_bytes,
+                                                  "us": kernels["coarse_attn"].get("us")},
+                             how="same attention kernel on a token-level cache (flat Transformer, read every token), on a "
+                                 "level-1 cache (hierarchical generation also reads it, once per 4 tokens) and on the top-level "
+                                 "cache (recursive generation reads only this, once per 16 tokens); eager calls, caches larger "
+                                 "than L2")},
         "device_status": bits,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
