@@ -189,7 +189,9 @@ typedef struct {
 photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, photon_stream stream);
 
 /* Reads (and optionally clears) the device status word.  Synchronises the
- * whole device; the only call that does. */
+ * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT also
+ * puts the context's arrival tickets back to zero, so the context stays
+ * usable after a kernel that gave up on a wait. */
 photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear);
 
 /* The paper has no counterpart to this call: it exists for hosts that must not

@@ -633,13 +633,8 @@ template <int DH, int GP>
 cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
     const int G = p.Hq / p.Hkv;
     const size_t smem = smem_bytes<DH>(G);
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(coarse_attn_kernel<DH, GP>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        smem_set = smem;
-    }
+    static size_t smem_set[kMaxDevices] = {};
+    if (const cudaError_t e = ensure_dynamic_smem(coarse_attn_kernel<DH, GP>, smem, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
     CUtensorMap mk, mv;
     if (!(t = ctx->tmaps.get(p.k, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BOX))) return cudaErrorInvalidValue;

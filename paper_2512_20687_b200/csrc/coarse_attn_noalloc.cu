@@ -35,7 +35,6 @@ constexpr size_t kScratchBytes = kPartialBytes + kTicketBytes + 256;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
-constexpr int kMaxDevices = 64;
 struct DeviceState {
     bool ready = false;
     photon_ctx ctx;                // host-side only: no device memory of its own

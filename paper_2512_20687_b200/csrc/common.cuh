@@ -79,6 +79,18 @@ struct ConvParams {
     int32_t *status;
 };
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device and per
+// function); `set` is the launcher's record of what each device already has.
+constexpr int kMaxDevices = 64;
+template <typename K>
+inline cudaError_t ensure_dynamic_smem(K kernel, size_t bytes, int device, size_t (&set)[kMaxDevices]) {
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (bytes <= set[device]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) set[device] = bytes;
+    return e;
+}
+
 // Launch with programmatic stream serialization (and, optionally, a cluster width): the kernel's launch
 // latency and its set-up before grid_dep_wait() overlap the tail of the kernel before it in the stream.
 template <typename... KArgs, typename... Args>

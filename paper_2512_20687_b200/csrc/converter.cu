@@ -205,13 +205,8 @@ template <int NT, bool IN_MAJOR>
 cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches) {
     p.x_rows = p.B > 64 ? 128 : p.B > 32 ? 64 : p.B > 16 ? 32 : 16;
     using T = ConvTile<NT>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(converter_umma_kernel<NT, IN_MAJOR>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static size_t smem_set[kMaxDevices] = {};
+    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR>, T::SMEM, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
     CUtensorMap mx, mw;
     if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, p.x_rows))) return cudaErrorInvalidValue;

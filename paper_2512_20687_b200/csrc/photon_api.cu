@@ -284,6 +284,10 @@ photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t c
     if (cudaMemcpy(bits_out, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
         return PHOTON_ERR_CUDA;
     if (clear && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return PHOTON_ERR_CUDA;
+    // a kernel that gave up on a wait may have left arrival tickets behind; they must read zero again
+    if (clear && (*bits_out & PHOTON_DEV_TIMEOUT) &&
+        cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
     return PHOTON_OK;
 }
 

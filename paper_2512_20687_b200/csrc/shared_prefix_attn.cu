@@ -494,13 +494,8 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
 template <int DH>
 cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launches) {
     using T = SpTile<DH>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(shared_prefix_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             T::SMEM);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static size_t smem_set[kMaxDevices] = {};
+    if (const cudaError_t e = ensure_dynamic_smem(shared_prefix_kernel<DH>, T::SMEM, ctx->device, smem_set)) return e;
     const int G = p.Hq / p.Hkv;
     const int upt = BM / G;
     const int groups = (p.n_q + upt - 1) / upt;
