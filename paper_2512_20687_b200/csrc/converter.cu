@@ -21,7 +21,7 @@ namespace {
 
 constexpr int BM = 128;                 // batch rows per CTA (UMMA M)
 constexpr int BK = 64;                  // K elements per swizzle atom (one 128-byte row)
-constexpr int KA = 2;                   // atoms per stage: one barrier round trip per 128 K elements
+template <int NT> __host__ __device__ constexpr int atoms_per_stage() { return NT >= 256 ? 1 : 2; }   // 128 (64) K elements per barrier round trip
 constexpr int CONV_THREADS = 224;       // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue
 // With narrow weight slabs two warps issue MMAs: they take alternate stages and accumulate into
 // separate TMEM columns, because issuing a tcgen05.mma costs one thread more time than a narrow
@@ -38,8 +38,8 @@ struct ConvTile {
     static constexpr int SMEM = RING_BYTES + BM * BK * 2 + 1024 + 512;
 };
 
-__host__ __device__ inline int conv_stages(int a_bytes, int b_bytes) {
-    const int s = RING_BYTES / (KA * (a_bytes + b_bytes));
+__host__ __device__ inline int conv_stages(int a_bytes, int b_bytes, int ka) {
+    const int s = RING_BYTES / (ka * (a_bytes + b_bytes));
     return s < MAX_STAGES ? s : MAX_STAGES;
 }
 
@@ -50,12 +50,13 @@ __global__ void __launch_bounds__(CONV_THREADS, 1)
 converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
                       const __grid_constant__ CUtensorMap tm_w) {
     using T = ConvTile<NT>;
+    constexpr int KA = atoms_per_stage<NT>();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
     const int a_bytes = p.x_rows * BK * 2;                       // x atom of this launch
     const int stage_bytes = KA * (a_bytes + T::B_BYTES);         // [x atoms][weight atoms]
-    const int n_stages = conv_stages(a_bytes, T::B_BYTES);
+    const int n_stages = conv_stages(a_bytes, T::B_BYTES, KA);
     constexpr int TAIL = RING_BYTES + BM * BK * 2;
     const uint32_t bars = base + TAIL;                           // full[s] +16s, empty[s] +16s+8
     const uint32_t bar_acc = bars + 16 * MAX_STAGES;
@@ -225,9 +226,14 @@ cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launc
 
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
     if (p.B == 0) return cudaSuccess;
-    // wider weight slabs once the batch is large enough for the tensor pipe to matter
+    // wider weight slabs once the batch is large enough for the tensor pipe to matter, as long as
+    // about one CTA per SM remains
+    const int m_tiles = (p.B + BM - 1) / BM;
     const bool wide = p.B > 128 && p.N % 128 == 0;
+    const bool wider = wide && p.N % 256 == 0 && (p.N / 256) * m_tiles >= 100;
     if (p.w_out_major)
-        return wide ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
-    return wide ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
+        return wider ? run<256, false>(ctx, p, st, launches)
+                     : wide ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
+    return wider ? run<256, true>(ctx, p, st, launches)
+                 : wide ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
 }
