@@ -454,12 +454,13 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                         M = -CUDART_INF_F; L = 0.f;
 #pragma unroll
                         for (int i = 0; i < MAXV; ++i) acc[i] = 0.f;
-                        for (int cc = c_first; cc <= c_last; cc += 2) {
-                            // two partials per trip: all their loads are in flight together
-                            float mj[2], lj[2];
-                            float2 a[2][MAXV / 2];
+                        // PB partials per trip: all their loads are in flight together
+                        constexpr int PB = MAXV <= 16 ? 4 : 2;
+                        for (int cc = c_first; cc <= c_last; cc += PB) {
+                            float mj[PB], lj[PB];
+                            float2 a[PB][MAXV / 2];
 #pragma unroll
-                            for (int t = 0; t < 2; ++t) {
+                            for (int t = 0; t < PB; ++t) {
                                 const int c2 = min(cc + t, c_last);
                                 const float *src = p.cta_partials +
                                                    ((size_t)(2 * c2 + (c2 < c_last ? 1 : 0)) * G + r) * (DH + 2);
@@ -468,10 +469,9 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                                 for (int i = 0; i < MAXV / 2; ++i)
                                     a[t][i] = __ldcg(reinterpret_cast<const float2 *>(src + d0) + i);
                             }
-                            if (cc + 1 > c_last) lj[1] = 0.f;
 #pragma unroll
-                            for (int t = 0; t < 2; ++t) {
-                                if (!(lj[t] > 0.f)) continue;
+                            for (int t = 0; t < PB; ++t) {
+                                if (cc + t > c_last || !(lj[t] > 0.f)) continue;
                                 const float Mn = fmaxf(M, mj[t]);
                                 const float f0 = exp2f(M - Mn), f1 = exp2f(mj[t] - Mn);   // M = -inf at first: f0 = 0
 #pragma unroll
