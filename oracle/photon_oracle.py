@@ -37,6 +37,7 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.oracle_kv_append.restype = ctypes.c_int
         _lib.oracle_attention.restype = ctypes.c_int
+        _lib.oracle_chunk_causal_attention.restype = ctypes.c_int
         _lib.oracle_hardware_threads.restype = ctypes.c_int
     return _lib
 
@@ -115,6 +116,28 @@ def chunk_attention(q, kc, vc, length, scale, slot=None, n_threads=1):
     [0, length[c]) of its own chunk buffer only (P prefix rows then the
     in-chunk rows)."""
     return attention(q, kc, vc, length, scale, slot=slot, n_threads=n_threads)
+
+
+def chunk_causal_attention(q, kc, vc, length, scale, row0=0, slot=None, n_threads=1,
+                           want_flags=False):
+    """The local decoder at R positions of every chunk at once (teacher-forced form
+    of Eq. 6 under the causal mask below Eq. 7).  q: [n, R, Hq, dh]; query t stands
+    at row row0 + t of its chunk buffer (kc, vc: [n_units, Hkv, cap, dh]) and attends
+    rows 0 .. row0 + t; positions >= length[u] give zero rows.  Returns float64
+    [n, R, Hq, dh]."""
+    q, kc, vc = _u16(q), _u16(kc), _u16(vc)
+    length = _i32(length)
+    n, R, Hq, dh = q.shape
+    n_units, Hkv, cap, dh2 = kc.shape
+    assert dh == dh2 and Hq % Hkv == 0 and vc.shape == kc.shape
+    slot = _i32(slot)
+    if slot is None:
+        assert n == n_units
+    out = np.empty((n, R, Hq, dh), dtype=np.float64)
+    flags = lib().oracle_chunk_causal_attention(_p(q), n, R, int(row0), _p(slot), _p(kc), _p(vc),
+                                                _p(length), n_units, Hq, Hkv, cap, dh,
+                                                ctypes.c_double(scale), _p(out), int(n_threads))
+    return (out, flags) if want_flags else out
 
 
 def attn_range(q_vec, k_rows, v_rows, r0, r1, scale):

@@ -238,6 +238,28 @@ def chunk_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False,
     }
 
 
+def chunk_causal_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False,
+                        full: bool = False, row0: int = 0, rows: int | None = None) -> dict:
+    """The chunk buffers of chunk_inputs with a query for `rows` consecutive
+    positions of every chunk, starting at row `row0` (default: all P + C rows):
+    q [Nc, rows, Hq, dh].  full=True makes every chunk complete (len = P + C),
+    the teacher-forced whole-chunk case; otherwise the lengths are the ragged
+    ones of chunk_inputs and positions >= len do not exist yet."""
+    tag = f"r{replica}"
+    a = chunk_inputs(cfg, replica=replica, poison=poison and not full)
+    cap = a["cap"]
+    rows = cap - row0 if rows is None else rows
+    if full:
+        shape = (cfg.Nc, cfg.Hkv, cap, cfg.dh)
+        a["kc"] = normal_bf16(cfg.seed, f"chunk_k/{tag}", shape)
+        a["vc"] = normal_bf16(cfg.seed, f"chunk_v/{tag}", shape)
+        a["len"] = np.full(cfg.Nc, cap, np.int32)
+        a["n_in"] = np.full(cfg.Nc, cfg.C, np.int32)
+    a["q"] = normal_bf16(cfg.seed, f"chunk_qrows/{tag}", (cfg.Nc, rows, cfg.Hq, cfg.dh))
+    a["row0"], a["rows"] = row0, rows
+    return a
+
+
 def step_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False) -> dict:
     """Everything one decode step consumes."""
     return {
