@@ -154,6 +154,22 @@ photon_status photon_chunk_attn(photon_ctx *ctx, const photon_kv *chunks, const 
                                 const int32_t *slot, photon_bf16 *out, int32_t Nc, float scale,
                                 photon_stream stream);
 
+/* The local decoder's attention at `rows` consecutive positions of every
+ * chunk at once: the teacher-forced form of Eq. 6 (all positions of a chunk in
+ * one pass, or the P-row pass over a fresh converter prefix) under the
+ * standard causal mask described below Eq. 7.  Query t of chunk c (q [Nc,
+ * rows, Hq, dh]) stands at row row0 + t of chunk buffer u = slot ? slot[c] : c
+ * and attends rows 0 .. row0 + t of that buffer and nothing else.  A position
+ * at or beyond len[u] does not exist yet: its output row is zero.  out [Nc,
+ * rows, Hq, dh], bf16, written in full.  Requires cap <= min(P + C, 64),
+ * row0 >= 0, rows >= 1, row0 + rows <= cap (else INVALID_ARG); q and out are
+ * device pointers, 16-byte aligned, owned by the caller; a slot outside
+ * [0, n_units) gives zero rows and sets PHOTON_DEV_BAD_INDEX.  One kernel on
+ * `stream`, no workspace.  Shared-prefix fields of `chunks` must be unset. */
+photon_status photon_chunk_causal_attn(photon_ctx *ctx, const photon_kv *chunks, const photon_bf16 *q,
+                                       const int32_t *slot, photon_bf16 *out, int32_t Nc, int32_t row0,
+                                       int32_t rows, float scale, photon_stream stream);
+
 /* One decode step on one stream, in the order of Section 2.3.3: append
  * (k_new, v_new) to `coarse`; coarse attention of q_coarse over the grown
  * cache -> out_coarse (lse_coarse optional); converter on x, or, when x is

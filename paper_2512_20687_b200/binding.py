@@ -87,6 +87,9 @@ def load() -> ctypes.CDLL:
     lib.photon_chunk_attn.restype = st
     lib.photon_chunk_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
                                       c_int32, c_float, c_void_p]
+    lib.photon_chunk_causal_attn.restype = st
+    lib.photon_chunk_causal_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
+                                             c_int32, c_int32, c_int32, c_float, c_void_p]
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_device_status.restype = st
@@ -191,6 +194,17 @@ def photon_converter(ctx, x, w, w_layout, bias, U, B=None, stream=None) -> None:
         B = x.shape[0]
     _check(load().photon_converter(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(U), int(B),
                                    _stream(stream)), "photon_converter")
+
+
+def photon_chunk_causal_attn(ctx, chunks: photon_kv, q, slot, out, Nc=None, row0=0, rows=None,
+                             scale=1.0, stream=None) -> None:
+    if Nc is None:
+        Nc = q.shape[0]
+    if rows is None:
+        rows = q.shape[1]
+    _check(load().photon_chunk_causal_attn(ctx, byref(chunks), _ptr(q), _ptr(slot), _ptr(out), int(Nc),
+                                           int(row0), int(rows), c_float(scale), _stream(stream)),
+           "photon_chunk_causal_attn")
 
 
 def photon_chunk_attn(ctx, chunks: photon_kv, q, slot, out, Nc=None, scale=1.0, stream=None) -> None:

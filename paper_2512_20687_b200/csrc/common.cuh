@@ -70,6 +70,21 @@ struct AttnParams {
     int32_t *status;
 };
 
+// Whole-chunk causal attention: query t of item i (q, out: [n, R, Hq, dh]) stands at row row0 + t of
+// chunk buffer u = slot ? slot[i] : i and sees rows 0 .. row0 + t of it.
+struct CausalParams {
+    const bf16 *q;
+    bf16 *out;
+    const bf16 *k, *v;
+    const int32_t *len;
+    const int32_t *slot;
+    int n_units, cap;
+    int n, R, row0;
+    int Hq, Hkv, dh;
+    float scale_log2;
+    int32_t *status;
+};
+
 struct ConvParams {
     const bf16 *x, *w, *bias;
     bf16 *U;
@@ -131,6 +146,8 @@ int coarse_attn_ctas_per_sm();
 int shared_prefix_units_per_cta(int G);
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);
+cudaError_t launch_chunk_causal_attention(photon_ctx *ctx, const CausalParams &p, cudaStream_t st,
+                                          long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);
 

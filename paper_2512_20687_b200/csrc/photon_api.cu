@@ -200,6 +200,33 @@ photon_status photon_chunk_attn(photon_ctx *ctx, const photon_kv *chunks, const 
                             static_cast<cudaStream_t>(stream));
 }
 
+photon_status photon_chunk_causal_attn(photon_ctx *ctx, const photon_kv *chunks, const photon_bf16 *q,
+                                       const int32_t *slot, photon_bf16 *out, int32_t Nc, int32_t row0,
+                                       int32_t rows, float scale, photon_stream stream) {
+    if (!ctx || !chunks) return PHOTON_ERR_INVALID_ARG;
+    if (!kv_ok(ctx, chunks, false)) return PHOTON_ERR_INVALID_ARG;
+    if (chunks->cap > ctx->cfg.P + ctx->cfg.C || chunks->cap > 64) return PHOTON_ERR_INVALID_ARG;
+    if (Nc < 0 || row0 < 0 || rows < 1 || row0 + rows > chunks->cap) return PHOTON_ERR_INVALID_ARG;
+    if (!slot && Nc > chunks->n_units) return PHOTON_ERR_INVALID_ARG;
+    if (Nc > 0 && (!q || !out)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !(scale == scale)) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    CausalParams p{};
+    p.q = reinterpret_cast<const bf16 *>(q);
+    p.out = reinterpret_cast<bf16 *>(out);
+    p.k = reinterpret_cast<const bf16 *>(chunks->k);
+    p.v = reinterpret_cast<const bf16 *>(chunks->v);
+    p.len = chunks->len;
+    p.slot = slot;
+    p.n_units = chunks->n_units; p.cap = chunks->cap;
+    p.n = Nc; p.R = rows; p.row0 = row0;
+    p.Hq = c.Hq; p.Hkv = c.Hkv; p.dh = c.dh;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.status = ctx->status;
+    const cudaError_t e = launch_chunk_causal_attention(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
 photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w,
                                int32_t w_layout, const photon_bf16 *bias, photon_bf16 *U, int32_t B,
                                photon_stream stream) {

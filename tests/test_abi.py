@@ -28,7 +28,8 @@ def declared_symbols():
 def test_header_declares_the_expected_calls():
     names = declared_symbols()
     for want in ("photon_create", "photon_destroy", "photon_kv_append", "photon_coarse_attn",
-                 "photon_flat_attn", "photon_converter", "photon_chunk_attn", "photon_decode_step",
+                 "photon_flat_attn", "photon_converter", "photon_chunk_attn", "photon_chunk_causal_attn",
+                 "photon_decode_step",
                  "photon_device_status", "photon_status_str"):
         assert want in names
 
