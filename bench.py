@@ -410,6 +410,37 @@ def run_gpu(args, cfg) -> None:
             del kk, vv, kvf
         torch.cuda.empty_cache()
 
+    # the widened row: the local decoder's attention at every position of every in-flight chunk in one launch
+    # (teacher-forced whole chunks).  It reuses the chunk buffers of the replicas with every row counted as
+    # present; its queries only feed a timing, so they are drawn on the device from a fixed torch seed.
+    widened = {}
+    if not args.no_parts:
+        cap = cfg.P + cfg.C
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(4321 + cfg.seed)
+        n_q = max(2, min(R, -(-2 * L2_BYTES // max(1, cfg.Nc * cap * cfg.Hq * cfg.dh * 2))))
+        qr = [torch.empty(cfg.Nc, cap, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+              for _ in range(n_q)]
+        orows = [torch.empty_like(t) for t in qr]
+        full_len = torch.full((cfg.Nc,), cap, dtype=torch.int32, device=dev)
+        full_kv = [ph.make_kv(t["kc"], t["vc"], full_len) for t in reps]
+        turn = {"i": 0}
+
+        def causal_call(t):
+            i = turn["i"] = turn["i"] + 1
+            ph.photon_chunk_causal_attn(ctx, full_kv[i % R], qr[i % n_q], None, orows[i % n_q], scale=scale)
+
+        us = graph_time_us(causal_call)
+        nbytes = 2 * cfg.Nc * cfg.Hkv * cap * cfg.dh * 2 + 2 * cfg.Nc * cap * cfg.Hq * cfg.dh * 2
+        flops = 4.0 * cfg.Nc * cfg.Hq * cfg.dh * cap * (cap + 1) / 2
+        widened["chunk_causal_attn"] = {
+            "workload": "all %d rows of each of the %d in-flight chunks, causal" % (cap, cfg.Nc),
+            "us": us, "algorithmic_bytes": nbytes, "GBps": nbytes / us * 1e-3,
+            "frac_hbm": nbytes / us * 1e-3 / hbm_peak, "TFLOPs": flops / us * 1e-6,
+            "note": "K, V, q and out each counted once; causal flops only"}
+        del qr, orows, full_kv
+        torch.cuda.empty_cache()
+
     # roofline of the dominant kernel = the attention part that takes the longest
     dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
     traffic, traffic_note = None, "no ncu capture on record for this kernel and workload"
@@ -505,6 +536,7 @@ def run_gpu(args, cfg) -> None:
         "step_hbm": {"algorithmic_bytes": step_bytes, "GBps": step_bytes / (sec_max / K) * 1e-9,
                      "frac": step_bytes / (sec_max / K) * 1e-9 / hbm_peak},
         "parts": parts,
+        "widened": widened,
         "kv_bytes_per_token": {
             "photon_coarse_per_step": coarse_bytes,
             "photon_per_token": coarse_bytes / cfg.compress / cfg.B + (chunk_bytes / cfg.Nc),

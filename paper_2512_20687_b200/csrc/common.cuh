@@ -38,6 +38,7 @@ struct photon_ctx {
     int32_t *tickets;        // one arrival counter per (unit, kv head); zero between calls
     size_t n_tickets;
     int32_t *status;         // device status word
+    int32_t *work;           // two counters of the whole-chunk attention's item hand-out; zero between calls
     long long launches;
     cudaStream_t side;       // lowest-priority stream for the chunk attention of a decode step
     cudaEvent_t ev_fork, ev_join;
@@ -80,6 +81,8 @@ struct CausalParams {
     const int32_t *slot;
     int n_units, cap;
     int n, R, row0;
+    int gsplit;              // filled by the launcher: warps that share a (chunk, KV head), 1 or Hq / Hkv
+    int32_t *work;           // filled by the launcher: {items handed out, CTAs that have finished}; zero between calls
     int Hq, Hkv, dh;
     float scale_log2;
     int32_t *status;

@@ -125,14 +125,15 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
     if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->cta_partials, size_t(2) * ctx->max_ctas * 16 * (c.dh + 2) * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->tickets, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
-        cudaMalloc(&ctx->status, sizeof(int32_t)) != cudaSuccess ||
+        cudaMalloc(&ctx->status, 64 * sizeof(int32_t)) != cudaSuccess ||     // the word, and the counters 128 B on
         cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
-        cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) {
+        cudaMemset(ctx->status, 0, 64 * sizeof(int32_t)) != cudaSuccess) {
         cudaFree(ctx->partials); cudaFree(ctx->cta_partials); cudaFree(ctx->tickets); cudaFree(ctx->status);
         cudaGetLastError();
         delete ctx;
         return PHOTON_ERR_CUDA;
     }
+    ctx->work = ctx->status + 32;
     int lo = 0, hi = 0;
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, lo) != cudaSuccess ||
