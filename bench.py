@@ -443,19 +443,28 @@ def run_gpu(args, cfg) -> None:
 
     # roofline of the dominant kernel = the attention part that takes the longest
     dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
-    traffic, traffic_note = None, "no ncu capture on record for this kernel and workload"
-    try:
-        rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.txt"))).get(
-            f"config{cfg.index}", {}).get(dom)
-        if rec:
-            import hashlib
-            src = os.path.join(ROOT, "paper_2512_20687_b200", "csrc", rec["source"])
-            if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["source_sha256"]:
-                traffic, traffic_note = rec["dram_bytes_per_launch"], rec.get("how", "")
-            else:
-                traffic_note = "kernel source changed since the ncu counters were taken"
-    except (OSError, ValueError, KeyError):
-        pass
+    def recorded_traffic(kernel_name):
+        """DRAM bytes per launch from the committed ncu capture, or None once the kernel's source has changed."""
+        note = "no ncu capture on record for this kernel and workload"
+        if args.batch:
+            return None, "reduced batch: the recorded traffic belongs to the full workload"
+        try:
+            rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.txt"))).get(
+                f"config{cfg.index}", {}).get(kernel_name)
+            if rec:
+                import hashlib
+                src = os.path.join(ROOT, "paper_2512_20687_b200", "csrc", rec["source"])
+                if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["source_sha256"]:
+                    return rec["dram_bytes_per_launch"], rec.get("how", "")
+                note = "kernel source changed since the ncu counters were taken"
+        except (OSError, ValueError, KeyError):
+            pass
+        return None, note
+
+    traffic, traffic_note = recorded_traffic(dom)
+    if "chunk_causal_attn" in widened:
+        widened["chunk_causal_attn"]["traffic"], widened["chunk_causal_attn"]["traffic_note"] = recorded_traffic(
+            "chunk_causal_attn")
     ach = kernels[dom]["bytes"] / kernels[dom]["us"] * 1e-3
     roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
                 "frac": ach / hbm_peak, "traffic": traffic, "traffic_note": traffic_note,
