@@ -375,17 +375,19 @@ def run_gpu(args, cfg) -> None:
     parts["note"] = ("each part timed as a CUDA graph of back-to-back calls rotating over the replicas; "
                      "kv_append's figure includes a %d-int length reset every %d calls" % (cfg.B * R, R))
 
-    # what a flat Transformer and hierarchical generation (every level keeps a global cache) would read
-    # for the same context, measured with the same attention kernel: a token-level cache (context rows per
-    # sequence) through photon_flat_attn, and a level-1 cache (context / C1 rows) through photon_coarse_attn.
-    # These caches only feed a timing, so they are filled on the device from a fixed torch seed.
-    kv_measured = {}
+    # The global caches of the three generation schedules (a flat Transformer; hierarchical generation,
+    # which keeps a cache at every level; recursive generation, which keeps the top level only) for the same
+    # context, read with the same attention kernel: measured time and bytes per read and, amortised over the
+    # tokens between reads, per generated token.  The lower-level caches only feed a timing, so they are
+    # filled on the device from a fixed torch seed; the top level is the step's own coarse attention.
+    kv_measured, schedules = {}, {}
     if not args.no_parts and cfg.compress == 16:
         gen = torch.Generator(device=dev)
         gen.manual_seed(1234 + cfg.seed)
-        c1 = 4                                                   # C1 of the two-level hierarchy
-        for name, rows, fn in (("flat_token_level", cfg.context + cfg.shared_context, ph.photon_flat_attn),
-                               ("level1_global", (cfg.context + cfg.shared_context) // c1, ph.photon_coarse_attn)):
+        per_level = {2: {"rows_per_sequence": cfg.S + cfg.shared_S, "kv_bytes_per_read": coarse_bytes,
+                         "us_per_read": kernels["coarse_attn"].get("us")}}
+        for level, fn in ((0, ph.photon_flat_attn), (1, ph.photon_coarse_attn)):
+            rows = wl.global_caches(cfg, "flat" if level == 0 else "hierarchical")[0]["rows"]
             nbytes = cfg.B * cfg.Hkv * rows * cfg.dh * 2 * 2
             if nbytes > (24 << 30):
                 continue
@@ -404,11 +406,26 @@ def run_gpu(args, cfg) -> None:
                 fn(ctx, kvf, q, o2, None, scale)
             b.record()
             torch.cuda.synchronize()
-            us = a.elapsed_time(b) * 1e3 / n_rep
-            kv_measured[name] = {"rows_per_sequence": rows, "kv_bytes_per_step": nbytes, "us": us,
-                             "GBps": nbytes / us * 1e-3}
+            per_level[level] = {"rows_per_sequence": rows, "kv_bytes_per_read": nbytes,
+                                "us_per_read": a.elapsed_time(b) * 1e3 / n_rep}
             del kk, vv, kvf
         torch.cuda.empty_cache()
+        kv_measured = {"flat_token_level": per_level.get(0), "level1_global": per_level.get(1),
+                       "recursive_top_level": per_level[2]}
+        for sch in wl.SCHEDULES:
+            caches = wl.global_caches(cfg, sch)
+            if any(c["level"] not in per_level for c in caches):
+                continue
+            schedules[sch] = {
+                "caches": [dict(c, **per_level[c["level"]]) for c in caches],
+                "kv_bytes_per_token": sum(per_level[c["level"]]["kv_bytes_per_read"] / c["tokens_per_read"]
+                                          for c in caches) / cfg.B,
+                "global_attention_us_per_token": sum(per_level[c["level"]]["us_per_read"] / c["tokens_per_read"]
+                                                     for c in caches)}
+        if schedules:
+            schedules["note"] = ("per sequence and layer, whole batch decoded in step; levels 0 and 1 hold a shared prefix "
+                                 "once per branch; eager calls on caches larger than L2 for levels 0 and 1, the "
+                                 "timed graph for the top level")
 
     # the widened row: the local decoder's attention at every position of every in-flight chunk in one launch
     # (teacher-forced whole chunks).  It reuses the chunk buffers of the replicas with every row counted as
@@ -551,13 +568,8 @@ def run_gpu(args, cfg) -> None:
             "photon_per_token": coarse_bytes / cfg.compress / cfg.B + (chunk_bytes / cfg.Nc),
             "flat_per_token": wl.flat_kv_bytes(cfg) / cfg.B,
             "note": "per sequence and layer; coarse step amortised over %d tokens" % cfg.compress,
-            "measured": dict(kv_measured,
-                             recursive_top_level={"rows_per_sequence": cfg.S + cfg.shared_S, "kv_bytes_per_step": coarse_bytes,
-                                                  "us": kernels["coarse_attn"].get("us")},
-                             how="same attention kernel on a token-level cache (flat Transformer, read every token), on a "
-                                 "level-1 cache (hierarchical generation also reads it, once per 4 tokens) and on the top-level "
-                                 "cache (recursive generation reads only this, once per 16 tokens); eager calls, caches larger "
-                                 "than L2")},
+            "measured": kv_measured},
+        "schedules": schedules,
         "device_status": bits,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -284,6 +284,58 @@ def flat_kv_bytes(cfg: DecodeConfig) -> int:
     return (cfg.B * cfg.context + cfg.shared_context) * per_row
 
 
+# ---- global caches of the generation schedules (Sections 2.3.2 and 2.3.3) ----
+
+SCHEDULES = ("flat", "hierarchical", "recursive")
+
+
+def global_caches(cfg: DecodeConfig, schedule: str, chunk_lengths=(4, 4)) -> list[dict]:
+    """The context-growing caches a schedule keeps for a context of cfg.context
+    tokens per sequence, and how often each is read while C_{<=L} tokens (one
+    meta-context) are generated.  A flat Transformer keeps one token-level
+    cache and reads it for every token.  Hierarchical generation keeps a
+    global cache at every level l (T / C_{<=l} rows) and advances level l once
+    per level-l chunk, i.e. C_{<=L} / C_{<=l} times per meta-context.
+    Recursive generation keeps the top level only and reads it once.
+    Returns [{level, rows, reads_per_meta, tokens_per_read}], lowest level first."""
+    assert schedule in SCHEDULES
+    total = int(np.prod(chunk_lengths))
+    assert total == cfg.compress
+    ctx = cfg.context + cfg.shared_context
+    if schedule == "flat":
+        return [{"level": 0, "rows": ctx, "reads_per_meta": total, "tokens_per_read": 1}]
+    out, upto = [], 1
+    for level, c in enumerate(chunk_lengths, start=1):
+        upto *= c
+        out.append({"level": level, "rows": ctx // upto, "reads_per_meta": total // upto,
+                    "tokens_per_read": upto})
+    return out if schedule == "hierarchical" else out[-1:]
+
+
+def global_kv_bytes_per_token(cfg: DecodeConfig, schedule: str, chunk_lengths=(4, 4)) -> float:
+    """K+V bytes of the global caches read per generated token and sequence at
+    the context length of the workload: sum over levels of rows * bytes per row
+    / tokens per read."""
+    per_row = cfg.Hkv * cfg.dh * 2 * 2
+    return sum(c["rows"] * per_row / c["tokens_per_read"] for c in global_caches(cfg, schedule, chunk_lengths))
+
+
+def cumulative_global_rows(T: int, schedule: str, chunk_lengths=(4, 4)) -> int:
+    """Cache rows read by the global attention while T tokens are generated from
+    an empty context: level l advances once per C_{<=l} tokens and its step g
+    attends g rows, sum_{g=1}^{M_l} g with M_l = T / C_{<=l} (the cumulative
+    global KV reads of Section 2.3.2); level 0 is the flat Transformer."""
+    assert schedule in SCHEDULES
+    tri = lambda m: m * (m + 1) // 2
+    if schedule == "flat":
+        return tri(T)
+    upto, per_level = 1, []
+    for c in chunk_lengths:
+        upto *= c
+        per_level.append(tri(T // upto))
+    return sum(per_level) if schedule == "hierarchical" else per_level[-1]
+
+
 def chunk_kv_bytes(cfg: DecodeConfig, lens: np.ndarray) -> int:
     return int(lens.astype(np.int64).sum()) * cfg.Hkv * cfg.dh * 2 * 2
 

@@ -84,6 +84,24 @@ def test_coarse_attention_matches_oracle_at_full_size(oracle, idx):
     assert np.abs(lse - want_lse).max() < 2e-3
 
 
+def test_level1_cache_of_hierarchical_generation(oracle):
+    """The cache hierarchical generation keeps one level below the top (context / C1
+    rows per sequence: 2048 for the 1B-class workload) through the same attention call:
+    the second global workload of the schedule comparison, at its full size."""
+    rows = wl.global_caches(wl.CONFIGS[1], "hierarchical")[0]["rows"]
+    assert rows == 2048
+    cfg = cfg_small(1, S=rows)
+    co = wl.coarse_inputs(cfg, poison=True)
+    oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"])
+    scale = cfg.dh ** -0.5
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        got, lse, _ = run_coarse(c, co, scale)
+        assert c.status() == 0
+    assert_close(got, want, "level-1 cache")
+    assert np.abs(lse - want_lse).max() < 2e-3
+
+
 @pytest.mark.parametrize("n_ctas", [1, 2, 3, 7, 37, 101, 0])
 def test_grid_size_and_cut_points_do_not_change_the_result(oracle, n_ctas):
     """Ragged lengths incl. 0 and 1; the grid size moves the points where caches

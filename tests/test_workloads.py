@@ -52,6 +52,43 @@ def test_kv_bytes_closed_forms():
         assert wl.flat_kv_bytes(c) / per_token_coarse == c.compress ** 2 == 256
 
 
+def test_generation_schedules_against_a_decode_loop():
+    """Count, token by token, the rows each schedule's global attention reads
+    (a level advances when its chunk fills and its newest row attends itself and
+    everything before it) and compare with the closed forms; the orders of
+    Section 2.3.2 / 2.3.3 follow: recursive generation reads C_{<=L}^2 times fewer
+    rows than a flat Transformer, hierarchical generation is dominated by level 1."""
+    C1, C2 = 4, 4
+    for T in (16, 64, 1024):
+        rows = {"flat": 0, "hierarchical": 0, "recursive": 0}
+        n1 = n2 = 0
+        for t in range(1, T + 1):
+            rows["flat"] += t                              # the new token sees t rows
+            if t % C1 == 0:
+                n1 += 1
+                rows["hierarchical"] += n1
+            if t % (C1 * C2) == 0:
+                n2 += 1
+                rows["hierarchical"] += n2
+                rows["recursive"] += n2
+        for sch in wl.SCHEDULES:
+            assert wl.cumulative_global_rows(T, sch) == rows[sch], (T, sch)
+    big = 1 << 20
+    flat, hier, rec = (wl.cumulative_global_rows(big, s) for s in wl.SCHEDULES)
+    assert abs(flat / rec / 256 - 1) < 1e-4               # (C1 C2)^2
+    assert abs(hier / rec / 17 - 1) < 1e-4                # 1 + C2^2
+    cfg = wl.CONFIGS[1]
+    per_row = cfg.Hkv * cfg.dh * 4
+    caches = wl.global_caches(cfg, "hierarchical")
+    assert [(c["rows"], c["reads_per_meta"]) for c in caches] == [(2048, 4), (512, 1)]
+    assert wl.global_caches(cfg, "recursive") == caches[-1:]
+    assert wl.global_caches(cfg, "flat")[0]["rows"] == 8192
+    assert wl.global_kv_bytes_per_token(cfg, "flat") == 8192 * per_row
+    assert wl.global_kv_bytes_per_token(cfg, "hierarchical") == (2048 / 4 + 512 / 16) * per_row
+    assert wl.global_kv_bytes_per_token(cfg, "recursive") == 512 / 16 * per_row
+    assert wl.global_kv_bytes_per_token(cfg, "recursive") * cfg.B == wl.coarse_kv_bytes(cfg) / cfg.compress
+
+
 def test_chunk_inputs_structure():
     cfg = wl.CONFIGS[0]
     ch = wl.chunk_inputs(cfg, poison=True)
