@@ -180,6 +180,38 @@ def converter(x, w, bias=None, w_out_major=False, n_threads=1):
     return out
 
 
+def rmsnorm(x, gamma=None, eps=0.0):
+    """Root-mean-square normalisation of each row of x [rows, cols] with an optional
+    per-column scale (first half of the context chunker).  Returns float64."""
+    x = _u16(x)
+    rows, cols = x.shape
+    gamma = None if gamma is None else _u16(gamma)
+    out = np.empty((rows, cols), dtype=np.float64)
+    lib().oracle_rmsnorm(_p(x), _p(gamma), ctypes.c_double(eps), rows, cols, _p(out))
+    return out
+
+
+def linear(x, w, bias=None, w_out_major=False, n_threads=1):
+    """y = x W + b.  x: [B, K]; w: [K, N] (or [N, K] when w_out_major).  Returns float64 [B, N]."""
+    x, w = _u16(x), _u16(w)
+    B, K = x.shape
+    N = w.shape[0] if w_out_major else w.shape[1]
+    assert (w.shape[1] if w_out_major else w.shape[0]) == K
+    bias = None if bias is None else _u16(bias)
+    out = np.empty((B, N), dtype=np.float64)
+    lib().oracle_linear(_p(x), _p(w), int(bool(w_out_major)), _p(bias), B, K, N, _p(out), int(n_threads))
+    return out
+
+
+def chunker(x, gamma, eps, w, bias=None, w_out_major=False, n_threads=1):
+    """Level-L context chunker (Section 2.1.1; step (ii) of Section 2.3.3): the C_L
+    reconstructed lower-level latents of a meta-context, concatenated (x: [B, C*D]),
+    normalised with a learned scale, rounded to bf16 (what the linear part reads),
+    then mapped to D_L.  Returns (normalised bf16 bits [B, C*D], float64 [B, N])."""
+    xn = round_bf16(rmsnorm(x, gamma, eps))
+    return xn, linear(xn, w, bias, w_out_major=w_out_major, n_threads=n_threads)
+
+
 def round_bf16(x):
     """float64 -> bf16 bits, round to nearest even."""
     x = np.ascontiguousarray(x, dtype=np.float64)

@@ -212,6 +212,24 @@ def converter_inputs(cfg: DecodeConfig, replica: int = 0, with_bias: bool = Fals
     return out
 
 
+def chunker_inputs(cfg: DecodeConfig, replica: int = 0, block: int = 4) -> dict:
+    """Level-L context chunker: per sequence the `block` reconstructed level-(L-1)
+    latents of the meta-context just decoded, concatenated (x [B, block*D], N(0,1)),
+    a per-feature scale around 1, a weight [block*D, D] of variance 1/(block*D) in
+    both storage orders, and a bias."""
+    tag = f"r{replica}"
+    K = block * cfg.D
+    w = normal_bf16(cfg.seed, f"chunker_w/{tag}", (K, cfg.D), std=K ** -0.5)
+    g = bf16_bits_to_f64(normal_bf16(cfg.seed, f"chunker_g/{tag}", (K,), std=0.1)) + 1.0
+    return {
+        "x": normal_bf16(cfg.seed, f"chunker_x/{tag}", (cfg.B, K)),
+        "gamma": f32_to_bf16_bits(g.astype(np.float32)),
+        "w_in_major": w, "w_out_major": np.ascontiguousarray(w.T),
+        "bias": normal_bf16(cfg.seed, f"chunker_b/{tag}", (cfg.D,), std=0.1),
+        "eps": 1e-5, "K": K, "N": cfg.D,
+    }
+
+
 def chunk_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False,
                  strict_paper: bool = False) -> dict:
     """Chunk-local tensors: Nc in-flight chunks, each a cache of cap = P + C
