@@ -458,6 +458,41 @@ def run_gpu(args, cfg) -> None:
         del qr, orows, full_kv
         torch.cuda.empty_cache()
 
+        # the top-level context chunker (step (ii) of a recursive-generation step): normalise the 4 concatenated
+        # lower-level latents per sequence, project [B, 4D] -> [B, D]; weights rotate like the converter's
+        ci = wl.chunker_inputs(cfg)
+        Kc = ci["K"]
+        cw = [dev_bf16(ci["w_out_major"] if out_major else ci["w_in_major"])]
+        cw += [cw[0].clone() for _ in range(R - 1)]
+        cx, cg, cb = dev_bf16(ci["x"]), dev_bf16(ci["gamma"]), dev_bf16(ci["bias"])
+        cxn = torch.empty_like(cx)
+        cy = torch.empty(cfg.B, cfg.D, dtype=torch.bfloat16, device=dev)
+        turn["i"] = 0
+
+        def norm_call(t):
+            ph.photon_rmsnorm(ctx, cx, cg, ci["eps"], cxn)
+
+        def linear_call(t):
+            i = turn["i"] = turn["i"] + 1
+            ph.photon_linear(ctx, cxn, cw[i % R], layout, cb, cy)
+
+        def chunker_call(t):
+            norm_call(t)
+            linear_call(t)
+
+        us_n, us_l, us_c = graph_time_us(norm_call), graph_time_us(linear_call), graph_time_us(chunker_call)
+        cbytes = Kc * cfg.D * 2 + cfg.B * Kc * 2 + cfg.B * cfg.D * 2
+        cflops = 2.0 * cfg.B * Kc * cfg.D
+        t_roof = max(cbytes / (hbm_peak * 1e3), cflops / (tensor_peak * 1e6))
+        widened["chunker"] = {
+            "workload": "[%d, %d] -> [%d, %d]: row normalisation, then linear with bias" % (cfg.B, Kc, cfg.B, cfg.D),
+            "us": us_c, "us_rmsnorm": us_n, "us_linear": us_l, "algorithmic_bytes": cbytes,
+            "GBps": cbytes / us_c * 1e-3, "frac_hbm": cbytes / us_c * 1e-3 / hbm_peak,
+            "TFLOPs": cflops / us_c * 1e-6, "frac_of_own_roofline": t_roof / us_c,
+            "note": "x, W and y counted once; the normalised copy of x is an intermediate"}
+        del cw
+        torch.cuda.empty_cache()
+
     # roofline of the dominant kernel = the attention part that takes the longest
     dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
     def recorded_traffic(kernel_name):

@@ -144,6 +144,29 @@ photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const phot
                                int32_t w_layout, const photon_bf16 *bias, photon_bf16 *U, int32_t B,
                                photon_stream stream);
 
+/* The two halves of the top-level context chunker C^(L) (Section 2.1.1; step
+ * (ii) of a recursive-generation step, Section 2.3.3: the C_L reconstructed
+ * lower-level latents of the meta-context just decoded are concatenated and
+ * summarised into the next input of the top-level encoder).  The parameter
+ * tables of Appendix B size it as a scale per concatenated feature, a weight
+ * [C_L * D, D] and a bias.
+ *
+ * photon_rmsnorm: out[r, c] = x[r, c] * gamma[c] / sqrt(mean_c x[r, c]^2 + eps),
+ * x, out [rows, cols] bf16 (out may alias x), gamma [cols] or NULL (ones),
+ * cols a multiple of 8, eps >= 0; fp32 sums, one rounding to bf16.
+ *
+ * photon_linear: y[b, n] = sum_k x[b, k] * W[k, n] (+ bias[n]); x [B, K], w in
+ * the order given by w_layout ([K, N] or [N, K]), bias [N] or NULL, y [B, N];
+ * K and N multiples of 64 (else INVALID_ARG); bf16 in, fp32 accumulation on the
+ * tensor cores, one rounding at the output; deterministic.  The converter is
+ * the case K = D, N = P * D.  All pointers device, 16-byte aligned, owned by
+ * the caller; one kernel each on `stream`, no workspace. */
+photon_status photon_rmsnorm(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *gamma, float eps,
+                             photon_bf16 *out, int32_t rows, int32_t cols, photon_stream stream);
+photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w, int32_t w_layout,
+                            const photon_bf16 *bias, photon_bf16 *y, int32_t B, int32_t K, int32_t N,
+                            photon_stream stream);
+
 /* Bounded causal attention of the local decoders G^(l) (Eq. 6-7): query c
  * (q [Nc, Hq, dh]) attends rows [0, len[u]) of chunk buffer u = slot ?
  * slot[c] : c of `chunks` (cap = P + C; rows 0..P-1 the converter prefix,

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     PHOTON_W_IN_MAJOR, PHOTON_W_OUT_MAJOR, PhotonError, load, make_kv, make_step_args,
     photon_chunk_attn, photon_chunk_causal_attn, photon_coarse_attn, photon_coarse_attn_noalloc, photon_config, photon_converter, photon_create,
     photon_decode_step, photon_destroy, photon_device_status, photon_flat_attn, photon_kv,
-    photon_kv_append, photon_launch_count, photon_set_attention_ctas, photon_status_str, photon_step_args,
+    photon_kv_append, photon_launch_count, photon_linear, photon_rmsnorm, photon_set_attention_ctas, photon_status_str, photon_step_args,
 )

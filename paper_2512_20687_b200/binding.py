@@ -90,6 +90,11 @@ def load() -> ctypes.CDLL:
     lib.photon_chunk_causal_attn.restype = st
     lib.photon_chunk_causal_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
                                              c_int32, c_int32, c_int32, c_float, c_void_p]
+    lib.photon_rmsnorm.restype = st
+    lib.photon_rmsnorm.argtypes = [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_int32, c_int32, c_void_p]
+    lib.photon_linear.restype = st
+    lib.photon_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32,
+                                  c_int32, c_void_p]
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_device_status.restype = st
@@ -194,6 +199,21 @@ def photon_converter(ctx, x, w, w_layout, bias, U, B=None, stream=None) -> None:
         B = x.shape[0]
     _check(load().photon_converter(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(U), int(B),
                                    _stream(stream)), "photon_converter")
+
+
+def photon_rmsnorm(ctx, x, gamma, eps, out, rows=None, cols=None, stream=None) -> None:
+    rows = x.shape[0] if rows is None else rows
+    cols = x.shape[1] if cols is None else cols
+    _check(load().photon_rmsnorm(ctx, _ptr(x), _ptr(gamma), c_float(eps), _ptr(out), int(rows), int(cols),
+                                 _stream(stream)), "photon_rmsnorm")
+
+
+def photon_linear(ctx, x, w, w_layout, bias, y, B=None, K=None, N=None, stream=None) -> None:
+    B = x.shape[0] if B is None else B
+    K = x.shape[1] if K is None else K
+    N = y.shape[1] if N is None else N
+    _check(load().photon_linear(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(y), int(B), int(K), int(N),
+                                _stream(stream)), "photon_linear")
 
 
 def photon_chunk_causal_attn(ctx, chunks: photon_kv, q, slot, out, Nc=None, row0=0, rows=None,

@@ -94,6 +94,7 @@ struct ConvParams {
     int B, D, N;             // N = P * D
     int w_out_major;
     int x_rows;              // filled by the launcher: x rows fetched per K block (16, 32, 64 or 128)
+    int ksplit;              // CTAs (one cluster) sharing an output tile, each on a slice of K; 0 or 1: none
     int32_t *status;
 };
 
@@ -151,6 +152,9 @@ cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStr
                                    long long *launches);
 cudaError_t launch_chunk_causal_attention(photon_ctx *ctx, const CausalParams &p, cudaStream_t st,
                                           long long *launches);
+cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches);
+cudaError_t launch_rmsnorm(const bf16 *x, const bf16 *gamma, float eps, bf16 *out, int rows, int cols,
+                           cudaStream_t st, long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);
 

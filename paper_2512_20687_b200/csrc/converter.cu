@@ -14,6 +14,15 @@
 // an elected lane does the issuing), four warps read the accumulator back with
 // tcgen05.ld, add the bias, round once to bf16 and store.  Every weight element leaves HBM exactly once; at small batch the
 // kernel is bound by that stream, at large batch by the tensor pipe.
+//
+// The same kernel serves any y = x W + b with K and N multiples of 64 (the
+// context chunker's linear map, Section 2.1.1: K = C_L * D, N = D).  When N is
+// so small that the output tiles would leave most SMs without a share of the
+// weight stream, the K range of a tile is split over the CTAs of a thread-block
+// cluster: each accumulates its slice, the others stage their fp32 tile in
+// their (by then free) ring and send it to the first CTA's ring with one bulk
+// copy through distributed shared memory; that CTA adds the tiles in rank order,
+// so the result does not depend on timing.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -60,12 +69,16 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     constexpr int TAIL = RING_BYTES + BM * BK * 2;
     const uint32_t bars = base + TAIL;                           // full[s] +16s, empty[s] +16s+8
     const uint32_t bar_acc = bars + 16 * MAX_STAGES;
+    const uint32_t bar_rx = bar_acc + 8;                         // split K: the other CTAs' tiles have landed here
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen + TAIL + 16 * MAX_STAGES + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * NT, m0 = blockIdx.y * BM;
+    const int ks = p.ksplit;                                     // CTAs (one cluster) that share an output tile
+    const int zr = ks > 1 ? (int)(blockIdx.x % ks) : 0;          // = rank in the cluster: which slice of K
+    const int n0 = (int)(blockIdx.x / ks) * NT, m0 = blockIdx.y * BM;
     constexpr int MMA_WARPS = mma_warps<NT>();
-    const int n_atoms = p.D / BK;
+    const uint32_t stg_bytes = (uint32_t)p.x_rows * NT * 4;      // the fetched rows of one fp32 tile, stored [column][row]
+    const int a_lo = (p.D / BK) * zr / ks, n_atoms = (p.D / BK) * (zr + 1) / ks - a_lo;
     const int n_steps = (n_atoms + KA - 1) / KA;
 
     if (threadIdx.x == 0) {
@@ -74,7 +87,9 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             ptx::mbar_init(bars + 16 * s + 8, 1);
         }
         ptx::mbar_init(bar_acc, MMA_WARPS);
+        ptx::mbar_init(bar_rx, 1);
         ptx::mbar_fence_init();
+        if (ks > 1 && zr == 0) ptx::mbar_arrive_expect_tx(bar_rx, (ks - 1) * stg_bytes);
         ptx::prefetch_tmap(&tm_x); ptx::prefetch_tmap(&tm_w);
     }
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), MMA_WARPS * NT);
@@ -99,7 +114,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             if (ptx::elect_one()) {
                 ptx::mbar_arrive_expect_tx(full, atoms * (a_bytes + T::B_BYTES));
                 for (int j = 0; j < atoms; ++j) {
-                    const int k0 = (st * KA + j) * BK;
+                    const int k0 = (a_lo + st * KA + j) * BK;
                     ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, k0, m0, full);              // x[m0.., k0..]
                     if (!W_IN_MAJOR) {
                         ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);       // W[n0.., k0..]  (K-major)
@@ -155,13 +170,24 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             __syncwarp();
             if (++s == n_stages) { s = 0; phase ^= 1; }
         }
-    } else if (warp >= 2 && warp <= 5) {
-        // epilogue: warp w reads TMEM lanes [32*(w%4), +32) = batch rows m0 + that range
-        const int quad = warp & 3;
-        const int b = m0 + quad * 32 + lane;
-        const bool ok = ptx::mbar_wait(bar_acc, 0);
+    }
+    // epilogue: warp w (2..5) reads TMEM lanes [32*(w%4), +32) = batch rows m0 + that range
+    const bool epi = warp >= 2 && warp <= 5;
+    const int quad = warp & 3;
+    bool ok = true;
+    if (epi) {
+        ok = ptx::mbar_wait(bar_acc, 0);
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
+    }
+    if (ks > 1) ptx::cluster_sync();        // every CTA of the cluster is done with its ring
+    if (epi) {
+        const int row = quad * 32 + lane, b = m0 + row;
+        if (ks > 1 && zr == 0) {
+            const bool got = ptx::mbar_wait(bar_rx, 0);
+            if (!got && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+            ok = ok && got;
+        }
 #pragma unroll 1
         for (int c0 = 0; c0 < NT; c0 += 32) {
             uint32_t r[32];
@@ -173,6 +199,20 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
                 ptx::tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) + __uint_as_float(r2[e]));
+            }
+            if (zr != 0) {                                 // stage this slice's tile for the first CTA
+                if (row < p.x_rows) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        *reinterpret_cast<uint32_t *>(gen + ((size_t)(c0 + e) * p.x_rows + row) * 4) = r[e];
+                }
+                continue;
+            }
+            for (int z = 1; z < ks && row < p.x_rows; ++z) {   // add the other slices in rank order
+                const float *part = reinterpret_cast<const float *>(gen + (size_t)(z - 1) * stg_bytes);
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    r[e] = __float_as_uint(__uint_as_float(r[e]) + part[(size_t)(c0 + e) * p.x_rows + row]);
             }
             if (ok && b < p.B) {
                 uint4 *dst = reinterpret_cast<uint4 *>(p.U + (size_t)b * p.N + n0 + c0);
@@ -193,7 +233,15 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
                 }
             }
         }
+        if (zr != 0) {
+            ptx::fence_proxy_async();                      // the staged tile is read by the bulk copy
+            ptx::named_bar_sync(1, 128);                   // the four epilogue warps
+            if (warp == 2 && ptx::elect_one())
+                ptx::bulk_copy_to_peer(ptx::map_cluster(base + (uint32_t)(zr - 1) * stg_bytes, 0), base, stg_bytes,
+                                       ptx::map_cluster(bar_rx, 0));
+        }
     }
+    if (ks > 1) ptx::cluster_sync();        // the first CTA has every tile: the senders' rings may go
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -216,13 +264,34 @@ cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launc
     else t = ctx->tmaps.get(p.w, (uint64_t)p.N, (uint64_t)p.D, NT);                 // [N, K], boxes of NT n x 64 k
     if (!t) return cudaErrorInvalidValue;
     mw = *t;
-    dim3 grid(p.N / NT, (p.B + BM - 1) / BM);
-    const cudaError_t e = launch_dependent(converter_umma_kernel<NT, IN_MAJOR>, grid, dim3(CONV_THREADS), T::SMEM, st, 0, p, mx, mw);
+    if (p.ksplit < 1) p.ksplit = 1;
+    dim3 grid(p.ksplit * (p.N / NT), (p.B + BM - 1) / BM);
+    const cudaError_t e = launch_dependent(converter_umma_kernel<NT, IN_MAJOR>, grid, dim3(CONV_THREADS), T::SMEM, st,
+                                           p.ksplit > 1 ? p.ksplit : 0, p, mx, mw);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
+
+// y = x W + b for any K (p.D) and N that are multiples of 64.  Few output tiles: narrow slabs, then the
+// K range split over clusters of 2 or 4 CTAs, as long as a CTA keeps at least 8 K blocks of 64.
+cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches) {
+    if (p.B == 0) return cudaSuccess;
+    const int m_tiles = (p.B + BM - 1) / BM;
+    const bool wide = p.B > 128 && p.N % 128 == 0 && (p.N / 128) * m_tiles * 2 >= ctx->sm_count;
+    const bool wider = wide && p.N % 256 == 0 && (p.N / 256) * m_tiles >= 100;
+    const int nt = wider ? 256 : wide ? 128 : 64;
+    p.ksplit = 1;
+    if (nt == 64)
+        while (p.ksplit < 4 && (p.N / nt) * m_tiles * p.ksplit * 2 <= ctx->sm_count && (p.D / BK) / (p.ksplit * 2) >= 8)
+            p.ksplit *= 2;
+    if (p.w_out_major)
+        return wider ? run<256, false>(ctx, p, st, launches)
+                     : wide ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
+    return wider ? run<256, true>(ctx, p, st, launches)
+                 : wide ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
+}
 
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
     if (p.B == 0) return cudaSuccess;

@@ -249,6 +249,36 @@ photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const phot
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 
+photon_status photon_rmsnorm(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *gamma, float eps,
+                             photon_bf16 *out, int32_t rows, int32_t cols, photon_stream stream) {
+    if (!ctx || rows < 0 || cols <= 0 || cols % 8 != 0) return PHOTON_ERR_INVALID_ARG;
+    if (rows > 0 && (!x || !out)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(gamma) || !aligned16(out) || !(eps >= 0.f)) return PHOTON_ERR_INVALID_ARG;
+    const cudaError_t e = launch_rmsnorm(reinterpret_cast<const bf16 *>(x), reinterpret_cast<const bf16 *>(gamma), eps,
+                                         reinterpret_cast<bf16 *>(out), rows, cols,
+                                         static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w, int32_t w_layout,
+                            const photon_bf16 *bias, photon_bf16 *y, int32_t B, int32_t K, int32_t N,
+                            photon_stream stream) {
+    if (!ctx || B < 0 || K <= 0 || N <= 0 || K % 64 != 0 || N % 64 != 0) return PHOTON_ERR_INVALID_ARG;
+    if (B > 0 && (!x || !w || !y)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias)) return PHOTON_ERR_INVALID_ARG;
+    if (w_layout != PHOTON_W_IN_MAJOR && w_layout != PHOTON_W_OUT_MAJOR) return PHOTON_ERR_INVALID_ARG;
+    ConvParams p{};
+    p.x = reinterpret_cast<const bf16 *>(x);
+    p.w = reinterpret_cast<const bf16 *>(w);
+    p.bias = reinterpret_cast<const bf16 *>(bias);
+    p.U = reinterpret_cast<bf16 *>(y);
+    p.B = B; p.D = K; p.N = N;
+    p.w_out_major = (w_layout == PHOTON_W_OUT_MAJOR);
+    p.status = ctx->status;
+    const cudaError_t e = launch_linear(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
 photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {
     if (!ctx || !a || !a->coarse) return PHOTON_ERR_INVALID_ARG;
     const photon_config &c = ctx->cfg;
