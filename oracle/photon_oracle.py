@@ -212,6 +212,55 @@ def chunker(x, gamma, eps, w, bias=None, w_out_major=False, n_threads=1):
     return xn, linear(xn, w, bias, w_out_major=w_out_major, n_threads=n_threads)
 
 
+def rope_split(qkv, pos, Hq, Hkv, dh, theta=10000.0):
+    """Split a fused projection [n, (Hq + 2 Hkv) dh] into q, k, v and rotate q and k
+    by the item's position (half-split pairing, base theta).  Returns float64
+    (q [n, Hq, dh], k [n, Hkv, dh], v [n, Hkv, dh])."""
+    qkv, pos = _u16(qkv), _i32(pos)
+    n = qkv.shape[0]
+    assert qkv.shape[1] == (Hq + 2 * Hkv) * dh and dh % 2 == 0
+    q = np.empty((n, Hq, dh)); k = np.empty((n, Hkv, dh)); v = np.empty((n, Hkv, dh))
+    lib().oracle_rope_split(_p(qkv), _p(pos), n, Hq, Hkv, dh, ctypes.c_double(theta), _p(q), _p(k), _p(v))
+    return q, k, v
+
+
+def swiglu(gu):
+    """silu(gate) * up for gu [n, 2F] = [gate | up].  Returns float64 [n, F]."""
+    gu = _u16(gu)
+    n, F2 = gu.shape
+    out = np.empty((n, F2 // 2))
+    lib().oracle_swiglu(_p(gu), n, F2 // 2, _p(out))
+    return out
+
+
+def encoder_step(x, lw, cache, scale, eps=1e-5, theta=10000.0, n_threads=1):
+    """STEP of one LLaMA layer of the top-level context encoder for the newest
+    latent of every sequence (Eq. 12 / Eq. 13 with the layer written out): x [B, D]
+    -> normalise -> fused q/k/v projection -> rotary encoding at position len[b]
+    -> append k, v -> attention over the grown cache -> output projection + residual
+    -> normalise -> gate/up projection -> silu(g) * u -> down projection + residual.
+    Every intermediate is rounded to bf16 where the next part reads it.  lw: dict of
+    bf16 weights g1 [D], wqkv [D, (Hq+2Hkv) dh], wo [Hq dh, D], g2 [D], wgu [D, 2F],
+    wdown [F, D] (all in-major).  cache: dict k, v [B, Hkv, cap, dh], len [B] (grown
+    in place).  Returns dict of the bf16 intermediates and y (float64 [B, D])."""
+    B, D = x.shape
+    Hkv, dh = cache["k"].shape[1], cache["k"].shape[3]
+    Hq = lw["wo"].shape[0] // dh
+    n1 = round_bf16(rmsnorm(x, lw["g1"], eps))
+    qkv = round_bf16(linear(n1, lw["wqkv"], n_threads=n_threads))
+    q, k_new, v_new = (round_bf16(t) for t in rope_split(qkv, cache["len"], Hq, Hkv, dh, theta))
+    flags = kv_append(cache["k"], cache["v"], cache["len"], k_new, v_new)
+    att, _ = attention(q, cache["k"], cache["v"], cache["len"], scale, n_threads=n_threads)
+    att = round_bf16(att).reshape(B, Hq * dh)
+    h = round_bf16(linear(att, lw["wo"], n_threads=n_threads) + widen_bf16(x))
+    n2 = round_bf16(rmsnorm(h, lw["g2"], eps))
+    gu = round_bf16(linear(n2, lw["wgu"], n_threads=n_threads))
+    act = round_bf16(swiglu(gu))
+    y = linear(act, lw["wdown"], n_threads=n_threads) + widen_bf16(h)
+    return {"n1": n1, "qkv": qkv, "q": q, "k_new": k_new, "v_new": v_new, "att": att, "h": h, "n2": n2,
+            "gu": gu, "act": act, "y": y, "flags": flags}
+
+
 def round_bf16(x):
     """float64 -> bf16 bits, round to nearest even."""
     x = np.ascontiguousarray(x, dtype=np.float64)

@@ -230,6 +230,23 @@ def chunker_inputs(cfg: DecodeConfig, replica: int = 0, block: int = 4) -> dict:
     }
 
 
+def encoder_layer_inputs(cfg: DecodeConfig, F: int | None = None, replica: int = 0) -> dict:
+    """Weights of one LLaMA layer of the top-level encoder (in-major, variance 1/K
+    each, norm scales around 1) and the step's input x [B, D].  F defaults to the
+    multiple of 64 nearest to 2.75 D (5632 for D = 2048, the usual 1B-class width)."""
+    tag = f"r{replica}"
+    D, dh, Hq, Hkv = cfg.D, cfg.dh, cfg.Hq, cfg.Hkv
+    F = F or max(64, int(round(2.75 * D / 64)) * 64)
+    one = lambda name, n: f32_to_bf16_bits(
+        (bf16_bits_to_f64(normal_bf16(cfg.seed, f"{name}/{tag}", (n,), std=0.1)) + 1.0).astype(np.float32))
+    mat = lambda name, k, n: normal_bf16(cfg.seed, f"{name}/{tag}", (k, n), std=k ** -0.5)
+    return {
+        "x": normal_bf16(cfg.seed, f"enc_x/{tag}", (cfg.B, D)), "F": F,
+        "g1": one("enc_g1", D), "wqkv": mat("enc_wqkv", D, (Hq + 2 * Hkv) * dh), "wo": mat("enc_wo", Hq * dh, D),
+        "g2": one("enc_g2", D), "wgu": mat("enc_wgu", D, 2 * F), "wdown": mat("enc_wdown", F, D),
+    }
+
+
 def chunk_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False,
                  strict_paper: bool = False) -> dict:
     """Chunk-local tensors: Nc in-flight chunks, each a cache of cap = P + C
