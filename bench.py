@@ -493,6 +493,43 @@ def run_gpu(args, cfg) -> None:
         del cw
         torch.cuda.empty_cache()
 
+        # STEP of one LLaMA layer of the top-level encoder (normalise, q/k/v, rotary, append, attention, output
+        # projection, MLP) on the step's own caches: ten launches; weights rotate over the replicas
+        if cfg.Hq * cfg.dh == cfg.D:
+            li = wl.encoder_layer_inputs(cfg)
+            F = li["F"]
+            names = ("g1", "wqkv", "wo", "g2", "wgu", "wdown")
+            lw0 = {n: dev_bf16(np.ascontiguousarray(li[n].T) if out_major and li[n].ndim == 2 else li[n]) for n in names}
+            layers = []
+            for r in range(R):
+                wr = lw0 if r == 0 else {n: (t.clone() if t.dim() == 2 else t) for n, t in lw0.items()}
+                layers.append(ph.make_layer(*(wr[n] for n in names), layout, F))
+            scr = ph.make_layer_scratch(cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, F, dev, torch.bfloat16)
+            ex = dev_bf16(li["x"])
+            ey = torch.empty_like(ex)
+            plain_kv = [ph.make_kv(t["k"], t["v"], lens[r], max_len=cfg.S) for r, t in enumerate(reps)]
+            turn["i"] = -1
+
+            def layer_call(t):
+                i = turn["i"] = turn["i"] + 1
+                ph.photon_encoder_step(ctx, layers[i % R], scr, ex, plain_kv[i % R], ey, scale=scale)
+
+            lens.copy_(lens0)
+            us_e = graph_time_us(layer_call, reset_lens=True)
+            lens.copy_(lens0)
+            QKV = (cfg.Hq + 2 * cfg.Hkv) * cfg.dh
+            wbytes = 2 * (cfg.D * QKV + cfg.D * cfg.D + cfg.D * 2 * F + F * cfg.D)
+            ebytes = wbytes + cfg.B * cfg.S * cfg.Hkv * cfg.dh * 4
+            eflops = 2.0 * cfg.B * (wbytes / 2)
+            widened["encoder_step"] = {
+                "workload": "one layer, batch %d: D %d, %dq/%dkv x %d, F %d, cache of %d latents per sequence" % (
+                    cfg.B, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh, F, cfg.S),
+                "us": us_e, "launches": 10, "algorithmic_bytes": ebytes, "GBps": ebytes / us_e * 1e-3,
+                "frac_hbm": ebytes / us_e * 1e-3 / hbm_peak, "TFLOPs": eflops / us_e * 1e-6,
+                "note": "weights and the sequences' own K/V rows counted once (no shared prefix), activations not counted"}
+            del layers, lw0
+            torch.cuda.empty_cache()
+
     # roofline of the dominant kernel = the attention part that takes the longest
     dom = max(("coarse_attn", "chunk_attn"), key=lambda n: kernels[n]["us"])
     def recorded_traffic(kernel_name):

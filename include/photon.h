@@ -155,17 +155,68 @@ photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const phot
  * x, out [rows, cols] bf16 (out may alias x), gamma [cols] or NULL (ones),
  * cols a multiple of 8, eps >= 0; fp32 sums, one rounding to bf16.
  *
- * photon_linear: y[b, n] = sum_k x[b, k] * W[k, n] (+ bias[n]); x [B, K], w in
- * the order given by w_layout ([K, N] or [N, K]), bias [N] or NULL, y [B, N];
- * K and N multiples of 64 (else INVALID_ARG); bf16 in, fp32 accumulation on the
- * tensor cores, one rounding at the output; deterministic.  The converter is
- * the case K = D, N = P * D.  All pointers device, 16-byte aligned, owned by
- * the caller; one kernel each on `stream`, no workspace. */
+ * photon_linear: y[b, n] = sum_k x[b, k] * W[k, n] (+ bias[n]) (+ residual[b, n]);
+ * x [B, K], w in the order given by w_layout ([K, N] or [N, K]), bias [N] or
+ * NULL, residual [B, N] or NULL (may alias y), y [B, N]; K and N multiples of
+ * 64 (else INVALID_ARG); bf16 in, fp32 accumulation on the tensor cores, one
+ * rounding at the output; deterministic.  The converter is the case K = D,
+ * N = P * D.  All pointers device, 16-byte aligned, owned by the caller; one
+ * kernel each on `stream`, no workspace. */
 photon_status photon_rmsnorm(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *gamma, float eps,
                              photon_bf16 *out, int32_t rows, int32_t cols, photon_stream stream);
 photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w, int32_t w_layout,
-                            const photon_bf16 *bias, photon_bf16 *y, int32_t B, int32_t K, int32_t N,
+                            const photon_bf16 *bias, const photon_bf16 *residual, photon_bf16 *y, int32_t B,
+                            int32_t K, int32_t N, photon_stream stream);
+
+/* The rest of one LLaMA layer of the top-level context encoder around the
+ * attention of STEP (Eq. 12 / Eq. 13; Section 3.1: every model is a LLaMA
+ * Transformer).  The paper fixes neither the rotary convention nor its base:
+ * the half-split pairing (feature j with j + dh/2) and the base `theta` given
+ * by the caller (10000 in the LLaMA reference) are used.
+ *
+ * photon_rope_split: qkv [n, (Hq + 2 Hkv) dh], the fused projection of n new
+ * latents, is taken apart into q [n, Hq, dh], k [n, Hkv, dh], v [n, Hkv, dh]
+ * (what photon_kv_append and photon_coarse_attn read); every head of q and k
+ * is rotated by the item's position pos[i] (device int32; for a decode step
+ * the cache length before the append).  Heads are those of the context.
+ *
+ * photon_swiglu: out[i, f] = silu(gu[i, f]) * gu[i, F + f]; gu [n, 2F], out
+ * [n, F], F a multiple of 8.
+ *
+ * photon_encoder_step: the whole layer for the newest latent of every
+ * sequence, ten kernels on `stream`: normalise x (g1) -> wqkv -> rope_split
+ * at position len[b] -> append k, v to `cache` (len += 1) -> attention over
+ * the grown cache -> wo + x -> normalise (g2) -> wgu -> swiglu -> wdown + h.
+ * x, y [B, D] with B = cache->n_units and D = Hq * dh of the context;
+ * weights in the order w_layout names: wqkv [D, (Hq + 2 Hkv) dh], wo [Hq dh,
+ * D], wgu [D, 2F], wdown [F, D]; g1, g2 [D].  F a multiple of 64.  The
+ * caller owns the intermediates in `scratch` (sizes beside the fields); each
+ * is rounded to bf16 where the next kernel reads it.  y may alias x. */
+typedef struct photon_layer {
+  const photon_bf16 *g1, *wqkv, *wo, *g2, *wgu, *wdown;
+  int32_t w_layout;          /* PHOTON_W_IN_MAJOR or PHOTON_W_OUT_MAJOR, all four weights */
+  int32_t F;                 /* width of the MLP */
+  float eps;                 /* of both normalisations */
+  float theta;               /* rotary base */
+} photon_layer;
+typedef struct photon_layer_scratch {
+  photon_bf16 *n;            /* [B, D]   normalised input of either half */
+  photon_bf16 *qkv;          /* [B, (Hq + 2 Hkv) dh] */
+  photon_bf16 *q;            /* [B, Hq, dh] */
+  photon_bf16 *k_new, *v_new;/* [B, Hkv, dh] */
+  photon_bf16 *att;          /* [B, Hq, dh] */
+  photon_bf16 *h;            /* [B, D]   after the attention half */
+  photon_bf16 *gu;           /* [B, 2F] */
+  photon_bf16 *act;          /* [B, F] */
+} photon_layer_scratch;
+photon_status photon_rope_split(photon_ctx *ctx, const photon_bf16 *qkv, const int32_t *pos, int32_t n,
+                                float theta, photon_bf16 *q, photon_bf16 *k, photon_bf16 *v,
+                                photon_stream stream);
+photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 *out, int32_t n, int32_t F,
                             photon_stream stream);
+photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
+                                  const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
+                                  photon_stream stream);
 
 /* Bounded causal attention of the local decoders G^(l) (Eq. 6-7): query c
  * (q [Nc, Hq, dh]) attends rows [0, len[u]) of chunk buffer u = slot ?

@@ -53,6 +53,15 @@ class photon_step_args(Structure):
     ]
 
 
+class photon_layer(Structure):
+    _fields_ = [(n, c_void_p) for n in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")] + [
+        ("w_layout", c_int32), ("F", c_int32), ("eps", c_float), ("theta", c_float)]
+
+
+class photon_layer_scratch(Structure):
+    _fields_ = [(n, c_void_p) for n in ("n", "qkv", "q", "k_new", "v_new", "att", "h", "gu", "act")]
+
+
 _lib = None
 
 
@@ -93,8 +102,16 @@ def load() -> ctypes.CDLL:
     lib.photon_rmsnorm.restype = st
     lib.photon_rmsnorm.argtypes = [c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_int32, c_int32, c_void_p]
     lib.photon_linear.restype = st
-    lib.photon_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32,
-                                  c_int32, c_void_p]
+    lib.photon_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
+                                  c_int32, c_int32, c_void_p]
+    lib.photon_rope_split.restype = st
+    lib.photon_rope_split.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_float, c_void_p, c_void_p,
+                                      c_void_p, c_void_p]
+    lib.photon_swiglu.restype = st
+    lib.photon_swiglu.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p]
+    lib.photon_encoder_step.restype = st
+    lib.photon_encoder_step.argtypes = [c_void_p, POINTER(photon_layer), POINTER(photon_layer_scratch), c_void_p,
+                                        POINTER(photon_kv), c_void_p, c_float, c_void_p]
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_device_status.restype = st
@@ -208,12 +225,51 @@ def photon_rmsnorm(ctx, x, gamma, eps, out, rows=None, cols=None, stream=None) -
                                  _stream(stream)), "photon_rmsnorm")
 
 
-def photon_linear(ctx, x, w, w_layout, bias, y, B=None, K=None, N=None, stream=None) -> None:
+def photon_linear(ctx, x, w, w_layout, bias, y, B=None, K=None, N=None, residual=None, stream=None) -> None:
     B = x.shape[0] if B is None else B
     K = x.shape[1] if K is None else K
     N = y.shape[1] if N is None else N
-    _check(load().photon_linear(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(y), int(B), int(K), int(N),
-                                _stream(stream)), "photon_linear")
+    _check(load().photon_linear(ctx, _ptr(x), _ptr(w), int(w_layout), _ptr(bias), _ptr(residual), _ptr(y), int(B),
+                                int(K), int(N), _stream(stream)), "photon_linear")
+
+
+def photon_rope_split(ctx, qkv, pos, q, k, v, theta=10000.0, n=None, stream=None) -> None:
+    n = qkv.shape[0] if n is None else n
+    _check(load().photon_rope_split(ctx, _ptr(qkv), _ptr(pos), int(n), c_float(theta), _ptr(q), _ptr(k), _ptr(v),
+                                    _stream(stream)), "photon_rope_split")
+
+
+def photon_swiglu(ctx, gu, out, n=None, F=None, stream=None) -> None:
+    n = gu.shape[0] if n is None else n
+    F = gu.shape[1] // 2 if F is None else F
+    _check(load().photon_swiglu(ctx, _ptr(gu), _ptr(out), int(n), int(F), _stream(stream)), "photon_swiglu")
+
+
+def make_layer(g1, wqkv, wo, g2, wgu, wdown, w_layout, F, eps=1e-5, theta=10000.0) -> photon_layer:
+    L = photon_layer()
+    L.g1, L.wqkv, L.wo, L.g2, L.wgu, L.wdown = (_ptr(t) for t in (g1, wqkv, wo, g2, wgu, wdown))
+    L.w_layout, L.F, L.eps, L.theta = int(w_layout), int(F), eps, theta
+    L._keep = (g1, wqkv, wo, g2, wgu, wdown)
+    return L
+
+
+def make_layer_scratch(B, Hq, Hkv, dh, F, device, dtype) -> photon_layer_scratch:
+    """Allocates the intermediates of photon_encoder_step with torch (the caller owns them)."""
+    import torch
+    D = Hq * dh
+    shapes = {"n": (B, D), "qkv": (B, (Hq + 2 * Hkv) * dh), "q": (B, Hq, dh), "k_new": (B, Hkv, dh),
+              "v_new": (B, Hkv, dh), "att": (B, Hq, dh), "h": (B, D), "gu": (B, 2 * F), "act": (B, F)}
+    sc = photon_layer_scratch()
+    sc.tensors = {k: torch.empty(v, dtype=dtype, device=device) for k, v in shapes.items()}
+    for k, t in sc.tensors.items():
+        setattr(sc, k, _ptr(t))
+    return sc
+
+
+def photon_encoder_step(ctx, layer: photon_layer, scratch: photon_layer_scratch, x, cache: photon_kv, y,
+                        scale=1.0, stream=None) -> None:
+    _check(load().photon_encoder_step(ctx, byref(layer), byref(scratch), _ptr(x), byref(cache), _ptr(y),
+                                      c_float(scale), _stream(stream)), "photon_encoder_step")
 
 
 def photon_chunk_causal_attn(ctx, chunks: photon_kv, q, slot, out, Nc=None, row0=0, rows=None,

@@ -216,12 +216,16 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             }
             if (ok && b < p.B) {
                 uint4 *dst = reinterpret_cast<uint4 *>(p.U + (size_t)b * p.N + n0 + c0);
+                const uint4 *res = p.residual ? reinterpret_cast<const uint4 *>(p.residual + (size_t)b * p.N + n0 + c0) : nullptr;
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     uint32_t w[4];
+                    const uint4 rv = res ? res[v] : make_uint4(0u, 0u, 0u, 0u);
+                    const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        float f0 = __uint_as_float(r[v * 8 + 2 * e]), f1 = __uint_as_float(r[v * 8 + 2 * e + 1]);
+                        float f0 = __uint_as_float(r[v * 8 + 2 * e]) + bf16_lo(rw[e]);
+                        float f1 = __uint_as_float(r[v * 8 + 2 * e + 1]) + bf16_hi(rw[e]);
                         if (p.bias) {
                             f0 += __bfloat162float(p.bias[n0 + c0 + v * 8 + 2 * e]);
                             f1 += __bfloat162float(p.bias[n0 + c0 + v * 8 + 2 * e + 1]);

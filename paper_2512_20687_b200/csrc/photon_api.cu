@@ -261,22 +261,77 @@ photon_status photon_rmsnorm(photon_ctx *ctx, const photon_bf16 *x, const photon
 }
 
 photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_bf16 *w, int32_t w_layout,
-                            const photon_bf16 *bias, photon_bf16 *y, int32_t B, int32_t K, int32_t N,
-                            photon_stream stream) {
+                            const photon_bf16 *bias, const photon_bf16 *residual, photon_bf16 *y, int32_t B,
+                            int32_t K, int32_t N, photon_stream stream) {
     if (!ctx || B < 0 || K <= 0 || N <= 0 || K % 64 != 0 || N % 64 != 0) return PHOTON_ERR_INVALID_ARG;
     if (B > 0 && (!x || !w || !y)) return PHOTON_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(bias) || !aligned16(residual))
+        return PHOTON_ERR_INVALID_ARG;
     if (w_layout != PHOTON_W_IN_MAJOR && w_layout != PHOTON_W_OUT_MAJOR) return PHOTON_ERR_INVALID_ARG;
     ConvParams p{};
     p.x = reinterpret_cast<const bf16 *>(x);
     p.w = reinterpret_cast<const bf16 *>(w);
     p.bias = reinterpret_cast<const bf16 *>(bias);
+    p.residual = reinterpret_cast<const bf16 *>(residual);
     p.U = reinterpret_cast<bf16 *>(y);
     p.B = B; p.D = K; p.N = N;
     p.w_out_major = (w_layout == PHOTON_W_OUT_MAJOR);
     p.status = ctx->status;
     const cudaError_t e = launch_linear(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_rope_split(photon_ctx *ctx, const photon_bf16 *qkv, const int32_t *pos, int32_t n,
+                                float theta, photon_bf16 *q, photon_bf16 *k, photon_bf16 *v,
+                                photon_stream stream) {
+    if (!ctx || n < 0 || !(theta > 1.f)) return PHOTON_ERR_INVALID_ARG;
+    if (n > 0 && (!qkv || !pos || !q || !k || !v)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(qkv) || !aligned16(q) || !aligned16(k) || !aligned16(v)) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    const cudaError_t e = launch_rope_split(reinterpret_cast<const bf16 *>(qkv), pos, n, c.Hq, c.Hkv, c.dh, theta,
+                                            reinterpret_cast<bf16 *>(q), reinterpret_cast<bf16 *>(k),
+                                            reinterpret_cast<bf16 *>(v), static_cast<cudaStream_t>(stream),
+                                            &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 *out, int32_t n, int32_t F,
+                            photon_stream stream) {
+    if (!ctx || n < 0 || F <= 0 || F % 8 != 0) return PHOTON_ERR_INVALID_ARG;
+    if (n > 0 && (!gu || !out)) return PHOTON_ERR_INVALID_ARG;
+    if (!aligned16(gu) || !aligned16(out)) return PHOTON_ERR_INVALID_ARG;
+    const cudaError_t e = launch_swiglu(reinterpret_cast<const bf16 *>(gu), reinterpret_cast<bf16 *>(out), n, F,
+                                        static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc,
+                                  const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
+                                  photon_stream stream) {
+    if (!ctx || !L || !sc || !cache || !x || !y) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    // everything is validated before the first launch, so that a bad argument leaves no partial step behind
+    if (!kv_ok(ctx, cache, false) || c.Hq * c.dh != c.D || L->F <= 0 || L->F % 64 != 0) return PHOTON_ERR_INVALID_ARG;
+    if (!L->g1 || !L->wqkv || !L->wo || !L->g2 || !L->wgu || !L->wdown || !(L->eps >= 0.f) || !(L->theta > 1.f))
+        return PHOTON_ERR_INVALID_ARG;
+    if (L->w_layout != PHOTON_W_IN_MAJOR && L->w_layout != PHOTON_W_OUT_MAJOR) return PHOTON_ERR_INVALID_ARG;
+    const void *ptrs[] = {L->g1, L->wqkv, L->wo, L->g2, L->wgu, L->wdown, sc->n, sc->qkv, sc->q, sc->k_new,
+                          sc->v_new, sc->att, sc->h, sc->gu, sc->act, x, y};
+    for (const void *q : ptrs)
+        if (!q || !aligned16(q)) return PHOTON_ERR_INVALID_ARG;
+    const int B = cache->n_units, D = c.D, QKV = (c.Hq + 2 * c.Hkv) * c.dh;
+    if ((size_t)B * c.Hkv > ctx->n_tickets) return PHOTON_ERR_WORKSPACE;
+    photon_status s = photon_rmsnorm(ctx, x, L->g1, L->eps, sc->n, B, D, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wqkv, L->w_layout, nullptr, nullptr, sc->qkv, B, D, QKV, stream);
+    if (s == PHOTON_OK) s = photon_rope_split(ctx, sc->qkv, cache->len, B, L->theta, sc->q, sc->k_new, sc->v_new, stream);
+    if (s == PHOTON_OK) s = photon_kv_append(ctx, cache, sc->k_new, sc->v_new, nullptr, B, 1, stream);
+    if (s == PHOTON_OK) s = photon_coarse_attn(ctx, cache, sc->q, sc->att, nullptr, scale, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->att, L->wo, L->w_layout, nullptr, x, sc->h, B, D, D, stream);
+    if (s == PHOTON_OK) s = photon_rmsnorm(ctx, sc->h, L->g2, L->eps, sc->n, B, D, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, B, D, 2 * L->F, stream);
+    if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, B, L->F, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->act, L->wdown, L->w_layout, nullptr, sc->h, y, B, L->F, D, stream);
+    return s;
 }
 
 photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {

@@ -33,6 +33,26 @@ def assert_close(got_f64: np.ndarray, want_f64: np.ndarray, what: str = ""):
     assert err.mean() <= MEAN_ABS, f"{what}: mean abs err {err.mean():.4g} > {MEAN_ABS}"
 
 
+def assert_close_scaled(got_f64: np.ndarray, want_f64: np.ndarray, what: str = "", slack: float = 1.0):
+    """The same bar for values that leave the range the bar was set for: 2e-2 covers the
+    bf16 rounding of magnitudes up to 2 with a margin; a value of magnitude m > 2 has a bf16
+    step m/2 times larger, so its bound grows by that factor.  Rounding a value to bf16 alone
+    costs a quarter of its bf16 step on average (about 2e-3 already for magnitudes between 1
+    and 2), so the mean bound is the usual 2e-3 or twice that pure-rounding mean, whichever
+    is larger: chained roundings may cost as much again as the last one.  `slack` widens
+    both bounds for the outputs of a chain of kernels, where a one-step difference in an
+    intermediate of magnitude m moves what depends on it by up to m * 2^-7."""
+    assert got_f64.shape == want_f64.shape, (got_f64.shape, want_f64.shape)
+    assert np.isfinite(got_f64).all(), f"{what}: non-finite output"
+    err = np.abs(got_f64 - want_f64)
+    bound = slack * MAX_ABS * np.maximum(1.0, np.abs(want_f64) / 2.0)
+    worst = (err / bound).max()
+    assert worst <= 1.0, f"{what}: abs err reaches {worst:.3g} of its bound"
+    step = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want_f64), 2.0 ** -20))) - 7)
+    mean_bound = slack * max(MEAN_ABS, 0.5 * float(step.mean()))
+    assert err.mean() <= mean_bound, f"{what}: mean abs err {err.mean():.4g} > {mean_bound:.4g}"
+
+
 class Ctx:
     def __init__(self, cfg, max_queries=None, max_splits=0):
         self.cfg = cfg

@@ -50,6 +50,8 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(ph.photon_kv) == 24 + 16 + 32 + 16
     assert ph.photon_kv.max_len.offset == 32 and ph.photon_kv.k_shared.offset == 40
     assert ph.photon_step_args.scale_coarse.offset == 48 and ph.photon_step_args.x.offset == 56
+    assert ctypes.sizeof(ph.photon_layer) == 6 * 8 + 4 * 4 and ph.photon_layer.F.offset == 52
+    assert ctypes.sizeof(ph.photon_layer_scratch) == 9 * 8
 
 
 def test_status_strings(lib):

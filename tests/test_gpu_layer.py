@@ -1,0 +1,169 @@
+"""Parity of the remaining kernels of an encoder layer (rotary encoding with the
+split of the fused projection, gated activation, residual in the linear map) and
+of the composed STEP of one layer with the CPU oracle, through the C boundary.
+bf16 outputs: max abs error 2e-2, mean abs error 2e-3 against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_20687_b200 as ph
+from paper_2512_20687_b200 import workloads as wl
+
+from gpu_util import Ctx, assert_close, assert_close_scaled, dev_bf16, dev_i32, host_bits, host_f64
+
+pytestmark = pytest.mark.gpu
+
+NT = 16     # oracle threads
+
+
+def cfg_small(i, **kw):
+    return wl.scaled(wl.CONFIGS[i], **kw)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 4])
+def test_rope_split_matches_oracle(oracle, idx):
+    cfg = cfg_small(idx, B=37)
+    Hq, Hkv, dh = cfg.Hq, cfg.Hkv, cfg.dh
+    qkv = wl.normal_bf16(41, "qkv", (cfg.B, (Hq + 2 * Hkv) * dh))
+    pos = (np.arange(cfg.B) * 229 % 8192).astype(np.int32)
+    pos[:3] = [0, 1, 8191]
+    wq, wk, wv = oracle.rope_split(qkv, pos, Hq, Hkv, dh, 10000.0)
+    with Ctx(cfg) as c:
+        q = torch.empty(cfg.B, Hq, dh, dtype=torch.bfloat16, device="cuda")
+        k = torch.empty(cfg.B, Hkv, dh, dtype=torch.bfloat16, device="cuda")
+        v = torch.empty_like(k)
+        ph.photon_rope_split(c.h, dev_bf16(qkv), dev_i32(pos), q, k, v)
+        assert c.status() == 0
+    # a rotation of O(1) values rounded once: within half a bf16 step of the oracle (|x| < 8 here)
+    assert np.abs(host_f64(q) - wq).max() <= 2.0 ** -6 and np.abs(host_f64(k) - wk).max() <= 2.0 ** -6
+    assert_close(host_f64(q), wq, "rope q")
+    assert_close(host_f64(k), wk, "rope k")
+    assert np.array_equal(host_bits(v).reshape(cfg.B, -1), qkv[:, (Hq + Hkv) * dh:])       # v: a bit copy
+    assert np.array_equal(host_bits(q)[0].reshape(-1), qkv[0, : Hq * dh])                   # position 0: identity
+
+
+@pytest.mark.parametrize("n,F", [(64, 5632), (3, 8), (513, 1024)])
+def test_swiglu_matches_oracle(oracle, n, F):
+    gu = wl.normal_bf16(42, "gu", (n, 2 * F), std=1.5)
+    want = oracle.swiglu(gu)
+    with Ctx(cfg_small(0)) as c:
+        out = torch.empty(n, F, dtype=torch.bfloat16, device="cuda")
+        ph.photon_swiglu(c.h, dev_bf16(gu), out)
+        assert c.status() == 0
+    got = host_f64(out)
+    # one rounding to bf16 (half a step is 2^-9 relative) on top of a fast exponential
+    assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-4)
+
+
+@pytest.mark.parametrize("B,K,N", [(64, 2048, 2048), (200, 1024, 8192)])
+def test_linear_adds_the_residual_before_rounding(oracle, B, K, N):
+    x = wl.normal_bf16(43, "x", (B, K))
+    w = wl.normal_bf16(43, "w", (K, N), std=K ** -0.5)
+    res = wl.normal_bf16(43, "r", (B, N))
+    want = oracle.linear(x, w, n_threads=NT) + wl.bf16_bits_to_f64(res)
+    with Ctx(cfg_small(0)) as c:
+        y = dev_bf16(res).clone()                                       # the residual aliases the output
+        ph.photon_linear(c.h, dev_bf16(x), dev_bf16(w), ph.PHOTON_W_IN_MAJOR, None, y, residual=y)
+        assert c.status() == 0
+    assert_close(host_f64(y), want, "linear + residual")
+
+
+@pytest.mark.parametrize("idx,B,S,F", [(0, 5, 40, 128), (1, 64, 512, 5632), (4, 130, 128, 2816)])
+def test_encoder_step_matches_oracle(oracle, idx, B, S, F):
+    """STEP of one layer: every intermediate that the next kernel reads, the grown
+    cache (bit-exact given the same appended rows) and the layer's output."""
+    cfg = cfg_small(idx, B=B, S=S)
+    lw = wl.encoder_layer_inputs(cfg, F=F)
+    co = wl.coarse_inputs(cfg, poison=True)
+    lens = (co["len"] - (np.arange(B) % 7)).clip(0).astype(np.int32)     # ragged positions
+    for u, n in enumerate(lens):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0x7FC1
+    scale = cfg.dh ** -0.5
+    cache = {"k": co["k"].copy(), "v": co["v"].copy(), "len": lens.copy()}
+    want = oracle.encoder_step(lw["x"], lw, cache, scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        dk, dv, dl = dev_bf16(co["k"]), dev_bf16(co["v"]), dev_i32(lens)
+        kv = ph.make_kv(dk, dv, dl)
+        W = {n: dev_bf16(lw[n]) for n in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")}
+        layer = ph.make_layer(W["g1"], W["wqkv"], W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, F)
+        sc = ph.make_layer_scratch(B, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        x = dev_bf16(lw["x"])
+        y = torch.empty_like(x)
+        ph.photon_encoder_step(c.h, layer, sc, x, kv, y, scale=scale)
+        assert c.status() == 0
+        assert np.array_equal(dl.cpu().numpy(), lens + 1)
+        t = sc.tensors
+        # the chain as a whole: intermediates and output against the oracle's chain, with the slack a
+        # chain of bf16 roundings needs (each kernel by itself is held to the plain bar below)
+        for name in ("n", "qkv", "q", "k_new", "att", "h", "gu", "act"):
+            key = "n2" if name == "n" else name                          # `n` holds the second normalisation at the end
+            got, ref = host_f64(t[name]).reshape(B, -1), wl.bf16_bits_to_f64(want[key]).reshape(B, -1)
+            assert_close_scaled(got, ref, f"encoder step {name}", slack=2.0)
+        # the appended rows are exactly the rotated key and the value the kernel produced
+        hk, hv = host_bits(dk), host_bits(dv)
+        for u in range(B):
+            assert np.array_equal(hk[u, :, lens[u]], host_bits(t["k_new"])[u])
+            assert np.array_equal(hv[u, :, lens[u]], host_bits(t["v_new"])[u])
+    assert_close_scaled(host_f64(y), want["y"], f"encoder step cfg{idx}", slack=2.0)
+
+
+@pytest.mark.parametrize("idx,B,S,F", [(1, 64, 512, 5632)])
+def test_each_kernel_of_the_layer_on_the_oracles_own_intermediates(oracle, idx, B, S, F):
+    """Every kernel of the layer fed with the oracle's bf16 intermediate, so that no
+    difference is carried from one kernel into the next: the plain bar per kernel."""
+    cfg = cfg_small(idx, B=B, S=S)
+    lw = wl.encoder_layer_inputs(cfg, F=F)
+    co = wl.coarse_inputs(cfg)
+    scale = cfg.dh ** -0.5
+    lens = co["len"].copy()
+    cache = {"k": co["k"].copy(), "v": co["v"].copy(), "len": lens.copy()}
+    w = oracle.encoder_step(lw["x"], lw, cache, scale, n_threads=NT)
+    f64 = wl.bf16_bits_to_f64
+    D, Hq, Hkv, dh = cfg.D, cfg.Hq, cfg.Hkv, cfg.dh
+    IN = ph.PHOTON_W_IN_MAJOR
+    with Ctx(cfg) as c:
+        def new(*shape):
+            return torch.empty(shape, dtype=torch.bfloat16, device="cuda")
+        n1, qkv, h, n2, gu, act, y = new(B, D), new(B, (Hq + 2 * Hkv) * dh), new(B, D), new(B, D), new(B, 2 * F), new(B, F), new(B, D)
+        q, k, v, att = new(B, Hq, dh), new(B, Hkv, dh), new(B, Hkv, dh), new(B, Hq, dh)
+        ph.photon_rmsnorm(c.h, dev_bf16(lw["x"]), dev_bf16(lw["g1"]), 1e-5, n1)
+        ph.photon_linear(c.h, dev_bf16(w["n1"]), dev_bf16(lw["wqkv"]), IN, None, qkv)
+        ph.photon_rope_split(c.h, dev_bf16(w["qkv"]), dev_i32(lens), q, k, v)
+        kv = ph.make_kv(dev_bf16(cache["k"]), dev_bf16(cache["v"]), dev_i32(cache["len"]))       # the oracle's grown cache
+        ph.photon_coarse_attn(c.h, kv, dev_bf16(w["q"]), att, None, scale)
+        ph.photon_linear(c.h, dev_bf16(w["att"]), dev_bf16(lw["wo"]), IN, None, h, residual=dev_bf16(lw["x"]))
+        ph.photon_rmsnorm(c.h, dev_bf16(w["h"]), dev_bf16(lw["g2"]), 1e-5, n2)
+        ph.photon_linear(c.h, dev_bf16(w["n2"]), dev_bf16(lw["wgu"]), IN, None, gu)
+        ph.photon_swiglu(c.h, dev_bf16(w["gu"]), act)
+        ph.photon_linear(c.h, dev_bf16(w["act"]), dev_bf16(lw["wdown"]), IN, None, y, residual=dev_bf16(w["h"]))
+        assert c.status() == 0
+    for got, ref, what in ((n1, w["n1"], "norm 1"), (qkv, w["qkv"], "q/k/v projection"), (q, w["q"], "rotated q"),
+                           (k, w["k_new"], "rotated k"), (att, w["att"], "attention"), (h, w["h"], "output projection"),
+                           (n2, w["n2"], "norm 2"), (gu, w["gu"], "gate/up projection"), (act, w["act"], "activation")):
+        assert_close_scaled(host_f64(got).reshape(B, -1), f64(ref).reshape(B, -1), what)
+    assert np.array_equal(host_bits(v), w["v_new"])
+    assert_close_scaled(host_f64(y), w["y"], "down projection")
+
+
+def test_encoder_step_refuses_bad_arguments():
+    cfg = cfg_small(0, B=2, S=8)
+    with Ctx(cfg) as c:
+        co = wl.coarse_inputs(cfg)
+        kv = ph.make_kv(dev_bf16(co["k"]), dev_bf16(co["v"]), dev_i32(co["len"]))
+        lw = wl.encoder_layer_inputs(cfg, F=64)
+        W = {n: dev_bf16(lw[n]) for n in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")}
+        sc = ph.make_layer_scratch(2, cfg.Hq, cfg.Hkv, cfg.dh, 64, "cuda", torch.bfloat16)
+        x = dev_bf16(lw["x"])
+        n0 = ph.photon_launch_count(c.h)
+        for bad in (dict(F=60), dict(theta=1.0), dict(eps=-1.0)):
+            kw = dict(F=64, eps=1e-5, theta=10000.0)
+            kw.update(bad)
+            layer = ph.make_layer(W["g1"], W["wqkv"], W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, **kw)
+            with pytest.raises(ph.PhotonError) as e:
+                ph.photon_encoder_step(c.h, layer, sc, x, kv, x)
+            assert e.value.code == ph.PHOTON_ERR_INVALID_ARG
+        layer = ph.make_layer(W["g1"], None, W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, 64)
+        with pytest.raises(ph.PhotonError):
+            ph.photon_encoder_step(c.h, layer, sc, x, kv, x)
+        assert ph.photon_launch_count(c.h) == n0 and c.status() == 0
