@@ -38,42 +38,47 @@ constexpr int CONV_THREADS = 224;       // warp 0: TMA, warps 1 and 6: MMA (1 ow
 template <int NT> __host__ __device__ constexpr int mma_warps() { return NT <= 64 ? 2 : 1; }
 
 constexpr int MAX_STAGES = 12;
-constexpr int RING_BYTES = 192 * 1024;
+constexpr int RING_BYTES = 192 * 1024;  // one CTA per SM
+// With more output tiles than SMs but no more than two per SM, two CTAs share an SM, each with a smaller
+// ring of single-atom stages, so that the tiles still run as one wave.
+constexpr int RING_BYTES_PAIR = 88 * 1024;
 
 template <int NT>
 struct ConvTile {
     static constexpr int B_BYTES = NT * BK * 2;           // weight atom: 8 / 16 KiB
     // slack after the ring: the MMA reads 128 rows from every x atom, also past a short x box
-    static constexpr int SMEM = RING_BYTES + BM * BK * 2 + 1024 + 512;
+    static constexpr int extra = BM * BK * 2 + 1024 + 512;
+    static constexpr int SMEM = RING_BYTES + extra;
 };
 
-__host__ __device__ inline int conv_stages(int a_bytes, int b_bytes, int ka) {
-    const int s = RING_BYTES / (ka * (a_bytes + b_bytes));
+__host__ __device__ inline int conv_stages(int ring_bytes, int a_bytes, int b_bytes, int ka) {
+    const int s = ring_bytes / (ka * (a_bytes + b_bytes));
     return s < MAX_STAGES ? s : MAX_STAGES;
 }
 
 // The loops of the TMA warp and of the MMA warp are run by the whole warp (so that their
 // address arithmetic stays warp-uniform); one elected lane issues the asynchronous operations.
-template <int NT, bool W_IN_MAJOR>
+template <int NT, bool W_IN_MAJOR, bool PAIR, bool SPLIT>
 __global__ void __launch_bounds__(CONV_THREADS, 1)
 converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
                       const __grid_constant__ CUtensorMap tm_w) {
     using T = ConvTile<NT>;
-    constexpr int KA = atoms_per_stage<NT>();
+    constexpr int KA = PAIR ? 1 : atoms_per_stage<NT>();
+    constexpr int RING = PAIR ? RING_BYTES_PAIR : RING_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
     const int a_bytes = p.x_rows * BK * 2;                       // x atom of this launch
     const int stage_bytes = KA * (a_bytes + T::B_BYTES);         // [x atoms][weight atoms]
-    const int n_stages = conv_stages(a_bytes, T::B_BYTES, KA);
-    constexpr int TAIL = RING_BYTES + BM * BK * 2;
+    const int n_stages = conv_stages(RING, a_bytes, T::B_BYTES, KA);
+    constexpr int TAIL = RING + BM * BK * 2;
     const uint32_t bars = base + TAIL;                           // full[s] +16s, empty[s] +16s+8
     const uint32_t bar_acc = bars + 16 * MAX_STAGES;
     const uint32_t bar_rx = bar_acc + 8;                         // split K: the other CTAs' tiles have landed here
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen + TAIL + 16 * MAX_STAGES + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ks = p.ksplit;                                     // CTAs (one cluster) that share an output tile
+    const int ks = SPLIT ? p.ksplit : 1;                         // CTAs (one cluster) that share an output tile
     const int zr = ks > 1 ? (int)(blockIdx.x % ks) : 0;          // = rank in the cluster: which slice of K
     const int n0 = (int)(blockIdx.x / ks) * NT, m0 = blockIdx.y * BM;
     constexpr int MMA_WARPS = mma_warps<NT>();
@@ -254,12 +259,20 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     }
 }
 
+template <int NT, bool IN_MAJOR, bool PAIR, bool SPLIT>
+cudaError_t run_as(photon_ctx *ctx, const ConvParams &p, const CUtensorMap &mx, const CUtensorMap &mw, dim3 grid,
+                   cudaStream_t st) {
+    using T = ConvTile<NT>;
+    constexpr size_t smem = (size_t)(PAIR ? RING_BYTES_PAIR : RING_BYTES) + T::extra;
+    static size_t smem_set[kMaxDevices] = {};
+    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR, PAIR, SPLIT>, smem, ctx->device, smem_set)) return e;
+    return launch_dependent(converter_umma_kernel<NT, IN_MAJOR, PAIR, SPLIT>, grid, dim3(CONV_THREADS), smem, st,
+                            p.ksplit > 1 ? p.ksplit : 0, p, mx, mw);
+}
+
 template <int NT, bool IN_MAJOR>
 cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches) {
     p.x_rows = p.B > 64 ? 128 : p.B > 32 ? 64 : p.B > 16 ? 32 : 16;
-    using T = ConvTile<NT>;
-    static size_t smem_set[kMaxDevices] = {};
-    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR>, T::SMEM, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
     CUtensorMap mx, mw;
     if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, p.x_rows))) return cudaErrorInvalidValue;
@@ -270,8 +283,16 @@ cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launc
     mw = *t;
     if (p.ksplit < 1) p.ksplit = 1;
     dim3 grid(p.ksplit * (p.N / NT), (p.B + BM - 1) / BM);
-    const cudaError_t e = launch_dependent(converter_umma_kernel<NT, IN_MAJOR>, grid, dim3(CONV_THREADS), T::SMEM, st,
-                                           p.ksplit > 1 ? p.ksplit : 0, p, mx, mw);
+    const long long ctas = (long long)grid.x * grid.y;
+    cudaError_t e;
+    if constexpr (NT == 64) {
+        const bool pair = p.ksplit == 1 && ctas > ctx->sm_count && ctas <= 2ll * ctx->sm_count;
+        e = pair ? run_as<NT, IN_MAJOR, true, false>(ctx, p, mx, mw, grid, st)
+                 : p.ksplit > 1 ? run_as<NT, IN_MAJOR, false, true>(ctx, p, mx, mw, grid, st)
+                                : run_as<NT, IN_MAJOR, false, false>(ctx, p, mx, mw, grid, st);
+    } else {
+        e = run_as<NT, IN_MAJOR, false, false>(ctx, p, mx, mw, grid, st);
+    }
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
