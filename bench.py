@@ -527,7 +527,37 @@ def run_gpu(args, cfg) -> None:
                 "us": us_e, "launches": 10, "algorithmic_bytes": ebytes, "GBps": ebytes / us_e * 1e-3,
                 "frac_hbm": ebytes / us_e * 1e-3 / hbm_peak, "TFLOPs": eflops / us_e * 1e-6,
                 "note": "weights and the sequences' own K/V rows counted once (no shared prefix), activations not counted"}
-            del layers, lw0
+
+            # the same layer of a local decoder for the newest in-chunk position of every in-flight chunk:
+            # chunk buffers of the replicas one row short of their recorded length (room for the append);
+            # the lengths are put back by a small copy before every call (inside the timed graph)
+            lcfg = wl.scaled(cfg, B=cfg.Nc)
+            dx = torch.empty(cfg.Nc, cfg.D, dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+            dy = torch.empty_like(dx)
+            dlen0 = (clen - 1).clamp(min=0)
+            dlen = dlen0.clone()
+            dkv = [ph.make_kv(t["kc"], t["vc"], dlen) for t in reps]
+            dscr = ph.make_layer_scratch(cfg.Nc, cfg.Hq, cfg.Hkv, cfg.dh, F, dev, torch.bfloat16)
+            turn["i"] = -1
+
+            def dec_call(t):
+                i = turn["i"] = turn["i"] + 1
+                dlen.copy_(dlen0)
+                ph.photon_decoder_step(ctx, layers[i % R], dscr, dx, dkv[i % R], dy, scale=scale)
+
+            us_d = graph_time_us(dec_call)
+            dbytes = wbytes + int(dlen0.sum().item() + cfg.Nc) * cfg.Hkv * cfg.dh * 4 + 2 * cfg.Nc * cfg.D * 2
+            dflops = 2.0 * cfg.Nc * (wbytes / 2)
+            t_roof = max(dbytes / (hbm_peak * 1e3), dflops / (tensor_peak * 1e6))
+            widened["decoder_step"] = {
+                "workload": "one layer, %d in-flight chunks (one new token each): D %d, F %d, windows of at most %d rows" % (
+                    cfg.Nc, cfg.D, F, cfg.P + cfg.C),
+                "us": us_d, "launches": 10, "algorithmic_bytes": dbytes, "GBps": dbytes / us_d * 1e-3,
+                "frac_hbm": dbytes / us_d * 1e-3 / hbm_peak, "TFLOPs": dflops / us_d * 1e-6,
+                "frac_of_own_roofline": t_roof / us_d,
+                "note": "weights, the chunks' K/V rows, x and y counted once; the figure includes one small copy that "
+                        "puts the lengths back before each call"}
+            del layers, lw0, dscr, dkv
             torch.cuda.empty_cache()
 
     # roofline of the dominant kernel = the attention part that takes the longest

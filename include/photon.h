@@ -191,7 +191,13 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
  * weights in the order w_layout names: wqkv [D, (Hq + 2 Hkv) dh], wo [Hq dh,
  * D], wgu [D, 2F], wdown [F, D]; g1, g2 [D].  F a multiple of 64.  The
  * caller owns the intermediates in `scratch` (sizes beside the fields); each
- * is rounded to bf16 where the next kernel reads it.  y may alias x. */
+ * is rounded to bf16 where the next kernel reads it.  y may alias x.
+ *
+ * photon_decoder_step: the same layer of a local decoder G^(l) (Eq. 6-7) for
+ * the newest in-chunk position of every in-flight chunk: `chunks` holds the
+ * chunk buffers (cap <= P + C; x, y [n_units, D]), the position is the
+ * buffer's length before the append (prefix rows count), and the attention
+ * is the bounded one of photon_chunk_attn. */
 typedef struct photon_layer {
   const photon_bf16 *g1, *wqkv, *wo, *g2, *wgu, *wdown;
   int32_t w_layout;          /* PHOTON_W_IN_MAJOR or PHOTON_W_OUT_MAJOR, all four weights */
@@ -216,6 +222,9 @@ photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 
                             photon_stream stream);
 photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
                                   const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
+                                  photon_stream stream);
+photon_status photon_decoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
+                                  const photon_bf16 *x, photon_kv *chunks, photon_bf16 *y, float scale,
                                   photon_stream stream);
 
 /* Bounded causal attention of the local decoders G^(l) (Eq. 6-7): query c

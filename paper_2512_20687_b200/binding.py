@@ -109,9 +109,10 @@ def load() -> ctypes.CDLL:
                                       c_void_p, c_void_p]
     lib.photon_swiglu.restype = st
     lib.photon_swiglu.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p]
-    lib.photon_encoder_step.restype = st
-    lib.photon_encoder_step.argtypes = [c_void_p, POINTER(photon_layer), POINTER(photon_layer_scratch), c_void_p,
-                                        POINTER(photon_kv), c_void_p, c_float, c_void_p]
+    for f in (lib.photon_encoder_step, lib.photon_decoder_step):
+        f.restype = st
+        f.argtypes = [c_void_p, POINTER(photon_layer), POINTER(photon_layer_scratch), c_void_p,
+                      POINTER(photon_kv), c_void_p, c_float, c_void_p]
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_device_status.restype = st
@@ -264,6 +265,12 @@ def make_layer_scratch(B, Hq, Hkv, dh, F, device, dtype) -> photon_layer_scratch
     for k, t in sc.tensors.items():
         setattr(sc, k, _ptr(t))
     return sc
+
+
+def photon_decoder_step(ctx, layer: photon_layer, scratch: photon_layer_scratch, x, chunks: photon_kv, y,
+                        scale=1.0, stream=None) -> None:
+    _check(load().photon_decoder_step(ctx, byref(layer), byref(scratch), _ptr(x), byref(chunks), _ptr(y),
+                                      c_float(scale), _stream(stream)), "photon_decoder_step")
 
 
 def photon_encoder_step(ctx, layer: photon_layer, scratch: photon_layer_scratch, x, cache: photon_kv, y,

@@ -305,9 +305,12 @@ photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 
-photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc,
-                                  const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
-                                  photon_stream stream) {
+namespace {
+// STEP of one layer for the newest position of every unit of `cache`; local: the cache is a set of chunk
+// buffers read by the chunk attention, else a coarse stream read by the coarse attention.
+photon_status layer_step(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc,
+                         const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale, bool local,
+                         photon_stream stream) {
     if (!ctx || !L || !sc || !cache || !x || !y) return PHOTON_ERR_INVALID_ARG;
     const photon_config &c = ctx->cfg;
     // everything is validated before the first launch, so that a bad argument leaves no partial step behind
@@ -320,18 +323,34 @@ photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *L, const 
     for (const void *q : ptrs)
         if (!q || !aligned16(q)) return PHOTON_ERR_INVALID_ARG;
     const int B = cache->n_units, D = c.D, QKV = (c.Hq + 2 * c.Hkv) * c.dh;
-    if ((size_t)B * c.Hkv > ctx->n_tickets) return PHOTON_ERR_WORKSPACE;
+    if (!local && (size_t)B * c.Hkv > ctx->n_tickets) return PHOTON_ERR_WORKSPACE;
+    if (local && cache->cap > c.P + c.C) return PHOTON_ERR_INVALID_ARG;
     photon_status s = photon_rmsnorm(ctx, x, L->g1, L->eps, sc->n, B, D, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wqkv, L->w_layout, nullptr, nullptr, sc->qkv, B, D, QKV, stream);
     if (s == PHOTON_OK) s = photon_rope_split(ctx, sc->qkv, cache->len, B, L->theta, sc->q, sc->k_new, sc->v_new, stream);
     if (s == PHOTON_OK) s = photon_kv_append(ctx, cache, sc->k_new, sc->v_new, nullptr, B, 1, stream);
-    if (s == PHOTON_OK) s = photon_coarse_attn(ctx, cache, sc->q, sc->att, nullptr, scale, stream);
+    if (s == PHOTON_OK)
+        s = local ? photon_chunk_attn(ctx, cache, sc->q, nullptr, sc->att, B, scale, stream)
+                  : photon_coarse_attn(ctx, cache, sc->q, sc->att, nullptr, scale, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->att, L->wo, L->w_layout, nullptr, x, sc->h, B, D, D, stream);
     if (s == PHOTON_OK) s = photon_rmsnorm(ctx, sc->h, L->g2, L->eps, sc->n, B, D, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, B, D, 2 * L->F, stream);
     if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, B, L->F, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->act, L->wdown, L->w_layout, nullptr, sc->h, y, B, L->F, D, stream);
     return s;
+}
+}  // namespace
+
+photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
+                                  const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
+                                  photon_stream stream) {
+    return layer_step(ctx, layer, scratch, x, cache, y, scale, false, stream);
+}
+
+photon_status photon_decoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
+                                  const photon_bf16 *x, photon_kv *chunks, photon_bf16 *y, float scale,
+                                  photon_stream stream) {
+    return layer_step(ctx, layer, scratch, x, chunks, y, scale, true, stream);
 }
 
 photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {

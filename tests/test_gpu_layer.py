@@ -146,6 +146,37 @@ def test_each_kernel_of_the_layer_on_the_oracles_own_intermediates(oracle, idx, 
     assert_close_scaled(host_f64(y), w["y"], "down projection")
 
 
+@pytest.mark.parametrize("idx,B,chunks_per_seq", [(4, 16, 32), (1, 40, 2)])
+def test_decoder_step_matches_oracle(oracle, idx, B, chunks_per_seq):
+    """The same layer for the newest in-chunk position of every in-flight chunk: ragged
+    chunk buffers (prefix rows + what has been written), positions = their lengths,
+    the bounded chunk attention in the middle."""
+    cfg = cfg_small(idx, B=B, chunks_per_seq=chunks_per_seq)
+    Nc, F = cfg.Nc, 1024
+    lcfg = wl.scaled(cfg, B=Nc)                                          # one token per chunk
+    lw = wl.encoder_layer_inputs(lcfg, F=F)
+    ch = wl.chunk_inputs(cfg, poison=True, strict_paper=True)            # len = P + n_in with room for one more row
+    assert ch["len"].max() < ch["cap"]
+    scale = cfg.dh ** -0.5
+    cache = {"k": ch["kc"].copy(), "v": ch["vc"].copy(), "len": ch["len"].copy()}
+    want = oracle.encoder_step(lw["x"], lw, cache, scale, n_threads=NT)
+    with Ctx(cfg) as c:
+        dk, dv, dl = dev_bf16(ch["kc"]), dev_bf16(ch["vc"]), dev_i32(ch["len"])
+        kv = ph.make_kv(dk, dv, dl)
+        W = {n: dev_bf16(lw[n]) for n in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")}
+        layer = ph.make_layer(W["g1"], W["wqkv"], W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, F)
+        sc = ph.make_layer_scratch(Nc, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        x = dev_bf16(lw["x"])
+        y = torch.empty_like(x)
+        ph.photon_decoder_step(c.h, layer, sc, x, kv, y, scale=scale)
+        assert c.status() == 0
+        assert np.array_equal(dl.cpu().numpy(), ch["len"] + 1)
+        for name in ("qkv", "q", "k_new", "att", "h", "act"):
+            got, ref = host_f64(sc.tensors[name]).reshape(Nc, -1), wl.bf16_bits_to_f64(want[name]).reshape(Nc, -1)
+            assert_close_scaled(got, ref, f"decoder step {name}", slack=2.0)
+    assert_close_scaled(host_f64(y), want["y"], f"decoder step cfg{idx}", slack=2.0)
+
+
 def test_encoder_step_refuses_bad_arguments():
     cfg = cfg_small(0, B=2, S=8)
     with Ctx(cfg) as c:
