@@ -47,6 +47,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parts", action="store_true")
     ap.add_argument("--max-splits", type=int, default=0)
+    ap.add_argument("--hierarchy", default="",
+                    help="chunk lengths C_1,...,C_L instead of 4,4 (e.g. 2,2): same model and context, other stream lengths")
     ap.add_argument("--batch", type=int, default=0,
                     help="shrink the workload to this many sequences (for profiler captures of a small case)")
     return ap.parse_args()
@@ -58,7 +60,7 @@ def workload_desc(cfg) -> dict:
                      f"{cfg.S} coarse latents, {cfg.Hq}q/{cfg.Hkv}kv heads x {cfg.dh}, d_model {cfg.D}, "
                      f"converter {cfg.D}->{cfg.P}x{cfg.D}, chunk attention P={cfg.P} C={cfg.C}, "
                      f"{cfg.chunks_per_seq} in-flight chunks per sequence",
-         "batch": cfg.B, "coarse_len": cfg.S, "context": cfg.context, "seed": cfg.seed,
+         "batch": cfg.B, "coarse_len": cfg.S, "context": cfg.context, "seed": cfg.seed, "tokens_per_coarse_latent": cfg.compress,
          "tokens_per_step": cfg.tokens_per_step}
     if cfg.shared_S:
         d["shared_prefix_len"] = cfg.shared_S
@@ -565,8 +567,8 @@ def run_gpu(args, cfg) -> None:
     def recorded_traffic(kernel_name):
         """DRAM bytes per launch from the committed ncu capture, or None once the kernel's source has changed."""
         note = "no ncu capture on record for this kernel and workload"
-        if args.batch:
-            return None, "reduced batch: the recorded traffic belongs to the full workload"
+        if args.batch or args.hierarchy:
+            return None, "reduced batch or another hierarchy: the recorded traffic belongs to the standard workload"
         try:
             rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.txt"))).get(
                 f"config{cfg.index}", {}).get(kernel_name)
@@ -688,6 +690,8 @@ def main():
     cfg = wl.CONFIGS[args.config]
     if args.batch and args.batch < cfg.B:
         cfg = wl.scaled(cfg, B=args.batch, tokens_per_step=cfg.tokens_per_step * args.batch // cfg.B)
+    if args.hierarchy:
+        cfg = wl.with_hierarchy(cfg, tuple(int(t) for t in args.hierarchy.split(",")))
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -159,6 +159,18 @@ def scaled(cfg: DecodeConfig, **kw) -> DecodeConfig:
     return dataclasses.replace(cfg, **kw)
 
 
+def with_hierarchy(cfg: DecodeConfig, chunk_lengths) -> DecodeConfig:
+    """The same model shapes and context under another hierarchy (C_1, ..., C_L): the
+    coarse stream holds context / prod(C_l) latents per sequence (a shared prefix
+    likewise) and the token-level chunks are C_1 long.  (4, 4) is the hierarchy of the
+    five configurations; the paper's ablation also runs (2, 2)."""
+    total = int(np.prod(chunk_lengths))
+    assert cfg.context % total == 0 and cfg.shared_context % total == 0
+    return dataclasses.replace(
+        cfg, name=f"{cfg.name}/{'x'.join(str(c) for c in chunk_lengths)}", compress=total,
+        S=cfg.context // total, shared_S=cfg.shared_context // total, C=int(chunk_lengths[0]))
+
+
 def coarse_inputs(cfg: DecodeConfig, replica: int = 0, poison: bool = False) -> dict:
     """Coarse-stream tensors for one decode step.
 

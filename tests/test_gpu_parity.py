@@ -387,6 +387,31 @@ def test_chunk_attention_at_the_largest_window(oracle, dh, Hq, Hkv):
     assert_close(got, want, f"chunk cap 64 dh={dh} G={Hq // Hkv}")
 
 
+@pytest.mark.parametrize("idx,lengths,B", [(1, (2, 2), 16), (1, (4, 4, 4), 64), (3, (2, 2), 64), (4, (2, 2), 8)])
+def test_decode_step_under_other_hierarchies(oracle, idx, lengths, B):
+    """The whole step on the shapes another hierarchy gives the same model: (2, 2) makes
+    the coarse stream four times longer and the token chunks two long; three levels
+    make it four times shorter."""
+    cfg = wl.with_hierarchy(cfg_small(idx, B=B), lengths)
+    s = wl.step_inputs(cfg, poison=True)
+    co, cv, ch = s["coarse"], s["converter"], s["chunks"]
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        d, dc = coarse_to_dev(co), chunks_to_dev(ch)
+        out = torch.empty_like(d["q"])
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        oc = torch.empty_like(dc["q"])
+        args = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out, scale, dev_bf16(cv["w_in_major"]),
+                                 ph.PHOTON_W_IN_MAJOR, U, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc,
+                                 Nc=cfg.Nc, scale_chunk=scale)
+        ph.photon_decode_step(c.h, args)
+        assert c.status() == 0
+    want = oracle.decode_step(co, cv, ch, scale, scale, chain=True, n_threads=NT)
+    assert_close(host_f64(out), want["out"], f"coarse {cfg.name}")
+    assert_close(host_f64(oc), want["chunk_out"], f"chunk {cfg.name}")
+    assert_close(host_f64(U), want["U"], f"U {cfg.name}")
+
+
 def test_calls_larger_than_the_context_was_made_for_are_refused():
     cfg = cfg_small(1, B=8, S=70)
     co = wl.coarse_inputs(cfg)

@@ -89,6 +89,36 @@ def test_generation_schedules_against_a_decode_loop():
     assert wl.global_kv_bytes_per_token(cfg, "recursive") * cfg.B == wl.coarse_kv_bytes(cfg) / cfg.compress
 
 
+def test_other_hierarchies():
+    """(2, 2), the paper's other ablation point, and three levels: the derived
+    configurations, and the closed forms against a decode loop that advances level l
+    once per C_{<=l} tokens."""
+    c22 = wl.with_hierarchy(wl.CONFIGS[1], (2, 2))
+    assert (c22.S, c22.compress, c22.C) == (2048, 4, 2) and wl.coarse_kv_bytes(c22) == 4 * wl.coarse_kv_bytes(wl.CONFIGS[1])
+    c444 = wl.with_hierarchy(wl.CONFIGS[2], (4, 4, 4))
+    assert (c444.S, c444.compress) == (2048, 64)
+    c3 = wl.with_hierarchy(wl.CONFIGS[3], (2, 2))
+    assert (c3.S, c3.shared_S) == (128, 8192)
+    for lengths in ((2, 2), (4, 4, 4), (2, 4, 8)):
+        T = 1024
+        upto = np.cumprod(lengths)
+        n = [0] * len(lengths)
+        hier = rec = 0
+        for t in range(1, T + 1):
+            for l, u in enumerate(upto):
+                if t % u == 0:
+                    n[l] += 1
+                    hier += n[l]
+                    if l == len(lengths) - 1:
+                        rec += n[l]
+        assert wl.cumulative_global_rows(T, "hierarchical", lengths) == hier
+        assert wl.cumulative_global_rows(T, "recursive", lengths) == rec
+        caches = wl.global_caches(c444 if len(lengths) == 3 and lengths == (4, 4, 4) else
+                                  wl.with_hierarchy(wl.CONFIGS[2], lengths), "hierarchical", lengths)
+        assert [c["tokens_per_read"] for c in caches] == list(upto)
+        assert [c["rows"] for c in caches] == [131072 // u for u in upto]
+
+
 def test_chunk_inputs_structure():
     cfg = wl.CONFIGS[0]
     ch = wl.chunk_inputs(cfg, poison=True)
