@@ -48,7 +48,6 @@ struct ConvTile {
     static constexpr int B_BYTES = NT * BK * 2;           // weight atom: 8 / 16 KiB
     // slack after the ring: the MMA reads 128 rows from every x atom, also past a short x box
     static constexpr int extra = BM * BK * 2 + 1024 + 512;
-    static constexpr int SMEM = RING_BYTES + extra;
 };
 
 __host__ __device__ inline int conv_stages(int ring_bytes, int a_bytes, int b_bytes, int ka) {
