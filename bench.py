@@ -460,6 +460,38 @@ def run_gpu(args, cfg) -> None:
         del qr, orows, full_kv
         torch.cuda.empty_cache()
 
+        # the coarse attention on a paged layout of the same cache: pages of 128 rows (64 when the stream is
+        # shorter), scattered over the pool by a fixed permutation; same bytes, one table look-up per tile
+        if cfg.S % 64 == 0 and not cfg.shared_S:
+            pr = 128 if cfg.S % 128 == 0 else 64
+            ppu = cfg.S // pr
+            perm = torch.randperm(cfg.B * ppu, generator=torch.Generator().manual_seed(99 + cfg.seed)).to(dev)
+            inv = torch.empty_like(perm)
+            inv[perm] = torch.arange(cfg.B * ppu, device=dev)
+
+            def paged(t):
+                pool = t.view(cfg.B, cfg.Hkv, ppu, pr, cfg.dh).permute(0, 2, 1, 3, 4).reshape(cfg.B * ppu, cfg.Hkv, pr, cfg.dh)
+                return pool[perm].contiguous()                 # pool[i] = page perm[i]; page j sits at inv[j]
+
+            table = inv.view(cfg.B, ppu).to(torch.int32).contiguous()
+            pkv = [ph.make_kv(paged(t["k"]), paged(t["v"]), lens[r], max_len=cfg.S, page_table=table)
+                   for r, t in enumerate(reps)]
+            turn["i"] = -1
+
+            def paged_call(t):
+                i = turn["i"] = turn["i"] + 1
+                ph.photon_coarse_attn(ctx, pkv[i % R], q, reps[i % R]["out"], None, scale)
+
+            us_p = graph_time_us(paged_call)
+            widened["paged_coarse_attn"] = {
+                "workload": "the coarse attention of the step on pages of %d rows scattered over a pool" % pr,
+                "us": us_p, "algorithmic_bytes": kernels["coarse_attn"]["bytes"],
+                "GBps": kernels["coarse_attn"]["bytes"] / us_p * 1e-3,
+                "frac_hbm": kernels["coarse_attn"]["bytes"] / us_p * 1e-3 / hbm_peak, "TFLOPs": 0.0,
+                "us_contiguous": kernels["coarse_attn"]["us"]}
+            del pkv
+            torch.cuda.empty_cache()
+
         # the top-level context chunker (step (ii) of a recursive-generation step): normalise the 4 concatenated
         # lower-level latents per sequence, project [B, 4D] -> [B, D]; weights rotate like the converter's
         ci = wl.chunker_inputs(cfg)

@@ -85,7 +85,16 @@ typedef struct {
  * if the prefix had been copied in front of its cache; the prefix is stored
  * and read once.  k_shared = NULL disables this.
  *   k_shared, v_shared [n_shared, Hkv, cap_shared, dh]; shared_len [n_shared];
- *   shared_id [n_units], -1 = none; max_shared_len like max_len. */
+ *   shared_id [n_units], -1 = none; max_shared_len like max_len.
+ * Optional paging (a serving layout; the paper has no counterpart): with
+ * page_table != NULL, k and v are pools [n_pages, Hkv, page_rows, dh] and row r
+ * of unit u lives in page page_table[u * pages_per_unit + r / page_rows] at row
+ * r % page_rows; cap must equal pages_per_unit * page_rows and page_rows must
+ * be a multiple of 64.  Pages of different units must be distinct.  A page id
+ * outside [0, n_pages) sets PHOTON_DEV_BAD_INDEX (page 0 is read instead; an
+ * append is dropped).  Accepted by photon_kv_append, photon_coarse_attn,
+ * photon_flat_attn and what is built on them; the chunk-local calls and the
+ * no-allocation call take contiguous caches only (INVALID_ARG). */
 typedef struct {
   photon_bf16 *k, *v;
   int32_t *len;
@@ -93,6 +102,8 @@ typedef struct {
   const photon_bf16 *k_shared, *v_shared;
   const int32_t *shared_len, *shared_id;
   int32_t n_shared, cap_shared, max_shared_len;
+  const int32_t *page_table;             /* [n_units, pages_per_unit] device int32, or NULL */
+  int32_t page_rows, pages_per_unit, n_pages;
 } photon_kv;
 
 /* Creates a context on the current CUDA device: validates cfg, allocates the

@@ -36,6 +36,7 @@ class photon_kv(Structure):
         ("k_shared", c_void_p), ("v_shared", c_void_p),
         ("shared_len", c_void_p), ("shared_id", c_void_p),
         ("n_shared", c_int32), ("cap_shared", c_int32), ("max_shared_len", c_int32),
+        ("page_table", c_void_p), ("page_rows", c_int32), ("pages_per_unit", c_int32), ("n_pages", c_int32),
     ]
 
 
@@ -159,12 +160,19 @@ def photon_status_str(code: int) -> str:
 
 
 def make_kv(k, v, length, max_len: int = 0, k_shared=None, v_shared=None, shared_len=None,
-            shared_id=None, max_shared_len: int = 0) -> photon_kv:
+            shared_id=None, max_shared_len: int = 0, page_table=None) -> photon_kv:
     """Fills a photon_kv from tensors k, v [n_units, Hkv, cap, dh], length [n_units]
-    (and the optional shared-prefix tensors).  The struct keeps the tensors alive."""
+    (and the optional shared-prefix tensors).  With page_table [n_units, pages_per_unit]
+    k and v are pools [n_pages, Hkv, page_rows, dh].  The struct keeps the tensors alive."""
     kv = photon_kv()
     kv.k, kv.v, kv.len = _ptr(k), _ptr(v), _ptr(length)
     kv.n_units, kv.cap, kv.max_len = k.shape[0], k.shape[2], max_len
+    if page_table is not None:
+        kv.page_table = _ptr(page_table)
+        kv.n_pages, kv.page_rows = k.shape[0], k.shape[2]
+        kv.n_units, kv.pages_per_unit = page_table.shape
+        kv.cap = kv.page_rows * kv.pages_per_unit
+    kv._pages = page_table
     if k_shared is not None:
         kv.k_shared, kv.v_shared = _ptr(k_shared), _ptr(v_shared)
         kv.shared_len, kv.shared_id = _ptr(shared_len), _ptr(shared_id)

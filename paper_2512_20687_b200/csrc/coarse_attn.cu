@@ -508,6 +508,15 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             for (; it < n_tiles; ++it, w.next(p)) {
                 const int s = it % STAGES;
                 if (*dead) break;
+                // row of the tile's first key in the cache tensor; for a paged cache through the page table
+                // (looked up before the wait for a free stage, which hides the load's latency)
+                int y = (w.u * p.Hkv + w.h) * p.cap + w.j * BN;
+                if (p.page_table) {
+                    const int row = w.j * BN;
+                    int id = __ldg(p.page_table + (size_t)w.u * p.pages_per_unit + row / p.page_rows);
+                    if (id < 0 || id >= p.n_pages) { atomicOr(p.status, PHOTON_DEV_BAD_INDEX); id = 0; }
+                    y = (id * p.Hkv + w.h) * p.page_rows + row % p.page_rows;
+                }
                 if (!ptx::mbar_wait(bars + 16 * s + 8, ((it / STAGES) & 1) ^ 1)) {
                     *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
                 }
@@ -517,7 +526,6 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 const int nbox = (rows + BOX - 1) / BOX;
                 const bool first = (it == 0 || w.j == 0);
                 ptx::mbar_arrive_expect_tx(full, nbox * R::HALVES * BOX_BYTES * 2 + (first ? G * DH * 2 : 0));
-                const int y = (w.u * p.Hkv + w.h) * p.cap + w.j * BN;
                 for (int b = 0; b < nbox; ++b)
 #pragma unroll
                     for (int hh = 0; hh < R::HALVES; ++hh) {
@@ -637,9 +645,10 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     if (const cudaError_t e = ensure_dynamic_smem(coarse_attn_kernel<DH, GP>, smem, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
     CUtensorMap mk, mv;
-    if (!(t = ctx->tmaps.get(p.k, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BOX))) return cudaErrorInvalidValue;
+    const uint64_t pool_rows = p.page_table ? (uint64_t)p.n_pages * p.Hkv * p.page_rows : (uint64_t)p.n_units * p.Hkv * p.cap;
+    if (!(t = ctx->tmaps.get(p.k, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
     mk = *t;
-    if (!(t = ctx->tmaps.get(p.v, (uint64_t)p.n_units * p.Hkv * p.cap, DH, BOX))) return cudaErrorInvalidValue;
+    if (!(t = ctx->tmaps.get(p.v, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
     mv = *t;
     const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
     const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, ctx->max_ctas));

@@ -55,6 +55,7 @@ extern "C" photon_status photon_coarse_attn_noalloc(const photon_config *cfg, co
     if (c.dh != 64 && c.dh != 128) return PHOTON_ERR_UNSUPPORTED;
     if (c.Hq / c.Hkv > 16) return PHOTON_ERR_UNSUPPORTED;
     if (cache->k_shared) return PHOTON_ERR_UNSUPPORTED;           // shared prefixes need the context's workspace
+    if (cache->page_table) return PHOTON_ERR_INVALID_ARG;         // contiguous caches only
     if (cache->n_units < 0 || cache->cap <= 0 || cache->max_len < 0 || cache->max_len > cache->cap)
         return PHOTON_ERR_INVALID_ARG;
     if ((long long)cache->n_units * c.Hkv > kMaxStreams) return PHOTON_ERR_WORKSPACE;   // beyond the static array

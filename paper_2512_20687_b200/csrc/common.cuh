@@ -61,6 +61,8 @@ struct AttnParams {
     const int32_t *sh_len, *sh_id;
     int n_shared, cap_sh;
     const int32_t *slot;
+    const int32_t *page_table;   // paged cache: [n_units, pages_per_unit] page ids, or NULL
+    int page_rows, pages_per_unit, n_pages;
     int n_q, Hq, Hkv, dh;
     int splits_sh;           // key ranges of a shared prefix = cluster size of its kernel (0: no shared prefix)
     int upc;                 // filled by the launcher: units per CTA on shared keys
@@ -140,9 +142,13 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 
 // launchers: enqueue on `st`, add the number of kernels launched to *launches,
 // return the launch error (cudaSuccess when fine)
+struct Paging {              // of a paged cache; table == nullptr: contiguous
+    const int32_t *table;
+    int page_rows, pages_per_unit, n_pages;
+};
 cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,
                              const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
-                             int n_rows, int32_t *status, cudaStream_t st, long long *launches);
+                             int n_rows, Paging pg, int32_t *status, cudaStream_t st, long long *launches);
 cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                              long long *launches);
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,

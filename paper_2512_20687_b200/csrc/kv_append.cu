@@ -10,7 +10,7 @@ __global__ void __launch_bounds__(128)
 kv_append_kernel(uint4 *__restrict__ k, uint4 *__restrict__ v, int32_t *__restrict__ len, int n_units,
                  int Hkv, int cap, int vec_per_row, const uint4 *__restrict__ k_new,
                  const uint4 *__restrict__ v_new, const int32_t *__restrict__ unit_ids, int n_rows,
-                 int32_t *__restrict__ status) {
+                 const Paging pg, int32_t *__restrict__ status) {
     const int i = blockIdx.x;
     ptx::grid_dep_wait();
     const int u = unit_ids ? unit_ids[i] : i;
@@ -24,12 +24,29 @@ kv_append_kernel(uint4 *__restrict__ k, uint4 *__restrict__ v, int32_t *__restri
         return;
     }
     const int per_item = n_rows * Hkv * vec_per_row;
+    if (pg.table) {
+        // a paged cache: every page the new rows fall into must exist before anything is written
+        for (int r = at / pg.page_rows; r <= (at + n_rows - 1) / pg.page_rows; ++r) {
+            const int id = pg.table[(size_t)u * pg.pages_per_unit + r];
+            if (id < 0 || id >= pg.n_pages) {
+                if (threadIdx.x == 0) atomicOr(status, PHOTON_DEV_BAD_INDEX);
+                return;
+            }
+        }
+    }
     for (int t = threadIdx.x; t < per_item; t += blockDim.x) {
         const int d = t % vec_per_row;
         const int h = (t / vec_per_row) % Hkv;
         const int r = t / (vec_per_row * Hkv);
         const size_t src = (size_t)i * per_item + t;      // [n, n_rows, Hkv, dh]
-        const size_t dst = (((size_t)u * Hkv + h) * cap + (at + r)) * vec_per_row + d;
+        size_t dst;
+        if (pg.table) {
+            const int row = at + r;
+            const int id = pg.table[(size_t)u * pg.pages_per_unit + row / pg.page_rows];
+            dst = (((size_t)id * Hkv + h) * pg.page_rows + row % pg.page_rows) * vec_per_row + d;
+        } else {
+            dst = (((size_t)u * Hkv + h) * cap + (at + r)) * vec_per_row + d;
+        }
         k[dst] = k_new[src];
         v[dst] = v_new[src];
     }
@@ -39,11 +56,11 @@ kv_append_kernel(uint4 *__restrict__ k, uint4 *__restrict__ v, int32_t *__restri
 
 cudaError_t launch_kv_append(bf16 *k, bf16 *v, int32_t *len, int n_units, int Hkv, int cap, int dh,
                              const bf16 *k_new, const bf16 *v_new, const int32_t *unit_ids, int n,
-                             int n_rows, int32_t *status, cudaStream_t st, long long *launches) {
+                             int n_rows, Paging pg, int32_t *status, cudaStream_t st, long long *launches) {
     if (n == 0) return cudaSuccess;
     const cudaError_t e = launch_dependent(kv_append_kernel, dim3(n), dim3(128), 0, st, 0, (uint4 *)k, (uint4 *)v, len, n_units, Hkv, cap, dh / 8,
                                         (const uint4 *)k_new, (const uint4 *)v_new, unit_ids, n_rows,
-                                        status);
+                                        pg, status);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }

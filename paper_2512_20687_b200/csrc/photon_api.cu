@@ -23,6 +23,10 @@ bool kv_ok(const photon_ctx *ctx, const photon_kv *c, bool allow_shared) {
             c->max_shared_len > c->cap_shared)
             return false;
     }
+    if (c->page_table) {
+        if (c->page_rows <= 0 || c->page_rows % 64 != 0 || c->pages_per_unit <= 0 || c->n_pages <= 0) return false;
+        if ((int64_t)c->page_rows * c->pages_per_unit != c->cap) return false;
+    }
     (void)ctx;
     return true;
 }
@@ -34,14 +38,16 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
                                const int32_t *slot, int n_q, photon_bf16 *out, float *lse,
                                float scale, bool chunk, cudaStream_t st) {
     if (!ctx) return PHOTON_ERR_INVALID_ARG;
-    if (!kv_ok(ctx, cache, !chunk)) return PHOTON_ERR_INVALID_ARG;
+    if (!kv_ok(ctx, cache, !chunk) || (chunk && cache->page_table)) return PHOTON_ERR_INVALID_ARG;
     if (n_q < 0 || (n_q > 0 && (!q || !out))) return PHOTON_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(out)) return PHOTON_ERR_INVALID_ARG;
     if (!(scale == scale)) return PHOTON_ERR_INVALID_ARG;
     if (n_q == 0) return PHOTON_OK;
     const photon_config &c = ctx->cfg;
     // TMA row coordinates are 32-bit
-    if ((uint64_t)cache->n_units * c.Hkv * cache->cap >= (1ull << 31)) return PHOTON_ERR_UNSUPPORTED;
+    const uint64_t pool_rows = cache->page_table ? (uint64_t)cache->n_pages * c.Hkv * cache->page_rows
+                                                 : (uint64_t)cache->n_units * c.Hkv * cache->cap;
+    if (pool_rows >= (1ull << 31)) return PHOTON_ERR_UNSUPPORTED;
     if (cache->k_shared && (uint64_t)cache->n_shared * c.Hkv * cache->cap_shared >= (1ull << 31))
         return PHOTON_ERR_UNSUPPORTED;
     AttnParams p{};
@@ -54,6 +60,8 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
     p.n_units = cache->n_units;
     p.cap = cache->cap;
     p.slot = slot;
+    p.page_table = cache->page_table;
+    p.page_rows = cache->page_rows; p.pages_per_unit = cache->pages_per_unit; p.n_pages = cache->n_pages;
     p.n_q = n_q;
     p.Hq = c.Hq; p.Hkv = c.Hkv; p.dh = c.dh;
     p.scale_log2 = scale * 1.4426950408889634f;
@@ -172,7 +180,8 @@ photon_status photon_kv_append(photon_ctx *ctx, photon_kv *cache, const photon_b
     const cudaError_t e = launch_kv_append(
         reinterpret_cast<bf16 *>(cache->k), reinterpret_cast<bf16 *>(cache->v), cache->len,
         cache->n_units, c.Hkv, cache->cap, c.dh, reinterpret_cast<const bf16 *>(k_new),
-        reinterpret_cast<const bf16 *>(v_new), unit_ids, n, n_rows, ctx->status,
+        reinterpret_cast<const bf16 *>(v_new), unit_ids, n, n_rows,
+        Paging{cache->page_table, cache->page_rows, cache->pages_per_unit, cache->n_pages}, ctx->status,
         static_cast<cudaStream_t>(stream), &ctx->launches);
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
@@ -205,7 +214,7 @@ photon_status photon_chunk_causal_attn(photon_ctx *ctx, const photon_kv *chunks,
                                        const int32_t *slot, photon_bf16 *out, int32_t Nc, int32_t row0,
                                        int32_t rows, float scale, photon_stream stream) {
     if (!ctx || !chunks) return PHOTON_ERR_INVALID_ARG;
-    if (!kv_ok(ctx, chunks, false)) return PHOTON_ERR_INVALID_ARG;
+    if (!kv_ok(ctx, chunks, false) || chunks->page_table) return PHOTON_ERR_INVALID_ARG;
     if (chunks->cap > ctx->cfg.P + ctx->cfg.C || chunks->cap > 64) return PHOTON_ERR_INVALID_ARG;
     if (Nc < 0 || row0 < 0 || rows < 1 || row0 + rows > chunks->cap) return PHOTON_ERR_INVALID_ARG;
     if (!slot && Nc > chunks->n_units) return PHOTON_ERR_INVALID_ARG;
@@ -324,7 +333,7 @@ photon_status layer_step(photon_ctx *ctx, const photon_layer *L, const photon_la
         if (!q || !aligned16(q)) return PHOTON_ERR_INVALID_ARG;
     const int B = cache->n_units, D = c.D, QKV = (c.Hq + 2 * c.Hkv) * c.dh;
     if (!local && (size_t)B * c.Hkv > ctx->n_tickets) return PHOTON_ERR_WORKSPACE;
-    if (local && cache->cap > c.P + c.C) return PHOTON_ERR_INVALID_ARG;
+    if (local && (cache->cap > c.P + c.C || cache->page_table)) return PHOTON_ERR_INVALID_ARG;
     photon_status s = photon_rmsnorm(ctx, x, L->g1, L->eps, sc->n, B, D, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wqkv, L->w_layout, nullptr, nullptr, sc->qkv, B, D, QKV, stream);
     if (s == PHOTON_OK) s = photon_rope_split(ctx, sc->qkv, cache->len, B, L->theta, sc->q, sc->k_new, sc->v_new, stream);

@@ -47,7 +47,7 @@ def test_binding_has_the_same_names():
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(ph.photon_config) == 8 * 4
     # pointers are 8-byte aligned: 3 ptr + 3 int32 (+pad) + 4 ptr + 3 int32 (+pad)
-    assert ctypes.sizeof(ph.photon_kv) == 24 + 16 + 32 + 16
+    assert ctypes.sizeof(ph.photon_kv) == 24 + 16 + 32 + 16 + 8 + 16 and ph.photon_kv.page_table.offset == 88
     assert ph.photon_kv.max_len.offset == 32 and ph.photon_kv.k_shared.offset == 40
     assert ph.photon_step_args.scale_coarse.offset == 48 and ph.photon_step_args.x.offset == 56
     assert ctypes.sizeof(ph.photon_layer) == 6 * 8 + 4 * 4 and ph.photon_layer.F.offset == 52
