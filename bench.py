@@ -104,9 +104,16 @@ def cpu_baseline(cfg, seconds: float = 10.0) -> dict:
         times.append(time_oracle_step(cfg, sub, s, threads))
     dt = sum(times) / len(times)
     tokens = cfg.tokens_per_step * sub.B / cfg.B
+    # the same program on one core, on a sample sized for about 2 s per step
+    sub1, s1 = oracle_sample(cfg, 2.0, 1)
+    time_oracle_step(cfg, sub1, s1, 1)
+    dt1 = time_oracle_step(cfg, sub1, s1, 1)
     return {"value": tokens / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"{len(times)} decode steps of the first {sub.B} of {cfg.B} sequences "
-                      f"({sub.Nc} chunks), {dt:.3f} s each, {sum(times) * threads:.0f} core-seconds"}
+                      f"({sub.Nc} chunks), {dt:.3f} s each, {sum(times) * threads:.0f} core-seconds",
+            "single_thread": {"value": cfg.tokens_per_step * sub1.B / cfg.B / dt1, "unit": UNIT,
+                              "sample": f"one decode step of the first {sub1.B} of {cfg.B} sequences, {dt1:.3f} s"},
+            "hardware_threads": threads}
 
 
 def run_reference(args, cfg) -> None:
@@ -622,7 +629,33 @@ def run_gpu(args, cfg) -> None:
     roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
                 "frac": ach / hbm_peak, "traffic": traffic, "traffic_note": traffic_note,
                 "algorithmic_bytes": kernels[dom]["bytes"], "us_per_launch": kernels[dom]["us"],
-                "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0}
+                "peak_source": peak_src, "frac_of_nominal_8TBs": ach / 8000.0,
+                # the replicas are meant to keep the reads in HBM: less DRAM traffic than 95 % of the
+                # algorithmic bytes would mean the L2 served part of them
+                "l2_assisted": None if traffic is None else bool(traffic < 0.95 * kernels[dom]["bytes"])}
+    if cfg.shared_S and "coarse_attn" in parts:
+        # a shared prefix makes the coarse attention a contraction over the prefix plus a stream over the own
+        # rows: its own roofline is the slower of the two, and the bytes a cache without sharing would read
+        # are reported as logical, not physical, throughput
+        pc = parts["coarse_attn"]
+        prefix_flops = 4.0 * cfg.B * cfg.Hq * cfg.shared_S * cfg.dh
+        logical = (cfg.B * (cfg.S + cfg.shared_S)) * cfg.Hkv * cfg.dh * 4
+        t_roof = max(pc["algorithmic_bytes"] / (hbm_peak * 1e3), prefix_flops / (tensor_peak * 1e6))
+        pc.update({"prefix_flops": prefix_flops, "TFLOPs": prefix_flops / pc["us"] * 1e-6,
+                   "frac_of_own_roofline": t_roof / pc["us"], "logical_kv_bytes": logical,
+                   "logical_GBps": logical / pc["us"] * 1e-3,
+                   "logical_note": "bytes a cache with the prefix copied into every branch would read; not physical traffic"})
+    # derived from the per-part times: a meta-context of C_{<=L} tokens per sequence needs the append and the
+    # coarse attention once, the converter once per level-2 latent plus once for the level above (1 + C_2
+    # times), and the chunk attention once per token
+    amortised = None
+    if all(n in parts for n in ("kv_append", "coarse_attn", "converter", "chunk_attn")):
+        c2 = 4 if cfg.compress == 16 else max(1, int(round(cfg.compress ** 0.5)))
+        t_meta = (parts["kv_append"]["us"] + parts["coarse_attn"]["us"] + (1 + c2) * parts["converter"]["us"]
+                  + cfg.compress * parts["chunk_attn"]["us"])
+        amortised = {"tokens_per_s": cfg.tokens_per_step * cfg.compress / t_meta * 1e6, "us_per_meta_context": t_meta,
+                     "note": "derived from the parts: append + coarse attention once, converter %d times, chunk attention "
+                             "%d times per meta-context of %d tokens per sequence" % (1 + c2, cfg.compress, cfg.compress)}
     step_bytes = sum(kernels[n]["bytes"] for n in kernels)
 
     # end to end through the public API with host buffers: every step its inputs (new K/V row, both
@@ -698,6 +731,7 @@ def run_gpu(args, cfg) -> None:
         "step_hbm": {"algorithmic_bytes": step_bytes, "GBps": step_bytes / (sec_max / K) * 1e-9,
                      "frac": step_bytes / (sec_max / K) * 1e-9 / hbm_peak},
         "parts": parts,
+        "amortised": amortised,
         "widened": widened,
         "kv_bytes_per_token": {
             "photon_coarse_per_step": coarse_bytes,
