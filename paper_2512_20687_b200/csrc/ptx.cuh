@@ -55,7 +55,7 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// ---- TMA (tiled tensor loads, no multicast) ---------------------------------
+// ---- TMA (tiled tensor loads, each into the issuing CTA only) ----------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
@@ -144,7 +144,7 @@ __device__ __forceinline__ uint32_t map_cluster(uint32_t addr, uint32_t rank) {
     return remote;
 }
 // Bulk copy from this CTA's shared memory into a peer CTA's (addresses from map_cluster); the bytes are
-// counted on the peer's mbarrier.  16-byte aligned addresses, size a multiple of 16.  No multicast.
+// counted on the peer's mbarrier.  16-byte aligned addresses, size a multiple of 16.  One destination CTA per copy.
 __device__ __forceinline__ void bulk_copy_to_peer(uint32_t remote_dst, uint32_t local_src, uint32_t bytes, uint32_t remote_bar) {
     asm volatile(
         "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
