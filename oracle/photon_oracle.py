@@ -261,6 +261,37 @@ def encoder_step(x, lw, cache, scale, eps=1e-5, theta=10000.0, n_threads=1):
             "gu": gu, "act": act, "y": y, "flags": flags}
 
 
+def decoder_prefill(U, lw, chunks, scale, unit_ids=None, eps=1e-5, theta=10000.0, n_threads=1):
+    """The pass of one local-decoder layer over a fresh converter prefix (the first R_l
+    positions of the sequence [U ; X_<j] of Eq. 6, before any in-chunk position exists):
+    U [n, P, D] -> normalise -> fused q/k/v projection -> rotary encoding at positions
+    0..P-1 -> the P key/value rows become rows 0..P-1 of the chunk buffers unit_ids[i]
+    (which must be empty) -> causal attention among the P rows -> output projection +
+    residual -> MLP + residual.  Intermediates are rounded to bf16 as in encoder_step.
+    chunks: dict k, v [n_units, Hkv, cap, dh], len [n_units] (grown in place).
+    Returns dict with y (float64 [n, P, D]) and the bf16 intermediates."""
+    n, P, D = U.shape
+    Hkv, dh = chunks["k"].shape[1], chunks["k"].shape[3]
+    Hq = lw["wo"].shape[0] // dh
+    x = np.ascontiguousarray(U).reshape(n * P, D)
+    pos = np.tile(np.arange(P, dtype=np.int32), n)
+    n1 = round_bf16(rmsnorm(x, lw["g1"], eps))
+    qkv = round_bf16(linear(n1, lw["wqkv"], n_threads=n_threads))
+    q, k_new, v_new = (round_bf16(t) for t in rope_split(qkv, pos, Hq, Hkv, dh, theta))
+    flags = kv_append(chunks["k"], chunks["v"], chunks["len"], k_new.reshape(n, P, Hkv, dh),
+                      v_new.reshape(n, P, Hkv, dh), unit_ids=unit_ids, n_rows=P)
+    att = chunk_causal_attention(q.reshape(n, P, Hq, dh), chunks["k"], chunks["v"], chunks["len"], scale,
+                                 slot=unit_ids, n_threads=n_threads)
+    att = round_bf16(att).reshape(n * P, Hq * dh)
+    h = round_bf16(linear(att, lw["wo"], n_threads=n_threads) + widen_bf16(x))
+    n2 = round_bf16(rmsnorm(h, lw["g2"], eps))
+    gu = round_bf16(linear(n2, lw["wgu"], n_threads=n_threads))
+    act = round_bf16(swiglu(gu))
+    y = linear(act, lw["wdown"], n_threads=n_threads) + widen_bf16(h)
+    return {"qkv": qkv, "q": q, "k_new": k_new, "v_new": v_new, "att": att, "h": h, "act": act,
+            "y": y.reshape(n, P, D), "flags": flags}
+
+
 def round_bf16(x):
     """float64 -> bf16 bits, round to nearest even."""
     x = np.ascontiguousarray(x, dtype=np.float64)

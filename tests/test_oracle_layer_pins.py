@@ -78,6 +78,38 @@ def test_swiglu_against_torch(oracle):
     np.testing.assert_allclose(oracle.swiglu(bf(big))[0], [120.0, -120.0 * math.exp(-40.0)], rtol=1e-12)
 
 
+def test_decoder_prefill_against_torch_causal_attention(oracle):
+    """The prefix pass: the P rows of every chunk attend causally among themselves at
+    positions 0..P-1; torch's is_causal attention on the oracle's rotated q, k and v,
+    and the chunk buffers afterwards."""
+    cfg = wl.scaled(wl.CONFIGS[0], B=3, D=256, chunks_per_seq=2)              # P = 4, cap = 8
+    lw = wl.encoder_layer_inputs(wl.scaled(cfg, B=cfg.Nc * cfg.P), F=128)
+    n, P, D, Hq, Hkv, dh = cfg.Nc, cfg.P, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh
+    U = lw["x"].reshape(n, P, D)
+    cap = cfg.P + cfg.C
+    chunks = {"k": np.full((n + 2, Hkv, cap, dh), 0x7FC1, np.uint16), "v": np.full((n + 2, Hkv, cap, dh), 0x7FC1, np.uint16),
+              "len": np.zeros(n + 2, np.int32)}
+    ids = np.array([5, 0, 7, 2, 3, 1], np.int32)
+    scale = dh ** -0.5
+    r = oracle.decoder_prefill(U, lw, chunks, scale, unit_ids=ids)
+    assert r["flags"] == 0
+    assert list(chunks["len"]) == [P, P, P, P, 0, P, 0, P]
+    T = lambda b: torch.from_numpy(f64(b))
+    for i, u in enumerate(ids):
+        assert np.array_equal(chunks["k"][u, :, :P], r["k_new"].reshape(n, P, Hkv, dh)[i].transpose(1, 0, 2))
+        assert np.all(chunks["k"][u, :, P:] == 0x7FC1)
+    q = T(r["q"]).reshape(n, P, Hq, dh).permute(0, 2, 1, 3)
+    k = T(r["k_new"]).reshape(n, P, Hkv, dh).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, dim=1)
+    v = T(r["v_new"]).reshape(n, P, Hkv, dh).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, dim=1)
+    att = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, scale=scale)
+    np.testing.assert_allclose(f64(r["att"]).reshape(n, P, Hq, dh), att.permute(0, 2, 1, 3).numpy(), rtol=2 ** -8, atol=1e-6)
+    # positions: row r of every chunk is rotated by r; row 0 is not rotated at all
+    X = T(r["qkv"]).reshape(n, P, -1)
+    assert np.array_equal(f64(r["q"]).reshape(n, P, Hq * dh)[:, 0], X[:, 0, : Hq * dh].numpy())
+    y = T(r["act"]) @ T(lw["wdown"]) + T(r["h"])
+    np.testing.assert_allclose(r["y"].reshape(n * P, D), y.numpy(), rtol=1e-11, atol=1e-12)
+
+
 def test_encoder_step_against_a_torch_llama_layer(oracle):
     """One layer, written with torch's own rms_norm / linear / silu / softmax in fp64
     on the oracle's bf16 intermediates where the chain is rounded, otherwise
