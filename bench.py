@@ -598,7 +598,32 @@ def run_gpu(args, cfg) -> None:
                 "frac_of_own_roofline": t_roof / us_d,
                 "note": "weights, the chunks' K/V rows, x and y counted once; the figure includes one small copy that "
                         "puts the lengths back before each call"}
-            del layers, lw0, dscr, dkv
+            # and over fresh converter prefixes: the P prefix vectors of (up to 4096) chunks go through the layer, are
+            # installed as rows 0..P-1 of emptied chunk buffers and attend causally among themselves
+            n_pre = min(cfg.Nc, 4096)
+            pU = torch.empty(n_pre, cfg.P, cfg.D, dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+            pY = torch.empty_like(pU)
+            plen = torch.zeros(cfg.Nc, dtype=torch.int32, device=dev)
+            pkv2 = [ph.make_kv(t["kc"].clone(), t["vc"].clone(), plen) for t in reps[:2]]
+            pscr = ph.make_layer_scratch(n_pre * cfg.P, cfg.Hq, cfg.Hkv, cfg.dh, F, dev, torch.bfloat16)
+            turn["i"] = -1
+
+            def prefill_call(t):
+                i = turn["i"] = turn["i"] + 1
+                plen.zero_()
+                ph.photon_decoder_prefill(ctx, layers[i % R], pscr, pU, pkv2[i % 2], None, pY, n=n_pre, scale=scale)
+
+            us_pf = graph_time_us(prefill_call)
+            pflops = 2.0 * n_pre * cfg.P * (wbytes / 2)
+            pbytes = wbytes + 2 * n_pre * cfg.P * cfg.D * 2 + 2 * n_pre * cfg.P * cfg.Hkv * cfg.dh * 2
+            t_roof = max(pbytes / (hbm_peak * 1e3), pflops / (tensor_peak * 1e6))
+            widened["decoder_prefill"] = {
+                "workload": "one layer over the %d prefix vectors of each of %d chunks" % (cfg.P, n_pre),
+                "us": us_pf, "launches": 10, "algorithmic_bytes": pbytes, "GBps": pbytes / us_pf * 1e-3,
+                "frac_hbm": pbytes / us_pf * 1e-3 / hbm_peak, "TFLOPs": pflops / us_pf * 1e-6,
+                "frac_of_own_roofline": t_roof / us_pf,
+                "note": "weights, U, y and the installed K/V rows counted once; includes the small kernel that empties the lengths"}
+            del layers, lw0, dscr, dkv, pscr, pkv2
             torch.cuda.empty_cache()
 
     # roofline of the dominant kernel = the attention part that takes the longest

@@ -208,7 +208,17 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
  * the newest in-chunk position of every in-flight chunk: `chunks` holds the
  * chunk buffers (cap <= P + C; x, y [n_units, D]), the position is the
  * buffer's length before the append (prefix rows count), and the attention
- * is the bounded one of photon_chunk_attn. */
+ * is the bounded one of photon_chunk_attn.
+ *
+ * photon_decoder_prefill: the same layer over a fresh converter prefix, the
+ * first R_l positions of the sequence [U ; X_<j] of Eq. 6: U [n, P, D] (what
+ * photon_converter wrote for n chunks) -> the P rows of item i are encoded at
+ * positions 0..P-1, their key/value rows become rows 0..P-1 of chunk buffer
+ * unit_ids[i] (or i; the buffer must be empty: len = 0, as after a chunk
+ * boundary) and they attend causally among themselves
+ * (photon_chunk_causal_attn); y [n, P, D].  `scratch` is sized for n * P rows.
+ * With this call the converter's output reaches the chunk buffers that
+ * photon_chunk_attn and photon_decoder_step read. */
 typedef struct photon_layer {
   const photon_bf16 *g1, *wqkv, *wo, *g2, *wgu, *wdown;
   int32_t w_layout;          /* PHOTON_W_IN_MAJOR or PHOTON_W_OUT_MAJOR, all four weights */
@@ -237,6 +247,9 @@ photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *layer, co
 photon_status photon_decoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
                                   const photon_bf16 *x, photon_kv *chunks, photon_bf16 *y, float scale,
                                   photon_stream stream);
+photon_status photon_decoder_prefill(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,
+                                     const photon_bf16 *U, photon_kv *chunks, const int32_t *unit_ids, int32_t n,
+                                     photon_bf16 *y, float scale, photon_stream stream);
 
 /* Bounded causal attention of the local decoders G^(l) (Eq. 6-7): query c
  * (q [Nc, Hq, dh]) attends rows [0, len[u]) of chunk buffer u = slot ?

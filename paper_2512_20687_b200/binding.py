@@ -97,6 +97,9 @@ def load() -> ctypes.CDLL:
     lib.photon_chunk_attn.restype = st
     lib.photon_chunk_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
                                       c_int32, c_float, c_void_p]
+    lib.photon_decoder_prefill.restype = st
+    lib.photon_decoder_prefill.argtypes = [c_void_p, POINTER(photon_layer), POINTER(photon_layer_scratch), c_void_p,
+                                           POINTER(photon_kv), c_void_p, c_int32, c_void_p, c_float, c_void_p]
     lib.photon_chunk_causal_attn.restype = st
     lib.photon_chunk_causal_attn.argtypes = [c_void_p, POINTER(photon_kv), c_void_p, c_void_p, c_void_p,
                                              c_int32, c_int32, c_int32, c_float, c_void_p]
@@ -273,6 +276,13 @@ def make_layer_scratch(B, Hq, Hkv, dh, F, device, dtype) -> photon_layer_scratch
     for k, t in sc.tensors.items():
         setattr(sc, k, _ptr(t))
     return sc
+
+
+def photon_decoder_prefill(ctx, layer: photon_layer, scratch: photon_layer_scratch, U, chunks: photon_kv, unit_ids, y,
+                           n=None, scale=1.0, stream=None) -> None:
+    n = U.shape[0] if n is None else n
+    _check(load().photon_decoder_prefill(ctx, byref(layer), byref(scratch), _ptr(U), byref(chunks), _ptr(unit_ids),
+                                         int(n), _ptr(y), c_float(scale), _stream(stream)), "photon_decoder_prefill")
 
 
 def photon_decoder_step(ctx, layer: photon_layer, scratch: photon_layer_scratch, x, chunks: photon_kv, y,

@@ -162,8 +162,8 @@ cudaError_t launch_chunk_causal_attention(photon_ctx *ctx, const CausalParams &p
 cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches);
 cudaError_t launch_rmsnorm(const bf16 *x, const bf16 *gamma, float eps, bf16 *out, int rows, int cols,
                            cudaStream_t st, long long *launches);
-cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int n, int Hq, int Hkv, int dh, float theta,
-                              bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches);
+cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh,
+                              float theta, bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches);
 cudaError_t launch_swiglu(const bf16 *gu, bf16 *out, int n, int F, cudaStream_t st, long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);

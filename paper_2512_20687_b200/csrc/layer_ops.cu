@@ -35,13 +35,13 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
 
 // one CTA per item; dh <= 256
 __global__ void __launch_bounds__(EW_THREADS)
-rope_split_kernel(const bf16 *qkv, const int32_t *pos, int Hq, int Hkv, int dh, double log2_theta,
+rope_split_kernel(const bf16 *qkv, const int32_t *pos, int period, int Hq, int Hkv, int dh, double log2_theta,
                   bf16 *q, bf16 *k, bf16 *v) {
     __shared__ float cs[128], sn[128];
     ptx::grid_dep_wait();                   // qkv is the output of the kernel before this one
     ptx::grid_dep_launch();
     const int i = blockIdx.x, half = dh / 2;
-    const int at = pos[i];
+    const int at = pos ? pos[i] : i % period;          // no position array: item i is row i % period of its group
     for (int j = threadIdx.x; j < half; j += EW_THREADS) {
         double s, c;
         sincos((double)at * exp2(-2.0 * j / dh * log2_theta), &s, &c);
@@ -93,10 +93,10 @@ swiglu_kernel(const bf16 *gu, bf16 *out, int n, int F) {
 
 }  // namespace
 
-cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int n, int Hq, int Hkv, int dh, float theta,
-                              bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches) {
+cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh,
+                              float theta, bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches) {
     if (n == 0) return cudaSuccess;
-    const cudaError_t e = launch_dependent(rope_split_kernel, dim3(n), dim3(EW_THREADS), 0, st, 0, qkv, pos, Hq, Hkv, dh,
+    const cudaError_t e = launch_dependent(rope_split_kernel, dim3(n), dim3(EW_THREADS), 0, st, 0, qkv, pos, period, Hq, Hkv, dh,
                                            log2((double)theta), q, k, v);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();

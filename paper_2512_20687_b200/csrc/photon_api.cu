@@ -297,7 +297,7 @@ photon_status photon_rope_split(photon_ctx *ctx, const photon_bf16 *qkv, const i
     if (n > 0 && (!qkv || !pos || !q || !k || !v)) return PHOTON_ERR_INVALID_ARG;
     if (!aligned16(qkv) || !aligned16(q) || !aligned16(k) || !aligned16(v)) return PHOTON_ERR_INVALID_ARG;
     const photon_config &c = ctx->cfg;
-    const cudaError_t e = launch_rope_split(reinterpret_cast<const bf16 *>(qkv), pos, n, c.Hq, c.Hkv, c.dh, theta,
+    const cudaError_t e = launch_rope_split(reinterpret_cast<const bf16 *>(qkv), pos, 1, n, c.Hq, c.Hkv, c.dh, theta,
                                             reinterpret_cast<bf16 *>(q), reinterpret_cast<bf16 *>(k),
                                             reinterpret_cast<bf16 *>(v), static_cast<cudaStream_t>(stream),
                                             &ctx->launches);
@@ -354,6 +354,42 @@ photon_status photon_encoder_step(photon_ctx *ctx, const photon_layer *layer, co
                                   const photon_bf16 *x, photon_kv *cache, photon_bf16 *y, float scale,
                                   photon_stream stream) {
     return layer_step(ctx, layer, scratch, x, cache, y, scale, false, stream);
+}
+
+photon_status photon_decoder_prefill(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc,
+                                     const photon_bf16 *U, photon_kv *chunks, const int32_t *unit_ids, int32_t n,
+                                     photon_bf16 *y, float scale, photon_stream stream) {
+    if (!ctx || !L || !sc || !chunks || n < 0) return PHOTON_ERR_INVALID_ARG;
+    const photon_config &c = ctx->cfg;
+    if (!kv_ok(ctx, chunks, false) || chunks->page_table || c.Hq * c.dh != c.D || L->F <= 0 || L->F % 64 != 0)
+        return PHOTON_ERR_INVALID_ARG;
+    if (chunks->cap > c.P + c.C || chunks->cap > 64 || c.P > chunks->cap) return PHOTON_ERR_INVALID_ARG;
+    if (!unit_ids && n > chunks->n_units) return PHOTON_ERR_INVALID_ARG;
+    if (!L->g1 || !L->wqkv || !L->wo || !L->g2 || !L->wgu || !L->wdown || !(L->eps >= 0.f) || !(L->theta > 1.f))
+        return PHOTON_ERR_INVALID_ARG;
+    if (L->w_layout != PHOTON_W_IN_MAJOR && L->w_layout != PHOTON_W_OUT_MAJOR) return PHOTON_ERR_INVALID_ARG;
+    const void *ptrs[] = {L->g1, L->wqkv, L->wo, L->g2, L->wgu, L->wdown, sc->n, sc->qkv, sc->q, sc->k_new,
+                          sc->v_new, sc->att, sc->h, sc->gu, sc->act, U, y};
+    for (const void *q : ptrs)
+        if (!q || !aligned16(q)) return PHOTON_ERR_INVALID_ARG;
+    if (n == 0) return PHOTON_OK;
+    const int P = c.P, T = n * P, D = c.D, QKV = (c.Hq + 2 * c.Hkv) * c.dh;      // T rows: the P prefix vectors of n chunks
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    photon_status s = photon_rmsnorm(ctx, U, L->g1, L->eps, sc->n, T, D, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wqkv, L->w_layout, nullptr, nullptr, sc->qkv, T, D, QKV, stream);
+    if (s == PHOTON_OK &&
+        launch_rope_split(reinterpret_cast<const bf16 *>(sc->qkv), nullptr, P, T, c.Hq, c.Hkv, c.dh, L->theta,
+                          reinterpret_cast<bf16 *>(sc->q), reinterpret_cast<bf16 *>(sc->k_new),
+                          reinterpret_cast<bf16 *>(sc->v_new), st, &ctx->launches) != cudaSuccess)
+        s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK) s = photon_kv_append(ctx, chunks, sc->k_new, sc->v_new, unit_ids, n, P, stream);
+    if (s == PHOTON_OK) s = photon_chunk_causal_attn(ctx, chunks, sc->q, unit_ids, sc->att, n, 0, P, scale, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->att, L->wo, L->w_layout, nullptr, U, sc->h, T, D, D, stream);
+    if (s == PHOTON_OK) s = photon_rmsnorm(ctx, sc->h, L->g2, L->eps, sc->n, T, D, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, T, D, 2 * L->F, stream);
+    if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, T, L->F, stream);
+    if (s == PHOTON_OK) s = photon_linear(ctx, sc->act, L->wdown, L->w_layout, nullptr, sc->h, y, T, L->F, D, stream);
+    return s;
 }
 
 photon_status photon_decoder_step(photon_ctx *ctx, const photon_layer *layer, const photon_layer_scratch *scratch,

@@ -177,6 +177,62 @@ def test_decoder_step_matches_oracle(oracle, idx, B, chunks_per_seq):
     assert_close_scaled(host_f64(y), want["y"], f"decoder step cfg{idx}", slack=2.0)
 
 
+@pytest.mark.parametrize("idx,B,chunks_per_seq", [(1, 24, 2), (4, 6, 32), (0, 2, 8)])
+def test_converter_output_reaches_the_chunk_buffers(oracle, idx, B, chunks_per_seq):
+    """The chain the decode step leaves open: the converter's prefix vectors go through a
+    decoder layer (positions 0..P-1), their keys and values become the first P rows of
+    empty chunk buffers picked by unit_ids, they attend causally among themselves, and one
+    decoder step for the first in-chunk position then reads exactly those rows."""
+    cfg = cfg_small(idx, B=B, chunks_per_seq=chunks_per_seq)
+    n, P, D, F = cfg.Nc, cfg.P, cfg.D, 1024
+    cv = wl.converter_inputs(wl.scaled(cfg, B=n))
+    lw = wl.encoder_layer_inputs(wl.scaled(cfg, B=n * P), F=F)
+    cap = cfg.P + cfg.C
+    n_units = n + 3
+    ids = np.random.default_rng(idx).permutation(n_units)[:n].astype(np.int32)
+    scale = cfg.dh ** -0.5
+    U_or = oracle.round_bf16(oracle.converter(cv["x"], cv["w_in_major"], n_threads=NT))
+    ochunks = {"k": np.full((n_units, cfg.Hkv, cap, cfg.dh), 0x7FC1, np.uint16),
+               "v": np.full((n_units, cfg.Hkv, cap, cfg.dh), 0xFFC1, np.uint16), "len": np.zeros(n_units, np.int32)}
+    want = oracle.decoder_prefill(U_or, lw, ochunks, scale, unit_ids=ids, n_threads=NT)
+    with Ctx(cfg, max_queries=max(n * P, n_units)) as c:
+        W = {k: dev_bf16(lw[k]) for k in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")}
+        layer = ph.make_layer(W["g1"], W["wqkv"], W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, F)
+        sc = ph.make_layer_scratch(n * P, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        dk, dv = dev_bf16(ochunks["k"] * 0 + 0x7FC1), dev_bf16(ochunks["v"] * 0 + 0xFFC1)
+        dl = dev_i32(np.zeros(n_units, np.int32))
+        kv = ph.make_kv(dk, dv, dl)
+        U = torch.empty(n, P, D, dtype=torch.bfloat16, device="cuda")
+        ph.photon_converter(c.h, dev_bf16(cv["x"]), dev_bf16(cv["w_in_major"]), ph.PHOTON_W_IN_MAJOR, None, U)
+        assert_close(host_f64(U), wl.bf16_bits_to_f64(U_or), "converter")
+        y = torch.empty_like(U)
+        ph.photon_decoder_prefill(c.h, layer, sc, U, kv, dev_i32(ids), y, scale=scale)
+        assert c.status() == 0
+        assert np.array_equal(dl.cpu().numpy(), ochunks["len"])
+        hk = host_bits(dk)
+        got_k = host_bits(sc.tensors["k_new"]).reshape(n, P, cfg.Hkv, cfg.dh)
+        for i, u in enumerate(ids):
+            assert np.array_equal(hk[u, :, :P], got_k[i].transpose(1, 0, 2))      # the device's own rows, installed bit-exactly
+            assert np.all(hk[u, :, P:] == 0x7FC1)
+        for name in ("qkv", "q", "k_new", "att", "h", "act"):
+            got, ref = host_f64(sc.tensors[name]).reshape(n * P, -1), wl.bf16_bits_to_f64(want[name]).reshape(n * P, -1)
+            # one kernel more ahead of it than the encoder step (the converter), and the activation multiplies
+            # two intermediates: three times the single-kernel bar
+            assert_close_scaled(got, ref, f"prefill {name}", slack=3.0)
+        assert_close_scaled(host_f64(y), want["y"], "prefill output", slack=3.0)
+        # one decoder step for the first in-chunk position of the first chunks: it sees the P installed rows and itself
+        m = min(n, cfg.Nc)
+        lw2 = wl.encoder_layer_inputs(wl.scaled(cfg, B=n_units), F=F, replica=1)
+        x2 = dev_bf16(lw2["x"])
+        y2 = torch.empty_like(x2)
+        sc2 = ph.make_layer_scratch(n_units, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        ph.photon_decoder_step(c.h, layer, sc2, x2, kv, y2, scale=scale)
+        assert c.status() == 0
+        want2 = oracle.encoder_step(lw2["x"], lw, ochunks, scale, n_threads=NT)
+        assert np.array_equal(dl.cpu().numpy(), ochunks["len"])
+        assert_close_scaled(host_f64(y2), want2["y"], "decoder step after prefill", slack=3.0)
+
+
 def test_encoder_step_refuses_bad_arguments():
     cfg = cfg_small(0, B=2, S=8)
     with Ctx(cfg) as c:
