@@ -286,7 +286,10 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
     p.B = B; p.D = K; p.N = N;
     p.w_out_major = (w_layout == PHOTON_W_OUT_MAJOR);
     p.status = ctx->status;
-    const cudaError_t e = launch_linear(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+    // thousands of rows: the persistent kernel with two accumulators in TMEM; else the converter's kernel
+    const cudaError_t e = linear_wants_large_tiles(ctx, p)
+                              ? launch_linear_large(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches)
+                              : launch_linear(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 

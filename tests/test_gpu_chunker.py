@@ -43,7 +43,9 @@ def test_rmsnorm_matches_oracle(oracle, rows, cols, with_gamma):
 # a tile count that needs no split, odd batch sizes, the smallest K that is still split, K too short to split
 # and more tiles than SMs (two CTAs per SM with smaller rings)
 SHAPES = [(64, 8192, 2048), (512, 4096, 1024), (64, 2048, 8192), (1, 1024, 64), (130, 1024, 128),
-          (17, 512, 64), (200, 4096, 256), (64, 1024, 11264), (130, 512, 6400)]
+          (17, 512, 64), (200, 4096, 256), (64, 1024, 11264), (130, 512, 6400),
+          # thousands of rows: the persistent kernel (one to several tiles per CTA, a ragged last row tile)
+          (9000, 512, 1280), (16384, 256, 768), (4100, 192, 2816)]
 
 
 @pytest.mark.parametrize("B,K,N", SHAPES)
