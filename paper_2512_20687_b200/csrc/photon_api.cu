@@ -254,7 +254,9 @@ photon_status photon_converter(photon_ctx *ctx, const photon_bf16 *x, const phot
     p.B = B; p.D = ctx->cfg.D; p.N = ctx->cfg.P * ctx->cfg.D;
     p.w_out_major = (w_layout == PHOTON_W_OUT_MAJOR);
     p.status = ctx->status;
-    const cudaError_t e = launch_converter(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+    const cudaError_t e = linear_wants_large_tiles(ctx, p)      // batches of more than a thousand latents
+                              ? launch_linear_large(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches)
+                              : launch_converter(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
     return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 

@@ -263,6 +263,22 @@ def test_converter_matches_oracle(oracle, idx, rows, layout):
     assert_close(host_f64(U)[pick], want, f"converter cfg{idx}")
 
 
+def test_converter_for_thousands_of_latents(oracle):
+    """A batch large enough for the persistent large-tile kernel (more than two tiles of
+    128 x 256 per SM), ragged last row tile, with bias; the oracle recomputes a sample of rows."""
+    cfg = cfg_small(4, B=5000)                                  # D 1024, P 8: 40 x 32 tiles
+    cv = wl.converter_inputs(cfg, with_bias=True)
+    pick = np.sort(np.random.default_rng(8).choice(cfg.B, 96, replace=False))
+    pick[-1] = cfg.B - 1
+    want = oracle.converter(cv["x"][pick], cv["w_out_major"], cv["bias"], w_out_major=True, n_threads=NT)
+    with Ctx(cfg) as c:
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        ph.photon_converter(c.h, dev_bf16(cv["x"]), dev_bf16(cv["w_out_major"]), ph.PHOTON_W_OUT_MAJOR,
+                            dev_bf16(cv["bias"]), U)
+        assert c.status() == 0
+    assert_close(host_f64(U)[pick], want, "converter, 5000 latents")
+
+
 def test_converter_one_hot_rows_are_bit_exact_and_ragged_batches_work():
     cfg = cfg_small(0, B=37)
     cv = wl.converter_inputs(cfg)
