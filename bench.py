@@ -556,6 +556,10 @@ def run_gpu(args, cfg) -> None:
                 ph.photon_encoder_step(ctx, layers[i % R], scr, ex, plain_kv[i % R], ey, scale=scale)
 
             lens.copy_(lens0)
+            n_l0 = ph.photon_launch_count(ctx)
+            layer_call(None)
+            launches_e = ph.photon_launch_count(ctx) - n_l0
+            lens.copy_(lens0)
             us_e = graph_time_us(layer_call, reset_lens=True)
             lens.copy_(lens0)
             QKV = (cfg.Hq + 2 * cfg.Hkv) * cfg.dh
@@ -565,7 +569,7 @@ def run_gpu(args, cfg) -> None:
             widened["encoder_step"] = {
                 "workload": "one layer, batch %d: D %d, %dq/%dkv x %d, F %d, cache of %d latents per sequence" % (
                     cfg.B, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh, F, cfg.S),
-                "us": us_e, "launches": 10, "algorithmic_bytes": ebytes, "GBps": ebytes / us_e * 1e-3,
+                "us": us_e, "launches": launches_e, "algorithmic_bytes": ebytes, "GBps": ebytes / us_e * 1e-3,
                 "frac_hbm": ebytes / us_e * 1e-3 / hbm_peak, "TFLOPs": eflops / us_e * 1e-6,
                 "note": "weights and the sequences' own K/V rows counted once (no shared prefix), activations not counted"}
 
@@ -586,6 +590,9 @@ def run_gpu(args, cfg) -> None:
                 dlen.copy_(dlen0)
                 ph.photon_decoder_step(ctx, layers[i % R], dscr, dx, dkv[i % R], dy, scale=scale)
 
+            n_l0 = ph.photon_launch_count(ctx)
+            dec_call(None)
+            launches_d = ph.photon_launch_count(ctx) - n_l0
             us_d = graph_time_us(dec_call)
             dbytes = wbytes + int(dlen0.sum().item() + cfg.Nc) * cfg.Hkv * cfg.dh * 4 + 2 * cfg.Nc * cfg.D * 2
             dflops = 2.0 * cfg.Nc * (wbytes / 2)
@@ -593,7 +600,7 @@ def run_gpu(args, cfg) -> None:
             widened["decoder_step"] = {
                 "workload": "one layer, %d in-flight chunks (one new token each): D %d, F %d, windows of at most %d rows" % (
                     cfg.Nc, cfg.D, F, cfg.P + cfg.C),
-                "us": us_d, "launches": 10, "algorithmic_bytes": dbytes, "GBps": dbytes / us_d * 1e-3,
+                "us": us_d, "launches": launches_d, "algorithmic_bytes": dbytes, "GBps": dbytes / us_d * 1e-3,
                 "frac_hbm": dbytes / us_d * 1e-3 / hbm_peak, "TFLOPs": dflops / us_d * 1e-6,
                 "frac_of_own_roofline": t_roof / us_d,
                 "note": "weights, the chunks' K/V rows, x and y counted once; the figure includes one small copy that "
@@ -613,13 +620,16 @@ def run_gpu(args, cfg) -> None:
                 plen.zero_()
                 ph.photon_decoder_prefill(ctx, layers[i % R], pscr, pU, pkv2[i % 2], None, pY, n=n_pre, scale=scale)
 
+            n_l0 = ph.photon_launch_count(ctx)
+            prefill_call(None)
+            launches_p = ph.photon_launch_count(ctx) - n_l0
             us_pf = graph_time_us(prefill_call)
             pflops = 2.0 * n_pre * cfg.P * (wbytes / 2)
             pbytes = wbytes + 2 * n_pre * cfg.P * cfg.D * 2 + 2 * n_pre * cfg.P * cfg.Hkv * cfg.dh * 2
             t_roof = max(pbytes / (hbm_peak * 1e3), pflops / (tensor_peak * 1e6))
             widened["decoder_prefill"] = {
                 "workload": "one layer over the %d prefix vectors of each of %d chunks" % (cfg.P, n_pre),
-                "us": us_pf, "launches": 10, "algorithmic_bytes": pbytes, "GBps": pbytes / us_pf * 1e-3,
+                "us": us_pf, "launches": launches_p, "algorithmic_bytes": pbytes, "GBps": pbytes / us_pf * 1e-3,
                 "frac_hbm": pbytes / us_pf * 1e-3 / hbm_peak, "TFLOPs": pflops / us_pf * 1e-6,
                 "frac_of_own_roofline": t_roof / us_pf,
                 "note": "weights, U, y and the installed K/V rows counted once; includes the small kernel that empties the lengths"}

@@ -202,7 +202,9 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
  * weights in the order w_layout names: wqkv [D, (Hq + 2 Hkv) dh], wo [Hq dh,
  * D], wgu [D, 2F], wdown [F, D]; g1, g2 [D].  F a multiple of 64.  The
  * caller owns the intermediates in `scratch` (sizes beside the fields); each
- * is rounded to bf16 where the next kernel reads it.  y may alias x.
+ * is rounded to bf16 where the next kernel reads it.  y may alias x.  With
+ * thousands of rows the gate/up projection and the activation are one launch
+ * and scratch->gu is left unwritten (nine launches).
  *
  * photon_decoder_step: the same layer of a local decoder G^(l) (Eq. 6-7) for
  * the newest in-chunk position of every in-flight chunk: `chunks` holds the

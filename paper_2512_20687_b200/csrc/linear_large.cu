@@ -12,6 +12,12 @@
 // boundaries.  Shared memory: 4 stages of one K block of 64 (x atom 16 KiB,
 // weight atom 32 KiB).  Every wait is bounded; a wait that gives up sets the
 // status bit and a flag that makes every role leave its loops.
+//
+// GATED: the gate/up projection of the MLP with its activation folded in.  The
+// weight is [gate | up] (N = 2F columns); a tile takes 128 gate columns and the
+// 128 up columns of the same features as its two halves, and the epilogue writes
+// silu(g) * u for those 128 features: out [B, F], and the [B, 2F] intermediate
+// never exists.
 #include <algorithm>
 
 #include "common.cuh"
@@ -26,7 +32,7 @@ constexpr int RING = STAGES * STAGE_BYTES;
 constexpr int LL_THREADS = 192;             // warp 0: TMA, warp 1: MMA (owns TMEM), warps 2-5: epilogue
 constexpr int LL_SMEM = RING + 1024 + 256;
 
-template <bool W_IN_MAJOR>
+template <bool W_IN_MAJOR, bool GATED>
 __global__ void __launch_bounds__(LL_THREADS, 1)
 linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
                     const __grid_constant__ CUtensorMap tm_w) {
@@ -39,7 +45,8 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
     volatile int *dead = reinterpret_cast<volatile int *>(gen + RING + 16 * STAGES + 40);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_tiles = (p.B + BM - 1) / BM, n_tiles = p.N / NT;
+    const int F = p.N / 2;                                      // GATED: features; a tile covers 128 of them
+    const int m_tiles = (p.B + BM - 1) / BM, n_tiles = GATED ? F / (NT / 2) : p.N / NT;
     const int tiles = m_tiles * n_tiles, n_atoms = p.D / BK;
 
     if (threadIdx.x == 0) {
@@ -72,7 +79,7 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
         int s = 0;
         uint32_t phase = 0;
         for (int t = blockIdx.x; t < tiles && !*dead; t += gridDim.x) {
-            const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * NT;
+            const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * (GATED ? NT / 2 : NT);
             for (int a = 0; a < n_atoms; ++a) {
                 if (!__all_sync(0xffffffffu, ptx::mbar_wait(bars + 16 * s + 8, phase ^ 1))) { give_up(); break; }
                 const uint32_t full = bars + 16 * s, a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_BYTES;
@@ -81,11 +88,18 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
                     const int k0 = a * BK;
                     ptx::tma_load_2d(a_dst, &tm_x, k0, m0, full);                        // x[m0.., k0..]
                     if (!W_IN_MAJOR) {
-                        ptx::tma_load_2d(b_dst, &tm_w, k0, n0, full);                    // W[n0.., k0..]  (K-major)
+                        if (GATED) {                                                      // boxes of 128 rows: gate, then up
+                            ptx::tma_load_2d(b_dst, &tm_w, k0, n0, full);
+                            ptx::tma_load_2d(b_dst + B_BYTES / 2, &tm_w, k0, F + n0, full);
+                        } else {
+                            ptx::tma_load_2d(b_dst, &tm_w, k0, n0, full);                // W[n0.., k0..]  (K-major)
+                        }
                     } else {
 #pragma unroll
-                        for (int jj = 0; jj < NT / 64; ++jj)                              // W[k0.., n0+64jj..] (N-major)
-                            ptx::tma_load_2d(b_dst + jj * (BK * 128), &tm_w, n0 + 64 * jj, k0, full);
+                        for (int jj = 0; jj < NT / 64; ++jj) {                            // W[k0.., n..] (N-major), 64 columns a box
+                            const int col = GATED ? (jj < 2 ? n0 + 64 * jj : F + n0 + 64 * (jj - 2)) : n0 + 64 * jj;
+                            ptx::tma_load_2d(b_dst + jj * (BK * 128), &tm_w, col, k0, full);
+                        }
                     }
                 }
                 __syncwarp();
@@ -129,10 +143,38 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
         int i = 0;
         for (int t = blockIdx.x; t < tiles && !*dead; t += gridDim.x, ++i) {
             const int buf = i & 1;
-            const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * NT;
+            const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * (GATED ? NT / 2 : NT);
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(acc_full + 8 * buf, (i >> 1) & 1))) { give_up(); break; }
             ptx::tc_fence_after();
             const int b = m0 + quad * 32 + lane;
+            if constexpr (GATED) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < NT / 2; c0 += 32) {
+                    uint32_t g[32], u[32];
+                    ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + buf * NT + c0, g);
+                    ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + buf * NT + NT / 2 + c0, u);
+                    ptx::tmem_ld_wait();
+                    if (b < p.B) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.U + (size_t)b * F + n0 + c0);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                // the projections are rounded to bf16 first, as when they are stored and read back
+                                const float g0 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(g[v * 8 + 2 * e])));
+                                const float g1 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(g[v * 8 + 2 * e + 1])));
+                                const float u0 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(u[v * 8 + 2 * e])));
+                                const float u1 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(u[v * 8 + 2 * e + 1])));
+                                __nv_bfloat162 o = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * u0,
+                                                                         g1 / (1.f + __expf(-g1)) * u1);
+                                w[e] = *reinterpret_cast<uint32_t *>(&o);
+                            }
+                            dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+            } else {
 #pragma unroll 1
             for (int c0 = 0; c0 < NT; c0 += 32) {
                 uint32_t r[32];
@@ -161,6 +203,7 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
                     }
                 }
             }
+            }
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * buf);          // the MMA warp may overwrite this buffer
@@ -174,20 +217,20 @@ linear_tiles_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x
     }
 }
 
-template <bool IN_MAJOR>
+template <bool IN_MAJOR, bool GATED>
 cudaError_t run_large(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
     static size_t smem_set[kMaxDevices] = {};
-    if (const cudaError_t e = ensure_dynamic_smem(linear_tiles_kernel<IN_MAJOR>, LL_SMEM, ctx->device, smem_set)) return e;
+    if (const cudaError_t e = ensure_dynamic_smem(linear_tiles_kernel<IN_MAJOR, GATED>, LL_SMEM, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
     CUtensorMap mx, mw;
     if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, BM))) return cudaErrorInvalidValue;
     mx = *t;
     if (IN_MAJOR) t = ctx->tmaps.get(p.w, (uint64_t)p.D, (uint64_t)p.N, BK);        // [K, N], boxes of 64 k x 64 n
-    else t = ctx->tmaps.get(p.w, (uint64_t)p.N, (uint64_t)p.D, NT);                 // [N, K], boxes of 256 n x 64 k
+    else t = ctx->tmaps.get(p.w, (uint64_t)p.N, (uint64_t)p.D, GATED ? NT / 2 : NT);   // [N, K], boxes of 256 (128) n x 64 k
     if (!t) return cudaErrorInvalidValue;
     mw = *t;
-    const int tiles = ((p.B + BM - 1) / BM) * (p.N / NT);
-    const cudaError_t e = launch_dependent(linear_tiles_kernel<IN_MAJOR>, dim3(std::min(tiles, ctx->sm_count)),
+    const int tiles = ((p.B + BM - 1) / BM) * (p.N / NT);                           // (the same count when gated)
+    const cudaError_t e = launch_dependent(linear_tiles_kernel<IN_MAJOR, GATED>, dim3(std::min(tiles, ctx->sm_count)),
                                            dim3(LL_THREADS), LL_SMEM, st, 0, p, mx, mw);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
@@ -201,5 +244,11 @@ bool linear_wants_large_tiles(const photon_ctx *ctx, const ConvParams &p) {
 }
 
 cudaError_t launch_linear_large(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
-    return p.w_out_major ? run_large<false>(ctx, p, st, launches) : run_large<true>(ctx, p, st, launches);
+    return p.w_out_major ? run_large<false, false>(ctx, p, st, launches) : run_large<true, false>(ctx, p, st, launches);
+}
+
+// out [B, F] = silu(x Wg) * (x Wu) for w = [Wg | Wu] with N = 2F columns; for the shapes
+// linear_wants_large_tiles accepts.  No bias, no residual.
+cudaError_t launch_gate_up_large(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
+    return p.w_out_major ? run_large<false, true>(ctx, p, st, launches) : run_large<true, true>(ctx, p, st, launches);
 }

@@ -320,6 +320,27 @@ photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 
 }
 
 namespace {
+// gate/up projection and activation: act [rows, F] = silu(n Wg) * (n Wu).  With thousands of rows one fused
+// launch of the large-tile kernel (gu is then not written); else the projection followed by photon_swiglu.
+photon_status gate_up(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc, int rows,
+                      photon_stream stream) {
+    const photon_config &c = ctx->cfg;
+    ConvParams p{};
+    p.x = reinterpret_cast<const bf16 *>(sc->n);
+    p.w = reinterpret_cast<const bf16 *>(L->wgu);
+    p.U = reinterpret_cast<bf16 *>(sc->act);
+    p.B = rows; p.D = c.D; p.N = 2 * L->F;
+    p.w_out_major = (L->w_layout == PHOTON_W_OUT_MAJOR);
+    p.status = ctx->status;
+    if (L->F % 128 == 0 && linear_wants_large_tiles(ctx, p)) {
+        const cudaError_t e = launch_gate_up_large(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+        return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+    }
+    photon_status s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, rows, c.D, 2 * L->F, stream);
+    if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, rows, L->F, stream);
+    return s;
+}
+
 // STEP of one layer for the newest position of every unit of `cache`; local: the cache is a set of chunk
 // buffers read by the chunk attention, else a coarse stream read by the coarse attention.
 photon_status layer_step(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc,
@@ -348,8 +369,7 @@ photon_status layer_step(photon_ctx *ctx, const photon_layer *L, const photon_la
                   : photon_coarse_attn(ctx, cache, sc->q, sc->att, nullptr, scale, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->att, L->wo, L->w_layout, nullptr, x, sc->h, B, D, D, stream);
     if (s == PHOTON_OK) s = photon_rmsnorm(ctx, sc->h, L->g2, L->eps, sc->n, B, D, stream);
-    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, B, D, 2 * L->F, stream);
-    if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, B, L->F, stream);
+    if (s == PHOTON_OK) s = gate_up(ctx, L, sc, B, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->act, L->wdown, L->w_layout, nullptr, sc->h, y, B, L->F, D, stream);
     return s;
 }
@@ -391,8 +411,7 @@ photon_status photon_decoder_prefill(photon_ctx *ctx, const photon_layer *L, con
     if (s == PHOTON_OK) s = photon_chunk_causal_attn(ctx, chunks, sc->q, unit_ids, sc->att, n, 0, P, scale, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->att, L->wo, L->w_layout, nullptr, U, sc->h, T, D, D, stream);
     if (s == PHOTON_OK) s = photon_rmsnorm(ctx, sc->h, L->g2, L->eps, sc->n, T, D, stream);
-    if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, T, D, 2 * L->F, stream);
-    if (s == PHOTON_OK) s = photon_swiglu(ctx, sc->gu, sc->act, T, L->F, stream);
+    if (s == PHOTON_OK) s = gate_up(ctx, L, sc, T, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->act, L->wdown, L->w_layout, nullptr, sc->h, y, T, L->F, D, stream);
     return s;
 }

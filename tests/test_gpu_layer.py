@@ -233,6 +233,36 @@ def test_converter_output_reaches_the_chunk_buffers(oracle, idx, B, chunks_per_s
         assert_close_scaled(host_f64(y2), want2["y"], "decoder step after prefill", slack=3.0)
 
 
+@pytest.mark.parametrize("layout", ["in", "out"])
+def test_decoder_step_with_thousands_of_chunks_fuses_the_activation(oracle, layout):
+    """5120 in-flight chunks: the gate/up projection takes the persistent large-tile kernel with
+    the activation in its epilogue (the [rows, 2F] intermediate is never written); both weight orders."""
+    cfg = cfg_small(0, B=640, chunks_per_seq=8)                          # D 256, 4q/2kv x 64, P = C = 4
+    Nc, F = cfg.Nc, 1024
+    lw = wl.encoder_layer_inputs(wl.scaled(cfg, B=Nc), F=F)
+    ch = wl.chunk_inputs(cfg, poison=True, strict_paper=True)
+    scale = cfg.dh ** -0.5
+    cache = {"k": ch["kc"].copy(), "v": ch["vc"].copy(), "len": ch["len"].copy()}
+    want = oracle.encoder_step(lw["x"], lw, cache, scale, n_threads=NT)
+    out_major = layout == "out"
+    with Ctx(cfg) as c:
+        kv = ph.make_kv(dev_bf16(ch["kc"]), dev_bf16(ch["vc"]), dev_i32(ch["len"]))
+        names = ("g1", "wqkv", "wo", "g2", "wgu", "wdown")
+        W = {n: dev_bf16(np.ascontiguousarray(lw[n].T) if out_major and lw[n].ndim == 2 else lw[n]) for n in names}
+        layer = ph.make_layer(*(W[n] for n in names), ph.PHOTON_W_OUT_MAJOR if out_major else ph.PHOTON_W_IN_MAJOR, F)
+        sc = ph.make_layer_scratch(Nc, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        sc.tensors["gu"].fill_(7.0)
+        x = dev_bf16(lw["x"])
+        y = torch.empty_like(x)
+        n0 = ph.photon_launch_count(c.h)
+        ph.photon_decoder_step(c.h, layer, sc, x, kv, y, scale=scale)
+        assert c.status() == 0
+        assert ph.photon_launch_count(c.h) - n0 == 9                     # one launch fewer than the ten of a small batch
+        assert bool((sc.tensors["gu"] == 7.0).all())                     # the intermediate was not written
+        assert_close_scaled(host_f64(sc.tensors["act"]), wl.bf16_bits_to_f64(want["act"]), "fused activation", slack=2.0)
+    assert_close_scaled(host_f64(y), want["y"], "decoder step, 5120 chunks", slack=2.0)
+
+
 def test_encoder_step_refuses_bad_arguments():
     cfg = cfg_small(0, B=2, S=8)
     with Ctx(cfg) as c:
