@@ -129,6 +129,35 @@ def test_gather_through_slots_and_bad_slots(oracle):
     assert_close(got, want, "causal chunk gather")
 
 
+def test_many_chunks_through_slots_handed_out_from_the_counter(oracle):
+    """Enough items for the kernel to hand them out from its global counter (more than 16
+    per warp), gathered through a random slot array with repeats and two bad entries;
+    twice, so that the counters are seen to be back at zero."""
+    cfg = cfg_small(4, B=64)                                  # 2048 chunk buffers, 8 KV heads
+    ch = wl.chunk_causal_inputs(cfg, poison=True)
+    scale = cfg.dh ** -0.5
+    n = 6000                                                  # 48 000 items over at most 1184 warps
+    slot = np.random.default_rng(6).integers(0, cfg.Nc, n).astype(np.int32)
+    slot[17], slot[n - 2] = -3, cfg.Nc
+    q = wl.normal_bf16(4, "qrows_many", (n, ch["rows"], cfg.Hq, cfg.dh))
+    pick = np.sort(np.random.default_rng(7).choice(n, 150, replace=False))
+    pick[0], pick[1], pick[-1] = 17, n - 2, n - 1
+    pick.sort()
+    want, flags = oracle.chunk_causal_attention(q[pick], ch["kc"], ch["vc"], ch["len"], scale, slot=slot[pick],
+                                                n_threads=NT, want_flags=True)
+    with Ctx(cfg, max_queries=n) as c:
+        d = chunks_to_dev(ch)
+        dq, ds = dev_bf16(q), dev_i32(slot)
+        a = run(c, d, dq, slot=ds, scale=scale)
+        assert c.status() == flags == ph.PHOTON_DEV_BAD_INDEX
+        b = run(c, d, dq, slot=ds, scale=scale, fill=3.0)
+        assert c.status() == ph.PHOTON_DEV_BAD_INDEX
+    got = host_f64(a)
+    assert np.array_equal(host_bits(a), host_bits(b))
+    assert np.all(got[17] == 0) and np.all(got[n - 2] == 0)
+    assert_close(got[pick], want, "causal chunk, handed out from the counter")
+
+
 def test_last_row_agrees_with_the_single_query_kernel():
     """The row at position len-1 is what the decode step's chunk attention computes
     for the newest position; two different kernels, same bf16 result up to rounding."""

@@ -67,6 +67,26 @@ def test_linear_matches_oracle(oracle, B, K, N, out_major):
     assert_close(host_f64(y), want, f"linear {B}x{K}x{N}")
 
 
+def test_large_tile_kernel_adds_bias_and_residual_and_is_deterministic(oracle):
+    """Thousands of rows with bias and a residual that aliases the output; the oracle
+    recomputes a sample of rows; two calls give the same bits."""
+    B, K, N = 6000, 320, 1792
+    x = wl.normal_bf16(24, "x", (B, K))
+    w = wl.normal_bf16(24, "w", (K, N), std=K ** -0.5)
+    bias, res = wl.normal_bf16(24, "b", (N,), std=0.5), wl.normal_bf16(24, "r", (B, N))
+    pick = np.sort(np.random.default_rng(3).choice(B, 200, replace=False))
+    pick[0], pick[-1] = 0, B - 1
+    want = oracle.linear(x[pick], w, bias, n_threads=NT) + wl.bf16_bits_to_f64(res[pick])
+    with Ctx(cfg_small(0)) as c:
+        dx, dw, db = dev_bf16(x), dev_bf16(w), dev_bf16(bias)
+        y1, y2 = dev_bf16(res).clone(), dev_bf16(res).clone()
+        ph.photon_linear(c.h, dx, dw, ph.PHOTON_W_IN_MAJOR, db, y1, residual=y1)
+        ph.photon_linear(c.h, dx, dw, ph.PHOTON_W_IN_MAJOR, db, y2, residual=y2)
+        assert c.status() == 0
+    assert np.array_equal(host_bits(y1), host_bits(y2))
+    assert_close(host_f64(y1)[pick], want, "large tiles, bias + residual")
+
+
 def test_linear_one_hot_rows_return_weight_rows_bit_exactly():
     K, N = 4096, 128                                                     # split over a cluster
     w = wl.normal_bf16(23, "w", (K, N))
