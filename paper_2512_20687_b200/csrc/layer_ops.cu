@@ -7,8 +7,10 @@
 //  * swiglu_kernel: out = silu(gate) * up for gu [n, 2F] = [gate | up].
 // Both are tiny and bound by launch and memory latency: 16-byte accesses, one
 // rounding to bf16 at the output.  The angles are computed in double precision
-// once per item (positions reach thousands of radians, which fast single-
-// precision sines do not survive) and shared by all heads through shared memory.
+// once per item and reduced to [-pi, pi] there (positions reach thousands of
+// radians, which single-precision sines do not survive); the remainder goes
+// through the fast single-precision sine and cosine, and all heads share the
+// table through shared memory.
 #include <algorithm>
 #include <cmath>
 
@@ -43,9 +45,13 @@ rope_split_kernel(const bf16 *qkv, const int32_t *pos, int period, int Hq, int H
     const int i = blockIdx.x, half = dh / 2;
     const int at = pos ? pos[i] : i % period;          // no position array: item i is row i % period of its group
     for (int j = threadIdx.x; j < half; j += EW_THREADS) {
-        double s, c;
-        sincos((double)at * exp2(-2.0 * j / dh * log2_theta), &s, &c);
-        cs[j] = (float)c; sn[j] = (float)s;
+        // the angle and its reduction to [-pi, pi] in double precision, sine and cosine of the remainder in single
+        const double a = (double)at * exp2(-2.0 * j / dh * log2_theta);
+        const double turns = rint(a * 0.15915494309189535);
+        const float r = (float)fma(turns, -6.283185307179586, a);
+        float s, c;
+        __sincosf(r, &s, &c);
+        cs[j] = c; sn[j] = s;
     }
     __syncthreads();
     const int width = (Hq + 2 * Hkv) * dh;

@@ -20,7 +20,8 @@ def cfg_small(i, **kw):
     return wl.scaled(wl.CONFIGS[i], **kw)
 
 
-@pytest.mark.parametrize("rows,cols,with_gamma", [(64, 8192, True), (5, 4096, False), (3, 8, True), (130, 1032, True)])
+@pytest.mark.parametrize("rows,cols,with_gamma", [(64, 8192, True), (5, 4096, False), (3, 8, True), (130, 1032, True),
+                                                  (3000, 1032, True), (1025, 2048, False), (1500, 8, True)])
 def test_rmsnorm_matches_oracle(oracle, rows, cols, with_gamma):
     x = wl.normal_bf16(21, "x", (rows, cols), std=3.0)
     g = wl.f32_to_bf16_bits((wl.bf16_bits_to_f64(wl.normal_bf16(21, "g", (cols,), std=0.2)) + 1.0).astype(np.float32))
