@@ -7,7 +7,7 @@
 //  * swiglu_kernel: out = silu(gate) * up for gu [n, 2F] = [gate | up].
 // Both are tiny and bound by launch and memory latency: 16-byte accesses, one
 // rounding to bf16 at the output.  The angles are computed in double precision
-// once per item and reduced to [-pi, pi] there (positions reach thousands of
+// per item and reduced to [-pi, pi] there (positions reach thousands of
 // radians, which single-precision sines do not survive); the remainder goes
 // through the fast single-precision sine and cosine, and all heads share the
 // table through shared memory.
@@ -35,48 +35,75 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
     return u;
 }
 
-// one CTA per item; dh <= 256
+// Items are dealt to the CTAs round-robin.  The sines and cosines of an item are shared by all its
+// heads through shared memory; the table of a CTA's next item (and the position of the one after)
+// is prepared while the current item's data is in flight, so one barrier per item is all the
+// synchronisation there is.  The inverse wavelengths do not depend on the item: once per thread.
 __global__ void __launch_bounds__(EW_THREADS)
-rope_split_kernel(const bf16 *qkv, const int32_t *pos, int period, int Hq, int Hkv, int dh, double log2_theta,
+rope_split_kernel(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh, double log2_theta,
                   bf16 *q, bf16 *k, bf16 *v) {
-    __shared__ float cs[128], sn[128];
+    __shared__ __align__(16) float cs[2][128], sn[2][128];
+    const int half = dh / 2, vec_half = half / 8;        // 16-byte pieces per half head
+    const int j0 = (threadIdx.x % vec_half) * 8;         // 256 is a multiple of vec_half: the same features for every piece
+    const double inv = exp2(-2.0 * (double)threadIdx.x / dh * log2_theta);
+    const int rotated = (Hq + Hkv) * vec_half, copied = Hkv * dh / 8;
+    const int width = (Hq + 2 * Hkv) * dh, step = gridDim.x;
     ptx::grid_dep_wait();                   // qkv is the output of the kernel before this one
     ptx::grid_dep_launch();
-    const int i = blockIdx.x, half = dh / 2;
-    const int at = pos ? pos[i] : i % period;          // no position array: item i is row i % period of its group
-    for (int j = threadIdx.x; j < half; j += EW_THREADS) {
+    auto where = [&](int i) { return i < n ? (pos ? pos[i] : i % period) : 0; };   // no position array: row i % period of its group
+    auto table = [&](int at, int buf) {
         // the angle and its reduction to [-pi, pi] in double precision, sine and cosine of the remainder in single
-        const double a = (double)at * exp2(-2.0 * j / dh * log2_theta);
+        const double a = (double)at * inv;
         const double turns = rint(a * 0.15915494309189535);
-        const float r = (float)fma(turns, -6.283185307179586, a);
-        float s, c;
-        __sincosf(r, &s, &c);
-        cs[j] = c; sn[j] = s;
+        __sincosf((float)fma(turns, -6.283185307179586, a), &sn[buf][threadIdx.x], &cs[buf][threadIdx.x]);
+    };
+    const bool tabler = (int)threadIdx.x < half;
+    int at_next = 0;
+    if (tabler) {
+        table(where(blockIdx.x), 0);
+        at_next = where(blockIdx.x + step);
     }
     __syncthreads();
-    const int width = (Hq + 2 * Hkv) * dh;
-    const bf16 *row = qkv + (size_t)i * width;
-    const int vec_half = half / 8;                       // 16-byte pieces per half head
-    // rotated heads: piece p of head h covers features [8p, 8p + 8) and their partners 8p + half ..
-    for (int w = threadIdx.x; w < (Hq + Hkv) * vec_half; w += EW_THREADS) {
-        const int h = w / vec_half, j0 = (w % vec_half) * 8;
-        const bf16 *x = row + (size_t)h * dh;
-        bf16 *o = h < Hq ? q + ((size_t)i * Hq + h) * dh : k + ((size_t)i * Hkv + (h - Hq)) * dh;
-        float a[8], b[8], ra[8], rb[8];
-        unpack8(*reinterpret_cast<const uint4 *>(x + j0), a);
-        unpack8(*reinterpret_cast<const uint4 *>(x + j0 + half), b);
+    int buf = 0;
+    for (int i = blockIdx.x; i < n; i += step, buf ^= 1) {
+        const bf16 *row = qkv + (size_t)i * width;
+        // piece p of head h covers features [8p, 8p + 8) and their partners 8p + half ..
+        for (int w0 = 0; w0 < rotated + copied; w0 += EW_THREADS) {
+            const int w = w0 + threadIdx.x;
+            uint4 ua = {}, ub = {};
+            const int h = w / vec_half;
+            if (w < rotated) {
+                ua = *reinterpret_cast<const uint4 *>(row + (size_t)h * dh + j0);
+                ub = *reinterpret_cast<const uint4 *>(row + (size_t)h * dh + j0 + half);
+            } else if (w < rotated + copied) {
+                ua = reinterpret_cast<const uint4 *>(row + (size_t)(Hq + Hkv) * dh)[w - rotated];
+            }
+            if (w0 == 0 && tabler) {                       // under the loads: the next item's table, the position after it
+                table(at_next, buf ^ 1);
+                at_next = where(i + 2 * step);
+            }
+            if (w < rotated) {
+                bf16 *o = h < Hq ? q + ((size_t)i * Hq + h) * dh : k + ((size_t)i * Hkv + (h - Hq)) * dh;
+                float a[8], b[8], c[8], s[8], ra[8], rb[8];
+                unpack8(ua, a);
+                unpack8(ub, b);
+                *reinterpret_cast<float4 *>(c) = *reinterpret_cast<const float4 *>(&cs[buf][j0]);
+                *reinterpret_cast<float4 *>(c + 4) = *reinterpret_cast<const float4 *>(&cs[buf][j0 + 4]);
+                *reinterpret_cast<float4 *>(s) = *reinterpret_cast<const float4 *>(&sn[buf][j0]);
+                *reinterpret_cast<float4 *>(s + 4) = *reinterpret_cast<const float4 *>(&sn[buf][j0 + 4]);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float c = cs[j0 + e], s = sn[j0 + e];
-            ra[e] = a[e] * c - b[e] * s;
-            rb[e] = b[e] * c + a[e] * s;
+                for (int e = 0; e < 8; ++e) {
+                    ra[e] = a[e] * c[e] - b[e] * s[e];
+                    rb[e] = b[e] * c[e] + a[e] * s[e];
+                }
+                *reinterpret_cast<uint4 *>(o + j0) = pack8(ra);
+                *reinterpret_cast<uint4 *>(o + j0 + half) = pack8(rb);
+            } else if (w < rotated + copied) {
+                reinterpret_cast<uint4 *>(v + (size_t)i * Hkv * dh)[w - rotated] = ua;
+            }
         }
-        *reinterpret_cast<uint4 *>(o + j0) = pack8(ra);
-        *reinterpret_cast<uint4 *>(o + j0 + half) = pack8(rb);
+        __syncthreads();
     }
-    const uint4 *vs = reinterpret_cast<const uint4 *>(row + (size_t)(Hq + Hkv) * dh);
-    uint4 *vd = reinterpret_cast<uint4 *>(v + (size_t)i * Hkv * dh);
-    for (int w = threadIdx.x; w < Hkv * dh / 8; w += EW_THREADS) vd[w] = vs[w];
 }
 
 __global__ void __launch_bounds__(EW_THREADS)
@@ -102,7 +129,7 @@ swiglu_kernel(const bf16 *gu, bf16 *out, int n, int F) {
 cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh,
                               float theta, bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches) {
     if (n == 0) return cudaSuccess;
-    const cudaError_t e = launch_dependent(rope_split_kernel, dim3(n), dim3(EW_THREADS), 0, st, 0, qkv, pos, period, Hq, Hkv, dh,
+    const cudaError_t e = launch_dependent(rope_split_kernel, dim3(std::min(n, 148 * 8)), dim3(EW_THREADS), 0, st, 0, qkv, pos, period, n, Hq, Hkv, dh,
                                            log2((double)theta), q, k, v);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
