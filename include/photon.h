@@ -195,16 +195,18 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
  * [n, F], F a multiple of 8.
  *
  * photon_encoder_step: the whole layer for the newest latent of every
- * sequence, ten kernels on `stream`: normalise x (g1) -> wqkv -> rope_split
- * at position len[b] -> append k, v to `cache` (len += 1) -> attention over
- * the grown cache -> wo + x -> normalise (g2) -> wgu -> swiglu -> wdown + h.
+ * sequence, nine kernels on `stream`: normalise x (g1) -> wqkv -> rope_split
+ * at position len[b], which here writes k and v straight into row len[b] of
+ * `cache` and sets len += 1 (contiguous or paged; the checks and status bits
+ * of photon_kv_append; scratch->k_new and v_new stay unwritten) -> attention
+ * over the grown cache -> wo + x -> normalise (g2) -> wgu -> swiglu -> wdown + h.
  * x, y [B, D] with B = cache->n_units and D = Hq * dh of the context;
  * weights in the order w_layout names: wqkv [D, (Hq + 2 Hkv) dh], wo [Hq dh,
  * D], wgu [D, 2F], wdown [F, D]; g1, g2 [D].  F a multiple of 64.  The
  * caller owns the intermediates in `scratch` (sizes beside the fields); each
  * is rounded to bf16 where the next kernel reads it.  y may alias x.  With
  * thousands of rows the gate/up projection and the activation are one launch
- * and scratch->gu is left unwritten (nine launches).
+ * and scratch->gu is left unwritten (eight launches).
  *
  * photon_decoder_step: the same layer of a local decoder G^(l) (Eq. 6-7) for
  * the newest in-chunk position of every in-flight chunk: `chunks` holds the
@@ -232,7 +234,7 @@ typedef struct photon_layer_scratch {
   photon_bf16 *n;            /* [B, D]   normalised input of either half */
   photon_bf16 *qkv;          /* [B, (Hq + 2 Hkv) dh] */
   photon_bf16 *q;            /* [B, Hq, dh] */
-  photon_bf16 *k_new, *v_new;/* [B, Hkv, dh] */
+  photon_bf16 *k_new, *v_new;/* [B, Hkv, dh]  written by photon_decoder_prefill only */
   photon_bf16 *att;          /* [B, Hq, dh] */
   photon_bf16 *h;            /* [B, D]   after the attention half */
   photon_bf16 *gu;           /* [B, 2F] */

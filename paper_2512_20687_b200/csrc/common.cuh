@@ -167,6 +167,10 @@ cudaError_t launch_rmsnorm(const bf16 *x, const bf16 *gamma, float eps, bf16 *ou
                            cudaStream_t st, long long *launches);
 cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh,
                               float theta, bf16 *q, bf16 *k, bf16 *v, cudaStream_t st, long long *launches);
+// the same split with k and v written into row len[i] of unit i of a cache (contiguous or paged) and len[i] += 1
+cudaError_t launch_rope_split_append(const bf16 *qkv, int n, int Hq, int Hkv, int dh, float theta, bf16 *q, bf16 *k_cache,
+                                     bf16 *v_cache, int32_t *len, int cap, Paging pg, int32_t *status, cudaStream_t st,
+                                     long long *launches);
 cudaError_t launch_swiglu(const bf16 *gu, bf16 *out, int n, int F, cudaStream_t st, long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);

@@ -362,8 +362,15 @@ photon_status layer_step(photon_ctx *ctx, const photon_layer *L, const photon_la
     if (local && (cache->cap > c.P + c.C || cache->page_table)) return PHOTON_ERR_INVALID_ARG;
     photon_status s = photon_rmsnorm(ctx, x, L->g1, L->eps, sc->n, B, D, stream);
     if (s == PHOTON_OK) s = photon_linear(ctx, sc->n, L->wqkv, L->w_layout, nullptr, nullptr, sc->qkv, B, D, QKV, stream);
-    if (s == PHOTON_OK) s = photon_rope_split(ctx, sc->qkv, cache->len, B, L->theta, sc->q, sc->k_new, sc->v_new, stream);
-    if (s == PHOTON_OK) s = photon_kv_append(ctx, cache, sc->k_new, sc->v_new, nullptr, B, 1, stream);
+    if (s == PHOTON_OK) {
+        // split, rotation by the unit's length and the append in one kernel: k and v go straight into the cache rows
+        const cudaError_t e = launch_rope_split_append(
+            reinterpret_cast<const bf16 *>(sc->qkv), B, c.Hq, c.Hkv, c.dh, L->theta, reinterpret_cast<bf16 *>(sc->q),
+            reinterpret_cast<bf16 *>(cache->k), reinterpret_cast<bf16 *>(cache->v), cache->len, cache->cap,
+            Paging{cache->page_table, cache->page_rows, cache->pages_per_unit, cache->n_pages}, ctx->status,
+            static_cast<cudaStream_t>(stream), &ctx->launches);
+        if (e != cudaSuccess) s = PHOTON_ERR_CUDA;
+    }
     if (s == PHOTON_OK)
         s = local ? photon_chunk_attn(ctx, cache, sc->q, nullptr, sc->att, B, scale, stream)
                   : photon_coarse_attn(ctx, cache, sc->q, sc->att, nullptr, scale, stream);

@@ -20,9 +20,10 @@ def cfg_small(i, **kw):
     return wl.scaled(wl.CONFIGS[i], **kw)
 
 
-@pytest.mark.parametrize("idx", [0, 1, 4])
-def test_rope_split_matches_oracle(oracle, idx):
-    cfg = cfg_small(idx, B=37)
+@pytest.mark.parametrize("idx,n", [(0, 37), (1, 37), (4, 37), (1, 2999), (4, 1185)])
+def test_rope_split_matches_oracle(oracle, idx, n):
+    # 2999 and 1185 items: more than the CTAs that are resident at once, so a CTA takes several, unevenly
+    cfg = cfg_small(idx, B=n)
     Hq, Hkv, dh = cfg.Hq, cfg.Hkv, cfg.dh
     qkv = wl.normal_bf16(41, "qkv", (cfg.B, (Hq + 2 * Hkv) * dh))
     pos = (np.arange(cfg.B) * 229 % 8192).astype(np.int32)
@@ -96,15 +97,22 @@ def test_encoder_step_matches_oracle(oracle, idx, B, S, F):
         t = sc.tensors
         # the chain as a whole: intermediates and output against the oracle's chain, with the slack a
         # chain of bf16 roundings needs (each kernel by itself is held to the plain bar below)
-        for name in ("n", "qkv", "q", "k_new", "att", "h", "gu", "act"):
+        for name in ("n", "qkv", "q", "att", "h", "gu", "act"):
             key = "n2" if name == "n" else name                          # `n` holds the second normalisation at the end
             got, ref = host_f64(t[name]).reshape(B, -1), wl.bf16_bits_to_f64(want[key]).reshape(B, -1)
             assert_close_scaled(got, ref, f"encoder step {name}", slack=2.0)
-        # the appended rows are exactly the rotated key and the value the kernel produced
+        # the split writes k and v straight into the cache: the new row holds the rotated key and a bit copy
+        # of the value part of the fused projection, and no other row has changed
         hk, hv = host_bits(dk), host_bits(dv)
+        v_part = host_bits(t["qkv"]).reshape(B, -1)[:, (cfg.Hq + cfg.Hkv) * cfg.dh:].reshape(B, cfg.Hkv, cfg.dh)
+        new_k = np.stack([hk[u, :, lens[u]] for u in range(B)])
+        assert_close_scaled(wl.bf16_bits_to_f64(new_k).reshape(B, -1), wl.bf16_bits_to_f64(want["k_new"]).reshape(B, -1),
+                            "encoder step appended k", slack=2.0)
         for u in range(B):
-            assert np.array_equal(hk[u, :, lens[u]], host_bits(t["k_new"])[u])
-            assert np.array_equal(hv[u, :, lens[u]], host_bits(t["v_new"])[u])
+            assert np.array_equal(hv[u, :, lens[u]], v_part[u])
+            hk[u, :, lens[u]] = co["k"][u, :, lens[u]]
+            hv[u, :, lens[u]] = co["v"][u, :, lens[u]]
+        assert np.array_equal(hk, co["k"]) and np.array_equal(hv, co["v"])
     assert_close_scaled(host_f64(y), want["y"], f"encoder step cfg{idx}", slack=2.0)
 
 
@@ -171,9 +179,13 @@ def test_decoder_step_matches_oracle(oracle, idx, B, chunks_per_seq):
         ph.photon_decoder_step(c.h, layer, sc, x, kv, y, scale=scale)
         assert c.status() == 0
         assert np.array_equal(dl.cpu().numpy(), ch["len"] + 1)
-        for name in ("qkv", "q", "k_new", "att", "h", "act"):
+        for name in ("qkv", "q", "att", "h", "act"):
             got, ref = host_f64(sc.tensors[name]).reshape(Nc, -1), wl.bf16_bits_to_f64(want[name]).reshape(Nc, -1)
             assert_close_scaled(got, ref, f"decoder step {name}", slack=2.0)
+        hk = host_bits(dk)
+        new_k = np.stack([hk[u, :, ch["len"][u]] for u in range(Nc)])          # written by the split itself
+        assert_close_scaled(wl.bf16_bits_to_f64(new_k).reshape(Nc, -1), wl.bf16_bits_to_f64(want["k_new"]).reshape(Nc, -1),
+                            "decoder step appended k", slack=2.0)
     assert_close_scaled(host_f64(y), want["y"], f"decoder step cfg{idx}", slack=2.0)
 
 
@@ -257,10 +269,59 @@ def test_decoder_step_with_thousands_of_chunks_fuses_the_activation(oracle, layo
         n0 = ph.photon_launch_count(c.h)
         ph.photon_decoder_step(c.h, layer, sc, x, kv, y, scale=scale)
         assert c.status() == 0
-        assert ph.photon_launch_count(c.h) - n0 == 9                     # one launch fewer than the ten of a small batch
+        assert ph.photon_launch_count(c.h) - n0 == 8                     # one launch fewer than the nine of a small batch
         assert bool((sc.tensors["gu"] == 7.0).all())                     # the intermediate was not written
         assert_close_scaled(host_f64(sc.tensors["act"]), wl.bf16_bits_to_f64(want["act"]), "fused activation", slack=2.0)
     assert_close_scaled(host_f64(y), want["y"], "decoder step, 5120 chunks", slack=2.0)
+
+
+def test_encoder_step_on_a_full_cache_and_on_pages(oracle):
+    """The split appends by itself.  A unit whose cache is full sets the capacity bit and keeps its
+    rows and its length while the other units step; a paged cache gives the bits of the contiguous one."""
+    cfg = cfg_small(0, B=6, S=128)
+    F = 128
+    lw = wl.encoder_layer_inputs(cfg, F=F)
+    co = wl.coarse_inputs(cfg)
+    cap = co["k"].shape[2]
+    lens = np.array([5, cap, 17, cap - 1, 0, 64], dtype=np.int32)
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        W = {n: dev_bf16(lw[n]) for n in ("g1", "wqkv", "wo", "g2", "wgu", "wdown")}
+        layer = ph.make_layer(W["g1"], W["wqkv"], W["wo"], W["g2"], W["wgu"], W["wdown"], ph.PHOTON_W_IN_MAJOR, F)
+        sc = ph.make_layer_scratch(cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, F, "cuda", torch.bfloat16)
+        x = dev_bf16(lw["x"])
+        dk, dv, dl = dev_bf16(co["k"]), dev_bf16(co["v"]), dev_i32(lens)
+        y = torch.empty_like(x)
+        ph.photon_encoder_step(c.h, layer, sc, x, ph.make_kv(dk, dv, dl), y, scale=scale)
+        assert c.status() == ph.PHOTON_DEV_CAPACITY
+        grown = lens + 1
+        grown[1] = cap
+        assert np.array_equal(dl.cpu().numpy(), grown)
+        assert np.array_equal(host_bits(dk)[1], co["k"][1]) and np.array_equal(host_bits(dv)[1], co["v"][1])
+        # the same step on pages scattered over a pool (cap = 2 pages of 64 rows per unit), lengths that fit
+        assert cap == 128
+        fit = np.minimum(lens, cap - 1).astype(np.int32)
+        ck, cv, cl = dev_bf16(co["k"]), dev_bf16(co["v"]), dev_i32(fit)
+        y1 = torch.empty_like(x)
+        ph.photon_encoder_step(c.h, layer, sc, x, ph.make_kv(ck, cv, cl), y1, scale=scale)
+        n_pages = 2 * cfg.B + 3
+        ids = np.random.default_rng(5).permutation(n_pages)[: 2 * cfg.B].astype(np.int32).reshape(cfg.B, 2)
+        pk = np.full((n_pages, cfg.Hkv, 64, cfg.dh), 0x7FC1, dtype=np.uint16)
+        pv = pk.copy()
+        for u in range(cfg.B):
+            for r in range(2):
+                pk[ids[u, r]] = co["k"][u, :, 64 * r: 64 * r + 64]
+                pv[ids[u, r]] = co["v"][u, :, 64 * r: 64 * r + 64]
+        gk, gv, gl = dev_bf16(pk), dev_bf16(pv), dev_i32(fit)
+        y2 = torch.empty_like(x)
+        ph.photon_encoder_step(c.h, layer, sc, x, ph.make_kv(gk, gv, gl, page_table=dev_i32(ids)), y2, scale=scale)
+        assert c.status() == 0
+        assert np.array_equal(gl.cpu().numpy(), fit + 1) and np.array_equal(host_bits(y2), host_bits(y1))
+        hk, hv, fk, fv = host_bits(gk), host_bits(gv), host_bits(ck), host_bits(cv)
+        for u in range(cfg.B):
+            for r in range(2):
+                assert np.array_equal(hk[ids[u, r]], fk[u, :, 64 * r: 64 * r + 64])
+                assert np.array_equal(hv[ids[u, r]], fv[u, :, 64 * r: 64 * r + 64])
 
 
 def test_encoder_step_refuses_bad_arguments():
