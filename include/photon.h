@@ -27,6 +27,7 @@
 #ifndef PHOTON_H
 #define PHOTON_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -314,6 +315,27 @@ typedef struct {
 } photon_step_args;
 
 photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, photon_stream stream);
+
+/* The same step for a caller whose inputs and results live in HOST memory
+ * (the serving loop around Section 2.3.3: what a step consumes arrives from the
+ * host, what it produces goes back).  In stream order: in_bytes from host_in
+ * to dev_in, photon_decode_step(ctx, args, stream), out_bytes from dev_out to
+ * host_out, then the call waits for `stream`; when it returns PHOTON_OK
+ * host_out holds the results.
+ *   host_in, host_out  host pointers owned by the caller; page-locked memory
+ *                      makes the copies asynchronous to the host, pageable
+ *                      memory works and is staged by the driver.
+ *   dev_in, dev_out    device staging areas owned by the caller: the input
+ *                      pointers of `args` (k_new, v_new, queries, lengths ...)
+ *                      point into dev_in and its output pointers into dev_out,
+ *                      packed however the caller likes; the call only moves
+ *                      the bytes.  Either size may be 0 (that copy is skipped).
+ * NULL ctx or args, or a NULL pointer beside a non-zero size: INVALID_ARG,
+ * nothing is enqueued.  An error of the step itself is returned before the
+ * copy back is enqueued; the stream is then left as the step left it. */
+photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *args, const void *host_in,
+                                      void *dev_in, size_t in_bytes, const void *dev_out, void *host_out,
+                                      size_t out_bytes, photon_stream stream);
 
 /* Reads (and optionally clears) the device status word.  Synchronises the
  * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT also

@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_int64, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libphoton.so")
@@ -119,6 +119,9 @@ def load() -> ctypes.CDLL:
                       POINTER(photon_kv), c_void_p, c_float, c_void_p]
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
+    lib.photon_decode_step_host.restype = st
+    lib.photon_decode_step_host.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p, c_void_p, c_size_t, c_void_p,
+                                            c_void_p, c_size_t, c_void_p]
     lib.photon_device_status.restype = st
     lib.photon_device_status.argtypes = [c_void_p, POINTER(c_int32), c_int32]
     lib.photon_set_attention_ctas.restype = st
@@ -338,6 +341,34 @@ def make_step_args(coarse: photon_kv, k_new, v_new, q_coarse, out_coarse, scale_
 
 def photon_decode_step(ctx, args: photon_step_args, stream=None) -> None:
     _check(load().photon_decode_step(ctx, byref(args), _stream(stream)), "photon_decode_step")
+
+
+class HostIO:
+    """The four buffers of photon_decode_step_host, checked once: host_in / host_out are CPU uint8
+    tensors (pinned for asynchronous copies), dev_in / dev_out the device staging tensors that the
+    pointers of the step's arguments look into; `stream` is looked up once, here (None: the
+    stream that is current now).  Keeps the tensors alive."""
+
+    def __init__(self, host_in, dev_in, dev_out, host_out, stream=None):
+        for h, d in ((host_in, dev_in), (host_out, dev_out)):
+            if h.is_cuda or not d.is_cuda or not h.is_contiguous() or not d.is_contiguous():
+                raise ValueError("host tensors on the CPU, staging tensors on the device, both contiguous")
+            if h.numel() * h.element_size() != d.numel() * d.element_size():
+                raise ValueError("a host buffer and its staging area differ in size")
+        self._keep = (host_in, dev_in, dev_out, host_out)
+        self.argv = (c_void_p(host_in.data_ptr()), c_void_p(dev_in.data_ptr()),
+                     c_size_t(host_in.numel() * host_in.element_size()), c_void_p(dev_out.data_ptr()),
+                     c_void_p(host_out.data_ptr()), c_size_t(host_out.numel() * host_out.element_size()),
+                     _stream(stream))
+        self._call = load().photon_decode_step_host
+
+
+def photon_decode_step_host(ctx, args: photon_step_args, io: HostIO) -> None:
+    """Copy in, decode step, copy out on io's stream; returns once io's host_out holds the results.
+    Nothing is looked up per call: the host's time before the first copy is enqueued is the step's latency."""
+    rc = io._call(ctx, byref(args), *io.argv)
+    if rc != PHOTON_OK:
+        _check(rc, "photon_decode_step_host")
 
 
 def photon_device_status(ctx, clear=True) -> int:

@@ -1,4 +1,5 @@
 // C boundary: context management, argument validation, launch sequencing.
+#include <chrono>
 #include <algorithm>
 #include <cstdio>
 #include <new>
@@ -484,6 +485,36 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, pho
         s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, stream);
     }
     return s;
+}
+
+photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *args, const void *host_in,
+                                      void *dev_in, size_t in_bytes, const void *dev_out, void *host_out,
+                                      size_t out_bytes, photon_stream stream) {
+    if (!ctx || !args) return PHOTON_ERR_INVALID_ARG;
+    if ((in_bytes && (!host_in || !dev_in)) || (out_bytes && (!dev_out || !host_out))) return PHOTON_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (in_bytes && cudaMemcpyAsync(dev_in, host_in, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
+    if (in_bytes) {
+        // Measured: launches enqueued within a microsecond of the copy make the whole step finish about 5 us later
+        // than launches that follow 1.5 us behind it (a stream query in between does not help, a pause does).
+        const auto g0 = std::chrono::steady_clock::now();
+        while (std::chrono::steady_clock::now() - g0 < std::chrono::nanoseconds(1500)) {}
+    }
+    const photon_status s = photon_decode_step(ctx, args, stream);
+    if (s != PHOTON_OK) return s;
+    if (out_bytes && cudaMemcpyAsync(host_out, dev_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PHOTON_ERR_CUDA;
+    // a step is tens of microseconds: poll for its end (a blocking wait pays a wake-up of several microseconds),
+    // and hand over to the blocking wait when the stream turns out to hold much more work than that
+    const auto t0 = std::chrono::steady_clock::now();
+    cudaError_t e;
+    while ((e = cudaStreamQuery(st)) == cudaErrorNotReady)
+        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(2)) {
+            e = cudaStreamSynchronize(st);
+            break;
+        }
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 
 photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear) {

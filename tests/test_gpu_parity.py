@@ -494,6 +494,66 @@ def test_decode_step_chain_matches_oracle(oracle, idx, layout):
         assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_from_host_buffers(oracle, pinned):
+    """The step whose inputs (new K/V rows, both query tensors, the lengths) start in host memory and
+    whose results end there: one packed buffer each way through the staging areas the arguments look into."""
+    cfg = cfg_small(1, B=24, S=300)
+    s = wl.step_inputs(cfg, poison=True)
+    co, cv, chk = s["coarse"], s["converter"], s["chunks"]
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        d, dc = coarse_to_dev(co), chunks_to_dev(chk)
+        lens0 = co["len"].copy()                                             # before the append
+        ins = [co["k_new"], co["v_new"], co["q"], chk["q"], lens0]
+        offs, total = [], 0
+        for a in ins:
+            offs.append(total)
+            total += (a.nbytes + 255) // 256 * 256
+        h_in = torch.zeros(total, dtype=torch.uint8)
+        for a, o in zip(ins, offs):
+            h_in[o:o + a.nbytes] = torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1))
+        d_in = torch.full((total,), 0xEE, dtype=torch.uint8, device="cuda")
+
+        def view(j, like, dtype):
+            return d_in[offs[j]:offs[j] + ins[j].nbytes].view(dtype).view(like.shape)
+        k_new, v_new, q, qc = (view(j, t, torch.bfloat16) for j, t in enumerate((d["k_new"], d["v_new"], d["q"], dc["q"])))
+        ln = view(4, d["len"], torch.int32)
+        n_out, n_oc = d["q"].numel() * 2, dc["q"].numel() * 2
+        d_out = torch.full((n_out + n_oc,), 0xEE, dtype=torch.uint8, device="cuda")
+        h_out = torch.zeros(n_out + n_oc, dtype=torch.uint8)
+        if pinned:
+            h_in, h_out = h_in.pin_memory(), h_out.pin_memory()
+        out = d_out[:n_out].view(torch.bfloat16).view(d["q"].shape)
+        oc = d_out[n_out:].view(torch.bfloat16).view(dc["q"].shape)
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        # the cache as it was before the newest row: the lengths come from the host with everything else
+        co0 = wl.coarse_inputs(cfg, poison=True)
+        kv = ph.make_kv(dev_bf16(co0["k"]), dev_bf16(co0["v"]), ln, max_len=cfg.S)
+        args = ph.make_step_args(kv, k_new, v_new, q, out, scale, dev_bf16(cv["w_in_major"]), ph.PHOTON_W_IN_MAJOR, U,
+                                 cfg.B, chunks=dc["kv"], q_chunk=qc, out_chunk=oc, Nc=cfg.Nc, scale_chunk=scale)
+        ph.photon_decode_step_host(c.h, args, ph.HostIO(h_in, d_in, d_out, h_out))      # returns with the results on the host
+        got = h_out.numpy().copy()
+        assert c.status() == 0
+        assert np.array_equal(ln.cpu().numpy(), lens0 + 1)
+        # the same step from device tensors gives the same bits
+        out2, oc2, U2 = torch.empty_like(d["q"]), torch.empty_like(dc["q"]), torch.empty_like(U)
+        args2 = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out2, scale, dev_bf16(cv["w_in_major"]),
+                                  ph.PHOTON_W_IN_MAJOR, U2, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc2,
+                                  Nc=cfg.Nc, scale_chunk=scale)
+        ph.photon_decode_step(c.h, args2)
+        assert np.array_equal(got[:n_out].view(np.uint16).reshape(out2.shape), host_bits(out2))
+        assert np.array_equal(got[n_out:].view(np.uint16).reshape(oc2.shape), host_bits(oc2))
+        n0 = ph.photon_launch_count(c.h)
+        assert ph.load().photon_decode_step_host(c.h, None, None, None, 0, None, None, 0, None) == ph.PHOTON_ERR_INVALID_ARG
+        with pytest.raises(ValueError):
+            ph.HostIO(h_in, d_in, d_out, h_out[:-1])
+        assert ph.photon_launch_count(c.h) == n0
+    r = oracle.decode_step(co, cv, chk, scale, scale, chain=True, n_threads=NT)
+    assert_close(wl.bf16_bits_to_f64(got[:n_out].view(np.uint16)).reshape(r["out"].shape), r["out"], "host step: coarse out")
+    assert_close(wl.bf16_bits_to_f64(got[n_out:].view(np.uint16)).reshape(r["chunk_out"].shape), r["chunk_out"], "host step: chunk out")
+
+
 def test_decode_step_with_given_x_and_no_chunks(oracle):
     cfg = wl.CONFIGS[0]
     s = wl.step_inputs(cfg)
