@@ -704,7 +704,7 @@ def run_gpu(args, cfg) -> None:
             total += (t.numel() * t.element_size() + 255) // 256 * 256
         return offs, total
 
-    in_src = [k_new, v_new, q, qc, lens0[0]]
+    in_src = [k_new, v_new, q, lens0[0], qc]              # the chunk attention's input last: it may travel apart
     in_offs, in_total = pack(in_src)
     h_in = torch.empty(in_total, dtype=torch.uint8).pin_memory()
     d_in = torch.empty(in_total, dtype=torch.uint8, device=dev)
@@ -713,7 +713,7 @@ def run_gpu(args, cfg) -> None:
         nb = t.numel() * t.element_size()
         h_in[o:o + nb].copy_(t.cpu().contiguous().view(-1).view(torch.uint8))
         views.append(d_in[o:o + nb].view(t.dtype).view(t.shape))
-    e_k_new, e_v_new, e_q, e_qc, e_len = views
+    e_k_new, e_v_new, e_q, e_len, e_qc = views
     out_src = [reps[0]["out"], reps[0]["oc"]]
     out_offs, out_total = pack(out_src)
     d_out = torch.empty(out_total, dtype=torch.uint8, device=dev)
@@ -728,7 +728,7 @@ def run_gpu(args, cfg) -> None:
         e2e_args.append(ph.make_step_args(kv_e, e_k_new, e_v_new, e_q, e_out, scale, t["w"], layout, t["U"], cfg.B,
                                           chunks=t["ckv"], q_chunk=e_qc, out_chunk=e_oc, Nc=cfg.Nc, scale_chunk=scale))
 
-    host_io = ph.HostIO(h_in, d_in, d_out, h_out)
+    host_io = ph.HostIO(h_in, d_in, d_out, h_out, in_split=in_offs[4], out_split=out_offs[1])
 
     def e2e_step(i):
         # one call of the library: host -> staging, the decode step, staging -> host, wait for the stream
@@ -759,7 +759,7 @@ def run_gpu(args, cfg) -> None:
                        w_layout=args.layout),
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": n_e2e, "note": "photon_decode_step_host: one pinned host buffer -> device (new K/V row, queries, lengths), decode step, both outputs -> host, wait, every step"},
+                "steps": n_e2e, "note": "photon_decode_step_host: one pinned host buffer -> device (new K/V row, queries, lengths), decode step, both outputs -> host, wait, every step; the chunk attention's query and output cross the bus beside the coarse part where that attention runs on the side stream"},
         "gpu_launches": launches_per_step * K,
         "roofline": roofline,
         "us_per_step": sec_max * 1e6 / K,

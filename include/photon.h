@@ -318,24 +318,35 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, 
 
 /* The same step for a caller whose inputs and results live in HOST memory
  * (the serving loop around Section 2.3.3: what a step consumes arrives from the
- * host, what it produces goes back).  In stream order: in_bytes from host_in
- * to dev_in, photon_decode_step(ctx, args, stream), out_bytes from dev_out to
- * host_out, then the call waits for `stream`; when it returns PHOTON_OK
- * host_out holds the results.
+ * host, what it produces goes back).  in_bytes travel from host_in to dev_in,
+ * the step runs, out_bytes travel from dev_out to host_out, and the call waits
+ * for `stream`; when it returns PHOTON_OK host_out holds the results.
  *   host_in, host_out  host pointers owned by the caller; page-locked memory
  *                      makes the copies asynchronous to the host, pageable
  *                      memory works and is staged by the driver.
  *   dev_in, dev_out    device staging areas owned by the caller: the input
  *                      pointers of `args` (k_new, v_new, queries, lengths ...)
- *                      point into dev_in and its output pointers into dev_out,
- *                      packed however the caller likes; the call only moves
- *                      the bytes.  Either size may be 0 (that copy is skipped).
- * NULL ctx or args, or a NULL pointer beside a non-zero size: INVALID_ARG,
- * nothing is enqueued.  An error of the step itself is returned before the
- * copy back is enqueued; the stream is then left as the step left it. */
+ *                      point into dev_in and its output pointers into dev_out;
+ *                      the call only moves the bytes.  Either size may be 0.
+ *   in_split           bytes [0, in_split) of the input are what the append,
+ *                      the coarse attention and the converter read; the rest is
+ *                      read by the chunk attention only (q_chunk, slot).
+ *   out_split          bytes [0, out_split) of the output are written by the
+ *                      coarse attention (out_coarse, lse_coarse); the rest by the
+ *                      chunk attention (out_chunk).
+ * With in_split == in_bytes and out_split == out_bytes everything is copied in
+ * before the step and out after it.  Otherwise, when the chunk attention runs
+ * on the context's side stream (see photon_decode_step), the two parts of a
+ * buffer travel apart: the chunk attention's inputs cross the bus while the
+ * append and the coarse attention already run, its results leave when it ends,
+ * and the coarse results leave beside the converter.  A buffer laid out
+ * otherwise than declared gives stale inputs or results: the call cannot tell.
+ * NULL ctx or args, a NULL pointer beside a non-zero size, or a split beyond
+ * its size: INVALID_ARG, nothing is enqueued.  An error of the step itself is
+ * returned without waiting; the stream is then left as the step left it. */
 photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *args, const void *host_in,
-                                      void *dev_in, size_t in_bytes, const void *dev_out, void *host_out,
-                                      size_t out_bytes, photon_stream stream);
+                                      void *dev_in, size_t in_bytes, size_t in_split, const void *dev_out,
+                                      void *host_out, size_t out_bytes, size_t out_split, photon_stream stream);
 
 /* Reads (and optionally clears) the device status word.  Synchronises the
  * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT also

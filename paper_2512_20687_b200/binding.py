@@ -120,8 +120,8 @@ def load() -> ctypes.CDLL:
     lib.photon_decode_step.restype = st
     lib.photon_decode_step.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p]
     lib.photon_decode_step_host.restype = st
-    lib.photon_decode_step_host.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p, c_void_p, c_size_t, c_void_p,
-                                            c_void_p, c_size_t, c_void_p]
+    lib.photon_decode_step_host.argtypes = [c_void_p, POINTER(photon_step_args), c_void_p, c_void_p, c_size_t, c_size_t,
+                                            c_void_p, c_void_p, c_size_t, c_size_t, c_void_p]
     lib.photon_device_status.restype = st
     lib.photon_device_status.argtypes = [c_void_p, POINTER(c_int32), c_int32]
     lib.photon_set_attention_ctas.restype = st
@@ -347,18 +347,21 @@ class HostIO:
     """The four buffers of photon_decode_step_host, checked once: host_in / host_out are CPU uint8
     tensors (pinned for asynchronous copies), dev_in / dev_out the device staging tensors that the
     pointers of the step's arguments look into; `stream` is looked up once, here (None: the
-    stream that is current now).  Keeps the tensors alive."""
+    stream that is current now).  in_split / out_split: the leading bytes that belong to the coarse
+    part of the step, the rest being the chunk attention's (None: no split, everything is copied
+    before and after the step).  Keeps the tensors alive."""
 
-    def __init__(self, host_in, dev_in, dev_out, host_out, stream=None):
+    def __init__(self, host_in, dev_in, dev_out, host_out, stream=None, in_split=None, out_split=None):
         for h, d in ((host_in, dev_in), (host_out, dev_out)):
             if h.is_cuda or not d.is_cuda or not h.is_contiguous() or not d.is_contiguous():
                 raise ValueError("host tensors on the CPU, staging tensors on the device, both contiguous")
             if h.numel() * h.element_size() != d.numel() * d.element_size():
                 raise ValueError("a host buffer and its staging area differ in size")
         self._keep = (host_in, dev_in, dev_out, host_out)
-        self.argv = (c_void_p(host_in.data_ptr()), c_void_p(dev_in.data_ptr()),
-                     c_size_t(host_in.numel() * host_in.element_size()), c_void_p(dev_out.data_ptr()),
-                     c_void_p(host_out.data_ptr()), c_size_t(host_out.numel() * host_out.element_size()),
+        n_in, n_out = host_in.numel() * host_in.element_size(), host_out.numel() * host_out.element_size()
+        self.argv = (c_void_p(host_in.data_ptr()), c_void_p(dev_in.data_ptr()), c_size_t(n_in),
+                     c_size_t(n_in if in_split is None else in_split), c_void_p(dev_out.data_ptr()),
+                     c_void_p(host_out.data_ptr()), c_size_t(n_out), c_size_t(n_out if out_split is None else out_split),
                      _stream(stream))
         self._call = load().photon_decode_step_host
 

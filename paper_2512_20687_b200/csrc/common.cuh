@@ -42,6 +42,8 @@ struct photon_ctx {
     long long launches;
     cudaStream_t side;       // lowest-priority stream for the chunk attention of a decode step
     cudaEvent_t ev_fork, ev_join;
+    cudaStream_t copy;       // carries the coarse results to the host beside the converter (photon_decode_step_host)
+    cudaEvent_t ev_mid, ev_copy;
     TmapCache tmaps;
 };
 

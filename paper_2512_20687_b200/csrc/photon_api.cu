@@ -147,7 +147,10 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, lo) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->copy, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_mid, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_copy, cudaEventDisableTiming) != cudaSuccess) {
         photon_destroy(ctx);
         cudaGetLastError();
         return PHOTON_ERR_CUDA;
@@ -165,6 +168,9 @@ photon_status photon_destroy(photon_ctx *ctx) {
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->side) cudaStreamDestroy(ctx->side);
+    if (ctx->ev_mid) cudaEventDestroy(ctx->ev_mid);
+    if (ctx->ev_copy) cudaEventDestroy(ctx->ev_copy);
+    if (ctx->copy) cudaStreamDestroy(ctx->copy);
     delete ctx;
     return PHOTON_OK;
 }
@@ -430,7 +436,26 @@ photon_status photon_decoder_step(photon_ctx *ctx, const photon_layer *layer, co
     return layer_step(ctx, layer, scratch, x, chunks, y, scale, true, stream);
 }
 
-photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {
+namespace {
+// Host buffers of a step: [0, in_split) of the input is what the coarse part reads, the rest what only the
+// chunk attention reads; [0, out_split) of the output is what the coarse part writes, the rest the chunk attention's.
+struct HostPlan {
+    const char *host_in;
+    char *dev_in;
+    size_t in_bytes, in_split;
+    const char *dev_out;
+    char *host_out;
+    size_t out_bytes, out_split;
+};
+
+bool copy_in(const HostPlan *hp, size_t from, size_t to, cudaStream_t st) {
+    return to <= from || cudaMemcpyAsync(hp->dev_in + from, hp->host_in + from, to - from, cudaMemcpyHostToDevice, st) == cudaSuccess;
+}
+bool copy_out(const HostPlan *hp, size_t from, size_t to, cudaStream_t st) {
+    return to <= from || cudaMemcpyAsync(hp->host_out + from, hp->dev_out + from, to - from, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+}
+
+photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_stream stream, const HostPlan *hp) {
     if (!ctx || !a || !a->coarse) return PHOTON_ERR_INVALID_ARG;
     const photon_config &c = ctx->cfg;
     const bool chain = (a->x == nullptr);
@@ -463,10 +488,26 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, pho
     const bool beside = a->Nc > 0 &&
                         (size_t)a->Nc * c.Hkv * a->chunks->cap * c.dh * 4 <= (size_t(32) << 20);
     photon_status s = PHOTON_OK;
+    // With host buffers and the chunk attention on its own stream the two halves of either buffer travel apart: the
+    // chunk attention's inputs follow the coarse part's over the bus while the append and the coarse attention already
+    // run, and each part's results leave as soon as that part ends, the coarse ones beside the converter.
+    const bool apart = hp && beside && (hp->in_split < hp->in_bytes || hp->out_split < hp->out_bytes);
+    if (hp) {
+        if (!copy_in(hp, 0, apart ? hp->in_split : hp->in_bytes, st)) return PHOTON_ERR_CUDA;
+        if (hp->in_bytes) {
+            // Measured: launches enqueued within a microsecond of the copy make the whole step finish about 5 us later
+            // than launches that follow 1.5 us behind it (a stream query in between does not help, a pause does).
+            const auto g0 = std::chrono::steady_clock::now();
+            while (std::chrono::steady_clock::now() - g0 < std::chrono::nanoseconds(1500)) {}
+        }
+    }
     if (beside) {
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
             return PHOTON_ERR_CUDA;
-        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, ctx->side);
+        if (apart && !copy_in(hp, hp->in_split, hp->in_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
+        if (s == PHOTON_OK)
+            s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, ctx->side);
+        if (s == PHOTON_OK && apart && !copy_out(hp, hp->out_split, hp->out_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
         if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return PHOTON_ERR_CUDA;
         if (s != PHOTON_OK) { cudaStreamWaitEvent(st, ctx->ev_join, 0); return s; }
     }
@@ -477,6 +518,16 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, pho
         s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse, a->scale_coarse, stream);
     if (s == PHOTON_OK && a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;
+    bool copying = false;
+    if (s == PHOTON_OK && apart && hp->out_split > 0) {
+        if (cudaEventRecord(ctx->ev_mid, st) != cudaSuccess || cudaStreamWaitEvent(ctx->copy, ctx->ev_mid, 0) != cudaSuccess)
+            s = PHOTON_ERR_CUDA;
+        else {
+            copying = true;
+            if (!copy_out(hp, 0, hp->out_split, ctx->copy)) s = PHOTON_ERR_CUDA;
+            if (cudaEventRecord(ctx->ev_copy, ctx->copy) != cudaSuccess) s = PHOTON_ERR_CUDA;
+        }
+    }
     if (s == PHOTON_OK)
         s = photon_converter(ctx, chain ? a->out_coarse : a->x, a->w, a->w_layout, a->bias, a->U, a->B, stream);
     if (beside) {
@@ -484,27 +535,27 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, pho
     } else if (s == PHOTON_OK && a->Nc > 0) {
         s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, stream);
     }
+    if (copying && cudaStreamWaitEvent(st, ctx->ev_copy, 0) != cudaSuccess && s == PHOTON_OK) s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK && hp && !apart && !copy_out(hp, 0, hp->out_bytes, st)) s = PHOTON_ERR_CUDA;
     return s;
+}
+}  // namespace
+
+photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *a, photon_stream stream) {
+    return step_impl(ctx, a, stream, nullptr);
 }
 
 photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *args, const void *host_in,
-                                      void *dev_in, size_t in_bytes, const void *dev_out, void *host_out,
-                                      size_t out_bytes, photon_stream stream) {
+                                      void *dev_in, size_t in_bytes, size_t in_split, const void *dev_out,
+                                      void *host_out, size_t out_bytes, size_t out_split, photon_stream stream) {
     if (!ctx || !args) return PHOTON_ERR_INVALID_ARG;
     if ((in_bytes && (!host_in || !dev_in)) || (out_bytes && (!dev_out || !host_out))) return PHOTON_ERR_INVALID_ARG;
+    if (in_split > in_bytes || out_split > out_bytes) return PHOTON_ERR_INVALID_ARG;
+    const HostPlan hp{static_cast<const char *>(host_in), static_cast<char *>(dev_in), in_bytes, in_split,
+                      static_cast<const char *>(dev_out), static_cast<char *>(host_out), out_bytes, out_split};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (in_bytes && cudaMemcpyAsync(dev_in, host_in, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return PHOTON_ERR_CUDA;
-    if (in_bytes) {
-        // Measured: launches enqueued within a microsecond of the copy make the whole step finish about 5 us later
-        // than launches that follow 1.5 us behind it (a stream query in between does not help, a pause does).
-        const auto g0 = std::chrono::steady_clock::now();
-        while (std::chrono::steady_clock::now() - g0 < std::chrono::nanoseconds(1500)) {}
-    }
-    const photon_status s = photon_decode_step(ctx, args, stream);
+    const photon_status s = step_impl(ctx, args, stream, &hp);
     if (s != PHOTON_OK) return s;
-    if (out_bytes && cudaMemcpyAsync(host_out, dev_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return PHOTON_ERR_CUDA;
     // a step is tens of microseconds: poll for its end (a blocking wait pays a wake-up of several microseconds),
     // and hand over to the blocking wait when the stream turns out to hold much more work than that
     const auto t0 = std::chrono::steady_clock::now();

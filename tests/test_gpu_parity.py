@@ -494,10 +494,11 @@ def test_decode_step_chain_matches_oracle(oracle, idx, layout):
         assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_decode_step_from_host_buffers(oracle, pinned):
+@pytest.mark.parametrize("pinned,split", [(True, True), (True, False), (False, True), (False, False)])
+def test_decode_step_from_host_buffers(oracle, pinned, split):
     """The step whose inputs (new K/V rows, both query tensors, the lengths) start in host memory and
-    whose results end there: one packed buffer each way through the staging areas the arguments look into."""
+    whose results end there: one packed buffer each way through the staging areas the arguments look into;
+    with the split declared, the chunk attention's half of either buffer travels beside the coarse part."""
     cfg = cfg_small(1, B=24, S=300)
     s = wl.step_inputs(cfg, poison=True)
     co, cv, chk = s["coarse"], s["converter"], s["chunks"]
@@ -505,7 +506,7 @@ def test_decode_step_from_host_buffers(oracle, pinned):
     with Ctx(cfg) as c:
         d, dc = coarse_to_dev(co), chunks_to_dev(chk)
         lens0 = co["len"].copy()                                             # before the append
-        ins = [co["k_new"], co["v_new"], co["q"], chk["q"], lens0]
+        ins = [co["k_new"], co["v_new"], co["q"], lens0, chk["q"]]              # the chunk attention's input last
         offs, total = [], 0
         for a in ins:
             offs.append(total)
@@ -517,8 +518,8 @@ def test_decode_step_from_host_buffers(oracle, pinned):
 
         def view(j, like, dtype):
             return d_in[offs[j]:offs[j] + ins[j].nbytes].view(dtype).view(like.shape)
-        k_new, v_new, q, qc = (view(j, t, torch.bfloat16) for j, t in enumerate((d["k_new"], d["v_new"], d["q"], dc["q"])))
-        ln = view(4, d["len"], torch.int32)
+        k_new, v_new, q = (view(j, t, torch.bfloat16) for j, t in enumerate((d["k_new"], d["v_new"], d["q"])))
+        ln, qc = view(3, d["len"], torch.int32), view(4, dc["q"], torch.bfloat16)
         n_out, n_oc = d["q"].numel() * 2, dc["q"].numel() * 2
         d_out = torch.full((n_out + n_oc,), 0xEE, dtype=torch.uint8, device="cuda")
         h_out = torch.zeros(n_out + n_oc, dtype=torch.uint8)
@@ -532,7 +533,8 @@ def test_decode_step_from_host_buffers(oracle, pinned):
         kv = ph.make_kv(dev_bf16(co0["k"]), dev_bf16(co0["v"]), ln, max_len=cfg.S)
         args = ph.make_step_args(kv, k_new, v_new, q, out, scale, dev_bf16(cv["w_in_major"]), ph.PHOTON_W_IN_MAJOR, U,
                                  cfg.B, chunks=dc["kv"], q_chunk=qc, out_chunk=oc, Nc=cfg.Nc, scale_chunk=scale)
-        ph.photon_decode_step_host(c.h, args, ph.HostIO(h_in, d_in, d_out, h_out))      # returns with the results on the host
+        io = ph.HostIO(h_in, d_in, d_out, h_out, in_split=offs[4], out_split=n_out) if split else ph.HostIO(h_in, d_in, d_out, h_out)
+        ph.photon_decode_step_host(c.h, args, io)                              # returns with the results on the host
         got = h_out.numpy().copy()
         assert c.status() == 0
         assert np.array_equal(ln.cpu().numpy(), lens0 + 1)
@@ -545,7 +547,10 @@ def test_decode_step_from_host_buffers(oracle, pinned):
         assert np.array_equal(got[:n_out].view(np.uint16).reshape(out2.shape), host_bits(out2))
         assert np.array_equal(got[n_out:].view(np.uint16).reshape(oc2.shape), host_bits(oc2))
         n0 = ph.photon_launch_count(c.h)
-        assert ph.load().photon_decode_step_host(c.h, None, None, None, 0, None, None, 0, None) == ph.PHOTON_ERR_INVALID_ARG
+        assert ph.load().photon_decode_step_host(c.h, None, None, None, 0, 0, None, None, 0, 0, None) == ph.PHOTON_ERR_INVALID_ARG
+        with pytest.raises(ph.PhotonError) as e:                               # a split beyond the buffer
+            ph.photon_decode_step_host(c.h, args, ph.HostIO(h_in, d_in, d_out, h_out, in_split=total + 1))
+        assert e.value.code == ph.PHOTON_ERR_INVALID_ARG
         with pytest.raises(ValueError):
             ph.HostIO(h_in, d_in, d_out, h_out[:-1])
         assert ph.photon_launch_count(c.h) == n0
