@@ -448,6 +448,27 @@ struct HostPlan {
     size_t out_bytes, out_split;
 };
 
+// The address under which kernels can reach page-locked, mapped host memory; nullptr for any other memory.
+// Looked up once per buffer and remembered in the context.
+char *device_alias(photon_ctx *ctx, int which, const void *host) {
+    if (ctx->io_host[which] != host) {
+        cudaPointerAttributes at{};
+        char *alias = nullptr;
+        if (cudaPointerGetAttributes(&at, host) == cudaSuccess && at.type == cudaMemoryTypeHost)
+            alias = static_cast<char *>(at.devicePointer);
+        else
+            cudaGetLastError();
+        ctx->io_host[which] = host;
+        ctx->io_alias[which] = alias;
+    }
+    return ctx->io_alias[which];
+}
+
+bool inside(const void *p, size_t n, const char *base, size_t from, size_t to) {
+    const char *c = static_cast<const char *>(p);
+    return c >= base + from && c + n <= base + to;
+}
+
 bool copy_in(const HostPlan *hp, size_t from, size_t to, cudaStream_t st) {
     return to <= from || cudaMemcpyAsync(hp->dev_in + from, hp->host_in + from, to - from, cudaMemcpyHostToDevice, st) == cudaSuccess;
 }
@@ -504,10 +525,32 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     if (beside) {
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
             return PHOTON_ERR_CUDA;
-        if (apart && !copy_in(hp, hp->in_split, hp->in_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
+        // Where both host buffers are mapped into the device and the chunk attention's arrays lie wholly in its
+        // halves of the staging areas, the kernel reads its queries from and writes its results to the host buffers
+        // themselves: no copy, and no hand-over between the copy engines and the SMs, on that side of the step.
+        const photon_bf16 *q_chunk = a->q_chunk;
+        const int32_t *slot = a->slot;
+        photon_bf16 *out_chunk = a->out_chunk;
+        bool direct = false;
+        if (apart) {
+            const size_t qb = (size_t)a->Nc * c.Hq * c.dh * sizeof(photon_bf16), sb = (size_t)a->Nc * sizeof(int32_t);
+            const bool slot_in = slot && inside(slot, sb, hp->dev_in, hp->in_split, hp->in_bytes);
+            const bool slot_off = !slot || (const char *)slot + sb <= hp->dev_in || (const char *)slot >= hp->dev_in + hp->in_bytes;
+            if (inside(q_chunk, qb, hp->dev_in, hp->in_split, hp->in_bytes) &&
+                inside(out_chunk, qb, hp->dev_out, hp->out_split, hp->out_bytes) && (slot_in || slot_off)) {
+                char *in_alias = device_alias(ctx, 0, hp->host_in), *out_alias = device_alias(ctx, 1, hp->host_out);
+                if (in_alias && out_alias) {
+                    direct = true;
+                    q_chunk = reinterpret_cast<const photon_bf16 *>(in_alias + ((const char *)q_chunk - hp->dev_in));
+                    out_chunk = reinterpret_cast<photon_bf16 *>(out_alias + ((const char *)out_chunk - hp->dev_out));
+                    if (slot_in) slot = reinterpret_cast<const int32_t *>(in_alias + ((const char *)slot - hp->dev_in));
+                }
+            }
+        }
+        if (apart && !direct && !copy_in(hp, hp->in_split, hp->in_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
         if (s == PHOTON_OK)
-            s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, ctx->side);
-        if (s == PHOTON_OK && apart && !copy_out(hp, hp->out_split, hp->out_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
+            s = photon_chunk_attn(ctx, a->chunks, q_chunk, slot, out_chunk, a->Nc, a->scale_chunk, ctx->side);
+        if (s == PHOTON_OK && apart && !direct && !copy_out(hp, hp->out_split, hp->out_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
         if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return PHOTON_ERR_CUDA;
         if (s != PHOTON_OK) { cudaStreamWaitEvent(st, ctx->ev_join, 0); return s; }
     }

@@ -537,6 +537,10 @@ def test_decode_step_from_host_buffers(oracle, pinned, split):
         ph.photon_decode_step_host(c.h, args, io)                              # returns with the results on the host
         got = h_out.numpy().copy()
         assert c.status() == 0
+        # page-locked buffers with the split declared: the chunk attention wrote to the host buffer itself and its
+        # half of the staging area was never touched; in every other case the results passed through it
+        staged = d_out[n_out:].cpu().numpy()
+        assert bool((staged == 0xEE).all()) if (pinned and split) else np.array_equal(staged, got[n_out:])
         assert np.array_equal(ln.cpu().numpy(), lens0 + 1)
         # the same step from device tensors gives the same bits
         out2, oc2, U2 = torch.empty_like(d["q"]), torch.empty_like(dc["q"]), torch.empty_like(U)
