@@ -509,12 +509,35 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     const bool beside = a->Nc > 0 &&
                         (size_t)a->Nc * c.Hkv * a->chunks->cap * c.dh * 4 <= (size_t(32) << 20);
     photon_status s = PHOTON_OK;
-    // With host buffers and the chunk attention on its own stream the two halves of either buffer travel apart: the
-    // chunk attention's inputs follow the coarse part's over the bus while the append and the coarse attention already
-    // run, and each part's results leave as soon as that part ends, the coarse ones beside the converter.
-    const bool apart = hp && beside && (hp->in_split < hp->in_bytes || hp->out_split < hp->out_bytes);
+    // With host buffers and a declared split the two halves of either buffer travel apart.  Where both host buffers are
+    // mapped into the device and the chunk attention's arrays lie wholly in its halves of the staging areas, that
+    // kernel reads its queries from and writes its results to the host buffers themselves: no copy, and no hand-over
+    // between the copy engines and the SMs, for those bytes (direct).  Otherwise, with the chunk attention on its own
+    // stream, its inputs follow the coarse part's over the bus while the append and the coarse attention already run
+    // and its results leave when it ends.  The coarse results leave beside the converter in both cases (apart).
+    const bool split = hp && a->Nc > 0 && (hp->in_split < hp->in_bytes || hp->out_split < hp->out_bytes);
+    const bool apart = split && beside;
+    const photon_bf16 *q_chunk = a->q_chunk;
+    const int32_t *slot = a->slot;
+    photon_bf16 *out_chunk = a->out_chunk;
+    bool direct = false;
+    if (split) {
+        const size_t qb = (size_t)a->Nc * c.Hq * c.dh * sizeof(photon_bf16), sb = (size_t)a->Nc * sizeof(int32_t);
+        const bool slot_in = slot && inside(slot, sb, hp->dev_in, hp->in_split, hp->in_bytes);
+        const bool slot_off = !slot || (const char *)slot + sb <= hp->dev_in || (const char *)slot >= hp->dev_in + hp->in_bytes;
+        if (inside(q_chunk, qb, hp->dev_in, hp->in_split, hp->in_bytes) &&
+            inside(out_chunk, qb, hp->dev_out, hp->out_split, hp->out_bytes) && (slot_in || slot_off)) {
+            char *in_alias = device_alias(ctx, 0, hp->host_in), *out_alias = device_alias(ctx, 1, hp->host_out);
+            if (in_alias && out_alias) {
+                direct = true;
+                q_chunk = reinterpret_cast<const photon_bf16 *>(in_alias + ((const char *)q_chunk - hp->dev_in));
+                out_chunk = reinterpret_cast<photon_bf16 *>(out_alias + ((const char *)out_chunk - hp->dev_out));
+                if (slot_in) slot = reinterpret_cast<const int32_t *>(in_alias + ((const char *)slot - hp->dev_in));
+            }
+        }
+    }
     if (hp) {
-        if (!copy_in(hp, 0, apart ? hp->in_split : hp->in_bytes, st)) return PHOTON_ERR_CUDA;
+        if (!copy_in(hp, 0, apart || direct ? hp->in_split : hp->in_bytes, st)) return PHOTON_ERR_CUDA;
         if (hp->in_bytes) {
             // Measured: launches enqueued within a microsecond of the copy make the whole step finish about 5 us later
             // than launches that follow 1.5 us behind it (a stream query in between does not help, a pause does).
@@ -525,28 +548,6 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     if (beside) {
         if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
             return PHOTON_ERR_CUDA;
-        // Where both host buffers are mapped into the device and the chunk attention's arrays lie wholly in its
-        // halves of the staging areas, the kernel reads its queries from and writes its results to the host buffers
-        // themselves: no copy, and no hand-over between the copy engines and the SMs, on that side of the step.
-        const photon_bf16 *q_chunk = a->q_chunk;
-        const int32_t *slot = a->slot;
-        photon_bf16 *out_chunk = a->out_chunk;
-        bool direct = false;
-        if (apart) {
-            const size_t qb = (size_t)a->Nc * c.Hq * c.dh * sizeof(photon_bf16), sb = (size_t)a->Nc * sizeof(int32_t);
-            const bool slot_in = slot && inside(slot, sb, hp->dev_in, hp->in_split, hp->in_bytes);
-            const bool slot_off = !slot || (const char *)slot + sb <= hp->dev_in || (const char *)slot >= hp->dev_in + hp->in_bytes;
-            if (inside(q_chunk, qb, hp->dev_in, hp->in_split, hp->in_bytes) &&
-                inside(out_chunk, qb, hp->dev_out, hp->out_split, hp->out_bytes) && (slot_in || slot_off)) {
-                char *in_alias = device_alias(ctx, 0, hp->host_in), *out_alias = device_alias(ctx, 1, hp->host_out);
-                if (in_alias && out_alias) {
-                    direct = true;
-                    q_chunk = reinterpret_cast<const photon_bf16 *>(in_alias + ((const char *)q_chunk - hp->dev_in));
-                    out_chunk = reinterpret_cast<photon_bf16 *>(out_alias + ((const char *)out_chunk - hp->dev_out));
-                    if (slot_in) slot = reinterpret_cast<const int32_t *>(in_alias + ((const char *)slot - hp->dev_in));
-                }
-            }
-        }
         if (apart && !direct && !copy_in(hp, hp->in_split, hp->in_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
         if (s == PHOTON_OK)
             s = photon_chunk_attn(ctx, a->chunks, q_chunk, slot, out_chunk, a->Nc, a->scale_chunk, ctx->side);
@@ -562,7 +563,7 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     if (s == PHOTON_OK && a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;
     bool copying = false;
-    if (s == PHOTON_OK && apart && hp->out_split > 0) {
+    if (s == PHOTON_OK && (apart || direct) && hp->out_split > 0) {
         if (cudaEventRecord(ctx->ev_mid, st) != cudaSuccess || cudaStreamWaitEvent(ctx->copy, ctx->ev_mid, 0) != cudaSuccess)
             s = PHOTON_ERR_CUDA;
         else {
@@ -576,10 +577,10 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     if (beside) {
         if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess && s == PHOTON_OK) s = PHOTON_ERR_CUDA;
     } else if (s == PHOTON_OK && a->Nc > 0) {
-        s = photon_chunk_attn(ctx, a->chunks, a->q_chunk, a->slot, a->out_chunk, a->Nc, a->scale_chunk, stream);
+        s = photon_chunk_attn(ctx, a->chunks, q_chunk, slot, out_chunk, a->Nc, a->scale_chunk, stream);
     }
     if (copying && cudaStreamWaitEvent(st, ctx->ev_copy, 0) != cudaSuccess && s == PHOTON_OK) s = PHOTON_ERR_CUDA;
-    if (s == PHOTON_OK && hp && !apart && !copy_out(hp, 0, hp->out_bytes, st)) s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK && hp && !copying && !copy_out(hp, 0, apart || direct ? hp->out_split : hp->out_bytes, st)) s = PHOTON_ERR_CUDA;
     return s;
 }
 }  // namespace

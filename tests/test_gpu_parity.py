@@ -494,15 +494,17 @@ def test_decode_step_chain_matches_oracle(oracle, idx, layout):
         assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
 
 
+@pytest.mark.parametrize("idx,B,S", [(1, 24, 300), (4, 12, 128)])      # chunk attention beside the coarse part / in line after it
 @pytest.mark.parametrize("pinned,split", [(True, True), (True, False), (False, True), (False, False)])
-def test_decode_step_from_host_buffers(oracle, pinned, split):
+def test_decode_step_from_host_buffers(oracle, pinned, split, idx, B, S):
     """The step whose inputs (new K/V rows, both query tensors, the lengths) start in host memory and
     whose results end there: one packed buffer each way through the staging areas the arguments look into;
     with the split declared, the chunk attention's half of either buffer travels beside the coarse part."""
-    cfg = cfg_small(1, B=24, S=300)
+    cfg = cfg_small(idx, B=B, S=S)
     s = wl.step_inputs(cfg, poison=True)
     co, cv, chk = s["coarse"], s["converter"], s["chunks"]
     scale = cfg.dh ** -0.5
+    assert (cfg.Nc * cfg.Hkv * chk["cap"] * cfg.dh * 4 <= 32 << 20) == (idx == 1)
     with Ctx(cfg) as c:
         d, dc = coarse_to_dev(co), chunks_to_dev(chk)
         lens0 = co["len"].copy()                                             # before the append
