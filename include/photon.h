@@ -342,8 +342,8 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, 
  * and the coarse results leave beside the converter.  Where both host buffers
  * are page-locked memory that the device can address and q_chunk, slot and
  * out_chunk lie wholly in the chunk attention's halves of the staging areas,
- * the chunk attention reads and writes the host buffers themselves, on
- * whichever stream it runs (the same bytes cross the bus, no copy is enqueued
+ * the chunk attention reads and writes the host buffers themselves when it runs
+ * in line, or beside the coarse part with at most 1 MiB each way (the same bytes cross the bus, no copy is enqueued
  * for them, the coarse results still leave beside the converter) and those
  * halves of the staging areas are left untouched.  A buffer laid out
  * otherwise than declared gives stale inputs or results: the call cannot tell.

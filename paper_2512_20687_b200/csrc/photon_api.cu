@@ -521,8 +521,13 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     const int32_t *slot = a->slot;
     photon_bf16 *out_chunk = a->out_chunk;
     bool direct = false;
-    if (split) {
-        const size_t qb = (size_t)a->Nc * c.Hq * c.dh * sizeof(photon_bf16), sb = (size_t)a->Nc * sizeof(int32_t);
+    // Beside the coarse part only small chunk workloads go direct: a kernel that waits for the bus keeps its CTAs
+    // resident for as long as the transfer takes, and they stand in the way of the coarse part's kernels (measured with
+    // 2 MB each way on the shared-prefix workload: 155-269 us per step, unstable, against 154 us with copies; with
+    // 0.5 MB on the default workload: 65 against 67-78 us).  In line nothing runs beside it.
+    const size_t qb_all = (size_t)a->Nc * c.Hq * c.dh * sizeof(photon_bf16);
+    if (split && (!beside || qb_all <= (size_t(1) << 20))) {
+        const size_t qb = qb_all, sb = (size_t)a->Nc * sizeof(int32_t);
         const bool slot_in = slot && inside(slot, sb, hp->dev_in, hp->in_split, hp->in_bytes);
         const bool slot_off = !slot || (const char *)slot + sb <= hp->dev_in || (const char *)slot >= hp->dev_in + hp->in_bytes;
         if (inside(q_chunk, qb, hp->dev_in, hp->in_split, hp->in_bytes) &&
