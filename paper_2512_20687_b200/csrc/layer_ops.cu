@@ -66,7 +66,11 @@ rope_split_kernel(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq
     const int rotated = (Hq + Hkv) * vec_half, copied = Hkv * dh / 8;
     const int width = (Hq + 2 * Hkv) * dh, step = gridDim.x;
     ptx::grid_dep_wait();                   // qkv is the output of the kernel before this one
-    ptx::grid_dep_launch();
+    // The appending form must not let the next kernel start early: it reads and then updates the lengths, so an SM
+    // can hold a line of len[] in L1 in which only its own unit is current, and the attention that follows reads
+    // the lengths through the read-only path.  Launched after this grid has ended (as after the append kernel, which
+    // never releases its dependents early either) the attention starts with a clean L1.
+    if (!APPEND) ptx::grid_dep_launch();
     auto where = [&](int i) { return i < n ? (pos ? pos[i] : i % period) : 0; };   // no position array: row i % period of its group
     auto table = [&](int at, int buf) {
         // the angle and its reduction to [-pi, pi] in double precision, sine and cosine of the remainder in single
