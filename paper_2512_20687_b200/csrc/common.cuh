@@ -44,8 +44,6 @@ struct photon_ctx {
     cudaEvent_t ev_fork, ev_join;
     cudaStream_t copy;       // carries the coarse results to the host beside the converter (photon_decode_step_host)
     cudaEvent_t ev_mid, ev_copy;
-    const void *io_host[2];  // host buffers last looked up for a device alias (photon_decode_step_host) ..
-    char *io_alias[2];       // .. and the alias, or nullptr when the memory is not mapped into the device
     TmapCache tmaps;
 };
 

@@ -449,19 +449,13 @@ struct HostPlan {
 };
 
 // The address under which kernels can reach page-locked, mapped host memory; nullptr for any other memory.
-// Looked up once per buffer and remembered in the context.
-char *device_alias(photon_ctx *ctx, int which, const void *host) {
-    if (ctx->io_host[which] != host) {
-        cudaPointerAttributes at{};
-        char *alias = nullptr;
-        if (cudaPointerGetAttributes(&at, host) == cudaSuccess && at.type == cudaMemoryTypeHost)
-            alias = static_cast<char *>(at.devicePointer);
-        else
-            cudaGetLastError();
-        ctx->io_host[which] = host;
-        ctx->io_alias[which] = alias;
-    }
-    return ctx->io_alias[which];
+// Asked every time: an address can come back from the allocator as another kind of memory.
+char *device_alias(const void *host) {
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, host) == cudaSuccess && at.type == cudaMemoryTypeHost)
+        return static_cast<char *>(at.devicePointer);
+    cudaGetLastError();
+    return nullptr;
 }
 
 bool inside(const void *p, size_t n, const char *base, size_t from, size_t to) {
@@ -532,7 +526,7 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         const bool slot_off = !slot || (const char *)slot + sb <= hp->dev_in || (const char *)slot >= hp->dev_in + hp->in_bytes;
         if (inside(q_chunk, qb, hp->dev_in, hp->in_split, hp->in_bytes) &&
             inside(out_chunk, qb, hp->dev_out, hp->out_split, hp->out_bytes) && (slot_in || slot_off)) {
-            char *in_alias = device_alias(ctx, 0, hp->host_in), *out_alias = device_alias(ctx, 1, hp->host_out);
+            char *in_alias = device_alias(hp->host_in), *out_alias = device_alias(hp->host_out);
             if (in_alias && out_alias) {
                 direct = true;
                 q_chunk = reinterpret_cast<const photon_bf16 *>(in_alias + ((const char *)q_chunk - hp->dev_in));
