@@ -384,11 +384,13 @@ photon_status photon_coarse_attn_noalloc(const photon_config *cfg, const photon_
                                          const photon_bf16 *q, photon_bf16 *out, float *lse, float scale,
                                          int32_t *dev_status, photon_stream stream);
 
-/* Caps the persistent grid of photon_coarse_attn / photon_flat_attn at n CTAs
- * (0 or more than the device holds: the default, two per SM).  The keys of a
- * call are dealt out evenly over the grid, so n also moves the points where a
- * long cache is cut and merged by log-sum-exp; a smaller grid leaves SMs free
- * for work on another stream.  Takes effect from the next call. */
+/* Sets the persistent grid of photon_coarse_attn / photon_flat_attn to n CTAs
+ * (0 or more than the device holds, two per SM: back to the default, where
+ * the library picks a grid of at most 7/8 of what the device holds, lined up
+ * with the number of (unit, KV head) streams of the call).  The keys of a call
+ * are dealt out evenly over the grid, so n also moves the points where a long
+ * cache is cut and merged by log-sum-exp; a smaller grid leaves SMs free for
+ * work on another stream.  Takes effect from the next call. */
 photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n);
 
 /* Number of kernels the library has launched through this context so far. */

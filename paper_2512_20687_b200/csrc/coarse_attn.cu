@@ -39,13 +39,17 @@ namespace {
 
 constexpr int NW = 4;                      // consumer warps per CTA
 constexpr int BN = 64;                     // keys per tile
-constexpr int BOX = 32;                    // rows per TMA box
+constexpr int BOX = 32;                    // rows per TMA box of a tile's ragged end; whole tiles use boxes of BN rows
 constexpr int THREADS = (NW + 2) * 32;     // + one producer warp + one finishing warp
 constexpr int STAGES = 3;
 constexpr int HALF_BYTES = BN * 128;       // 64 rows x 64 elements, swizzled
 constexpr int BOX_BYTES = BOX * 128;
 constexpr int CTAS_PER_SM = 2;
-constexpr int SNAP = 8;                    // streams of at most this many tiles are never cut
+#ifndef COARSE_SNAP
+#define COARSE_SNAP 8
+#endif
+constexpr int SNAP = COARSE_SNAP;          // streams of at most this many tiles are never cut
+constexpr int NLEN = 768;                  // lengths of the first NLEN units are kept in shared memory
 
 template <int DH>
 struct Ring {
@@ -59,26 +63,62 @@ __host__ __device__ inline int q_slot_bytes(int G, int dh) { return (G * dh * 2 
 template <int DH>
 size_t smem_bytes(int G) {
     return 1024 /*alignment slack*/ + size_t(STAGES) * (Ring<DH>::STAGE_BYTES + q_slot_bytes(G, DH)) +
-           size_t(NW) * G * (DH + 2) * sizeof(float) + 128 /*barriers*/ + 128 /*scalars*/;
+           size_t(NW) * G * (DH + 2) * sizeof(float) + 128 /*barriers*/ + 128 /*scalars*/ + NLEN * sizeof(int);
 }
 
 __device__ __forceinline__ int clamp_len(int len, int cap) { return max(0, min(len, cap)); }
 __device__ __forceinline__ int tiles_of(int len) { return (len + BN - 1) / BN; }
 
-// Position in the sequence of tiles: tile j of the stream (unit u, KV head h).
+// Index arrays (lengths, page ids, prefix ids) are read through the L2 only: another kernel may have
+// written them just before this one, and a line of them left in an SM's L1 by an earlier kernel is not
+// refreshed by a dependent launch.
+__device__ __forceinline__ int ld_len(const AttnParams &p, int u) { return clamp_len(__ldcg(p.len + u), p.cap); }
+
+constexpr int LPT = NLEN / THREADS;        // lengths per thread when a batch fits the shared-memory copy
+static_assert(NLEN % THREADS == 0, "a thread's units must fit its registers");
+
+// The lengths of units [ub, ue), at most LPT of them, requested before any is used.
+__device__ __forceinline__ void load_lengths(const AttnParams &p, int ub, int ue, int (&len)[LPT]) {
+#pragma unroll
+    for (int i = 0; i < LPT; ++i) len[i] = ub + i < ue ? __ldcg(p.len + ub + i) : 0;
+#pragma unroll
+    for (int i = 0; i < LPT; ++i) len[i] = clamp_len(len[i], p.cap);
+}
+
+// A CTA's part of the tile sequence.
+struct Share {
+    long long T;             // tiles in the whole call
+    int n_cta;               // CTAs that take part
+    long long t0, t1;        // this CTA's tiles [t0, t1)
+    int u0, rem;             // tile t0 is tile `rem` of the Hkv * nt tiles of unit u0
+};
+
+// Position in the sequence of tiles: tile j of the stream (unit u, KV head h).  The lengths of units
+// [0, NLEN) sit in shared memory, read once per CTA; those of later units come from the L2.
 struct Walker {
     int u, h, j, nt, len;
+    const int *slen;
     __device__ __forceinline__ void load(const AttnParams &p) {
-        len = clamp_len(p.len[u], p.cap);
+        len = u < NLEN ? slen[u] : ld_len(p, u);
         nt = tiles_of(len);
     }
+    // false: the share does not start at a tile of unit u0 (the lengths changed under the kernel)
+    __device__ __forceinline__ bool start(const AttnParams &p, const Share &sh, const int *lens) {
+        slen = lens; u = sh.u0; h = 0; j = 0; nt = 0; len = 0;
+        if (u < 0 || u >= p.n_units) return false;
+        load(p);
+        if (nt == 0 || sh.rem < 0 || sh.rem >= nt * p.Hkv) return false;
+        h = sh.rem / nt; j = sh.rem % nt;
+        return true;
+    }
+    __device__ __forceinline__ bool valid(const AttnParams &p) const { return u < p.n_units; }
     __device__ __forceinline__ void next(const AttnParams &p) {
         if (++j < nt) return;
         j = 0;
         if (++h < p.Hkv) return;
         h = 0;
         do {
-            if (++u >= p.n_units) { nt = 0; len = 0; return; }
+            if (++u >= p.n_units) { u = p.n_units; nt = 0; len = 0; return; }
             load(p);
         } while (nt == 0);
     }
@@ -95,7 +135,7 @@ template <int DH>
 __device__ __forceinline__ void emit(const AttnParams &p, int u, int hq, int d, float acc, float M, float L) {
     const size_t qh = (size_t)u * p.Hq + hq;
     if (p.splits_sh > 0) {
-        const int s = p.sh_id[u];
+        const int s = __ldcg(p.sh_id + u);
         if (s >= p.n_shared) {                       // bad shared id voids the query
             if (d == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
             L = 0.f; acc = 0.f;
@@ -129,7 +169,7 @@ template <int DH, int MAXV>
 __device__ __forceinline__ void fetch_shared(const AttnParams &p, int u, int hq, int d0, SharedPart<MAXV> &sp) {
     sp.sid = -1;
     if (p.splits_sh <= 0) return;
-    sp.sid = p.sh_id[u];
+    sp.sid = __ldcg(p.sh_id + u);
     if (sp.sid < 0 || sp.sid >= p.n_shared) return;
     const float *pj = p.partials + ((size_t)u * p.Hq + hq) * (DH + 2);
     sp.l = __ldcg(pj + DH + 1);
@@ -261,51 +301,31 @@ __device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, 
     }
 }
 
-// GP: the group size G rounded up to a power of two (1 .. 16); it fixes how the finishing warp's lanes
-// map to (query head, features) and how many n-tiles of 8 heads the MMAs span.
-template <int DH, int GP>
-__global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
-coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ CUtensorMap tm_v) {
-    using R = Ring<DH>;
-    constexpr int NT8 = GP > 8 ? 2 : 1;
-    extern __shared__ uint8_t smem_raw[];
-    const int G = p.Hq / p.Hkv;
-    const int QB = q_slot_bytes(G, DH);
-    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
-    const uint32_t q_base = base + STAGES * R::STAGE_BYTES;
-    float *red = reinterpret_cast<float *>(gen + STAGES * (R::STAGE_BYTES + QB));      // [NW][G][DH + 2]
-    uint8_t *tail = reinterpret_cast<uint8_t *>(red) + (size_t)NW * G * (DH + 2) * sizeof(float);
-    const uint32_t bars = ptx::smem_u32(tail);                  // full[s] at +16s, empty[s] at +16s+8
-    const uint32_t red_full = bars + 16 * STAGES, red_empty = red_full + 8;
-    int *sc = reinterpret_cast<int *>(tail + 128);              // [0..5] warp sums, [8] u0, [9] rem, [10] len(u0), [11] dead, [12] t0, [14] t1,
-    volatile int *dead = sc + 11;                               // [16..23] description of the stream in `red`
-    volatile int *meta = sc + 16;
-
+// The even deal of the tile sequence over the grid, found by all threads of the CTA from len[]: every
+// length is read once (and left in shared memory for units below NLEN), a block-wide prefix sum of tile
+// counts follows, then the two boundaries of this CTA's share.  Boundary c is tile T*c/n_cta; where it
+// falls inside a short stream (<= SNAP tiles) it moves to the nearer end of that stream (finishing a
+// cut stream costs round trips to global memory, more than a few tiles of imbalance); long streams are
+// cut.  sc: [0..5] warp sums, [8] u0, [9] rem, [12] t0, [14] t1.
+__device__ __forceinline__ Share deal(const AttnParams &p, int *sc, int *slen, int cta) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cta = blockIdx.x;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(bars + 16 * s, 1);
-            ptx::mbar_init(bars + 16 * s + 8, NW);
-        }
-        ptx::mbar_init(red_full, NW);
-        ptx::mbar_init(red_empty, 1);
-        sc[8] = -1; sc[9] = 0; sc[10] = 0; sc[11] = 0; sc[12] = 0; sc[14] = -1;
-        ptx::mbar_fence_init();
-        ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
-    }
-
-    ptx::grid_dep_wait();                   // lengths, caches and queries may come from the kernel before this one
-    ptx::grid_dep_launch();                 // one wave of CTAs, all resident: the next kernel may line up behind them
-
-    // ---- where this CTA's share of the tile sequence starts: block-wide prefix sum of tile counts
+    auto len_of = [&](int u) { return u < NLEN ? slen[u] : ld_len(p, u); };
     const int per = (p.n_units + THREADS - 1) / THREADS;
     const int ub = min(p.n_units, (int)threadIdx.x * per), ue = min(p.n_units, ub + per);
     int mine = 0;
-    for (int u = ub; u < ue; ++u) mine += tiles_of(clamp_len(__ldg(p.len + u), p.cap));
+    if (per <= LPT) {                                             // all loads in flight together
+        int len[LPT];
+        load_lengths(p, ub, ue, len);
+#pragma unroll
+        for (int i = 0; i < LPT; ++i)
+            if (ub + i < ue) { slen[ub + i] = len[i]; mine += tiles_of(len[i]); }
+    } else {
+        for (int u = ub; u < ue; ++u) {
+            const int len = ld_len(p, u);
+            if (u < NLEN) slen[u] = len;
+            mine += tiles_of(len);
+        }
+    }
     int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -320,39 +340,38 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         if (w < warp) before += sc[w];
         all += sc[w];
     }
-    const long long T = (long long)all * p.Hkv;                  // tiles in the whole call
+    Share sh;
+    sh.T = (long long)all * p.Hkv;
     // every CTA that takes part owns at least one tile of the even deal, so the CTAs holding a cut stream
     // are consecutive
-    const int n_cta = (int)min((long long)gridDim.x, T);
-    // Boundary c of the even deal is tile T*c/n_cta.  Where it falls inside a short stream (<= SNAP
-    // tiles) it moves to the nearer end of that stream: finishing a cut stream costs several round trips
-    // to global memory at the end of a CTA, more than a few tiles of imbalance.  Long streams are cut.
+    sh.n_cta = (int)min((long long)gridDim.x, sh.T);
     {
         const long long lo = (long long)(before + incl - mine) * p.Hkv, hi = lo + (long long)mine * p.Hkv;
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
             const int c = cta + which;
-            if (cta >= n_cta || c >= n_cta) continue;
-            const long long x = T * c / n_cta;
+            if (cta >= sh.n_cta || c >= sh.n_cta) continue;
+            // (64-bit division is a long instruction sequence on the way to the first load)
+            const long long x = sh.T < (1 << 20) ? (long long)((unsigned)sh.T * (unsigned)c / (unsigned)sh.n_cta)
+                                                 : sh.T * c / sh.n_cta;
             if (!(lo <= x && x < hi)) continue;
             long long pre = lo;
             for (int u = ub; u < ue; ++u) {
-                const int len = clamp_len(__ldg(p.len + u), p.cap);
-                const int nt = tiles_of(len);
+                const int nt = tiles_of(len_of(u));
                 const long long k = (long long)nt * p.Hkv;
-                if (x < pre + k) {
-                    int rem = (int)(x - pre), uu = u, ll = len;
+                if (x < pre + k) {                                // nt > 0 here
+                    int rem = (int)(x - pre), uu = u;
                     const int j = rem % nt;
                     long long bx = x;
                     if (nt <= SNAP && j != 0) {
                         if (2 * j <= nt) { bx = x - j; rem -= j; }
                         else { bx = x + (nt - j); rem += nt - j; }
                     }
-                    if (rem == nt * p.Hkv) {                      // moved to the start of the next stream's unit
+                    if (rem == nt * p.Hkv) {                      // moved to the start of the next unit that has keys
                         rem = 0;
-                        do { ++uu; ll = uu < p.n_units ? clamp_len(p.len[uu], p.cap) : 0; } while (uu < p.n_units && ll == 0);
+                        do { ++uu; } while (uu < p.n_units && len_of(uu) == 0);
                     }
-                    if (which == 0) { sc[8] = uu; sc[9] = rem; sc[10] = ll; sc[12] = (int)bx; }
+                    if (which == 0) { sc[8] = uu; sc[9] = rem; sc[12] = (int)bx; }
                     else sc[14] = (int)bx;
                     break;
                 }
@@ -361,14 +380,108 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         }
     }
     __syncthreads();
-    const long long t0 = cta < n_cta ? sc[12] : 0;
-    const long long t1 = cta < n_cta ? (sc[14] >= 0 ? sc[14] : T) : 0;
+    const bool in = cta < sh.n_cta;
+    sh.t0 = in ? sc[12] : 0;
+    sh.t1 = in ? (sc[14] >= 0 ? sc[14] : sh.T) : 0;
+    sh.u0 = sc[8]; sh.rem = sc[9];
+    return sh;
+}
+
+// Address of the first key row of tile w.j of the stream (w.u, w.h) as a row of the cache tensor
+// (contiguous, or through the page table); -1 for a page id out of range.
+__device__ __forceinline__ int tile_row(const AttnParams &p, const Walker &w) {
+    if (!p.page_table) return (w.u * p.Hkv + w.h) * p.cap + w.j * BN;
+    const int row = w.j * BN;
+    const int id = __ldcg(p.page_table + (size_t)w.u * p.pages_per_unit + row / p.page_rows);
+    if (id < 0 || id >= p.n_pages) return -1;
+    return (id * p.Hkv + w.h) * p.page_rows + row % p.page_rows;
+}
+
+// GP: the group size G rounded up to a power of two (1 .. 16); it fixes how the finishing warp's lanes
+// map to (query head, features) and how many n-tiles of 8 heads the MMAs span.
+template <int DH, int GP>
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM)
+coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                   const __grid_constant__ CUtensorMap tm_k_end, const __grid_constant__ CUtensorMap tm_v_end) {
+    using R = Ring<DH>;
+    constexpr int NT8 = GP > 8 ? 2 : 1;
+    extern __shared__ uint8_t smem_raw[];
+    const int G = p.Hq / p.Hkv;
+    const int QB = q_slot_bytes(G, DH);
+    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+    const uint32_t q_base = base + STAGES * R::STAGE_BYTES;
+    float *red = reinterpret_cast<float *>(gen + STAGES * (R::STAGE_BYTES + QB));      // [NW][G][DH + 2]
+    uint8_t *tail = reinterpret_cast<uint8_t *>(red) + (size_t)NW * G * (DH + 2) * sizeof(float);
+    const uint32_t bars = ptx::smem_u32(tail);                  // full[s] at +16s, empty[s] at +16s+8
+    const uint32_t red_full = bars + 16 * STAGES, red_empty = red_full + 8;
+    int *sc = reinterpret_cast<int *>(tail + 128);              // scalars of the deal, [11] dead,
+    volatile int *dead = sc + 11;                               // [16..23] description of the stream in `red`
+    volatile int *meta = sc + 16;
+    int *slen = sc + 32;                                        // [NLEN] lengths of the first units
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(bars + 16 * s, 1);
+            ptx::mbar_init(bars + 16 * s + 8, NW);
+        }
+        ptx::mbar_init(red_full, NW);
+        ptx::mbar_init(red_empty, 1);
+        sc[8] = -1; sc[9] = 0; sc[11] = 0; sc[12] = 0; sc[14] = -1;
+        ptx::mbar_fence_init();
+        ptx::prefetch_tmap(&tm_k); ptx::prefetch_tmap(&tm_v);
+        ptx::prefetch_tmap(&tm_k_end); ptx::prefetch_tmap(&tm_v_end);
+    }
+
+    // ---- the deal, ahead of the kernel before this one.  The lengths as they read now may still change
+    // (an append in flight), and no key or value is touched yet; after the dependency wait every length is
+    // read again, and the deal stands if no unit's tile count differs (it depends on nothing else), so
+    // that one trip to the L2 and one barrier are all that separates the wait from the first load.
+    // Batches beyond NLEN units keep no copy to compare with and deal after the wait.
+    const bool ahead = p.n_units <= NLEN;
+    Share sh;
+    Walker w;
+    bool started = false;
+    if (ahead) {
+        sh = deal(p, sc, slen, cta);
+        if (sh.t0 < sh.t1) started = w.start(p, sh, slen);
+    }
+
+    ptx::grid_dep_wait();                   // lengths, caches and queries may come from the kernel before this one
+    ptx::grid_dep_launch();                 // one wave of CTAs, all resident: the next kernel may line up behind them
+
+    bool redo = !ahead;
+    if (ahead) {
+        const int per = (p.n_units + THREADS - 1) / THREADS;
+        const int ub = min(p.n_units, (int)threadIdx.x * per), ue = min(p.n_units, ub + per);
+        int diff = 0, len[LPT];
+        load_lengths(p, ub, ue, len);
+#pragma unroll
+        for (int i = 0; i < LPT; ++i)
+            if (ub + i < ue) {
+                diff |= (tiles_of(len[i]) != tiles_of(slen[ub + i]));
+                slen[ub + i] = len[i];
+            }
+        redo = __syncthreads_or(diff);
+    }
+    if (redo) {
+        if (threadIdx.x == 0) { sc[8] = -1; sc[9] = 0; sc[12] = 0; sc[14] = -1; }
+        sh = deal(p, sc, slen, cta);
+        started = sh.t0 < sh.t1 && w.start(p, sh, slen);
+    } else if (started) {
+        w.load(p);                          // same tile counts, but the unit may have grown within its last tile
+    }
+    const long long T = sh.T, t0 = sh.t0, t1 = sh.t1;
+    const int n_cta = sh.n_cta;
 
     // ---- units without own keys are visited by no tile: they are finished by whoever has time for it
     // (the whole CTA when it has no tiles, else the finishing warp before its first stream arrives)
     auto finish_empty_units = [&](int tid, int nthreads) {
         for (int u = cta; u < p.n_units; u += gridDim.x) {
-            if (clamp_len(__ldg(p.len + u), p.cap) != 0) continue;
+            if ((u < NLEN ? slen[u] : ld_len(p, u)) != 0) continue;
             for (int idx = tid; idx < p.Hq * DH; idx += nthreads)
                 emit<DH>(p, u, idx / DH, idx % DH, 0.f, -CUDART_INF_F, 0.f);
         }
@@ -379,6 +492,11 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     }
 
     const int n_tiles = (int)(t1 - t0);
+    if (!started) {
+        // the deal and the lengths disagree: len[] changed while the kernel ran.  Nothing is loaded or written.
+        if (threadIdx.x == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+        return;
+    }
 
     if (warp == NW + 1) {
         // ======================= finishing warp =======================
@@ -389,19 +507,25 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         const bool row_ok = r < G, lead = row_ok && (lane % lpr == 0);
         finish_empty_units(lane, 32);
         // it walks the streams of this CTA in the consumers' order, one step ahead of them
-        Walker fw;
-        fw.u = sc[8]; fw.len = sc[10]; fw.nt = tiles_of(fw.len);
-        fw.h = sc[9] / fw.nt; fw.j = sc[9] % fw.nt;
+        Walker fw = w;
         for (int sidx = 0;; ++sidx) {
             SharedPart<MAXV> sp;
             sp.sid = -1;
-            if (row_ok && fw.u < p.n_units) fetch_shared<DH, MAXV>(p, fw.u, fw.h * G + r, d0, sp);
+            if (row_ok && fw.valid(p)) fetch_shared<DH, MAXV>(p, fw.u, fw.h * G + r, d0, sp);
             if (*dead || !ptx::mbar_wait(red_full, sidx & 1)) {
                 if (!*dead) { *dead = 1; if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT); }
                 break;
             }
             const int u = meta[0], h = meta[1], flags = meta[2], c_first = meta[3], c_last = meta[4];
             const bool whole = flags & 1, final_seg = flags & 2;
+            if (flags & 4) break;                               // the consumers finish the CTA's last stream themselves
+            if (u < 0 || u >= p.n_units || h < 0 || h >= p.Hkv || c_first < 0 || c_last >= (int)gridDim.x ||
+                c_first > c_last) {
+                // no such stream: the consumers ran past the last unit
+                if (lane == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+                *dead = 1;
+                break;
+            }
             float acc[MAXV], M = -CUDART_INF_F, L = 0.f;
 #pragma unroll
             for (int i = 0; i < MAXV; ++i) acc[i] = 0.f;
@@ -494,13 +618,6 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         return;
     }
 
-    Walker w;
-    w.u = sc[8];
-    w.len = sc[10];
-    w.nt = tiles_of(w.len);
-    w.h = sc[9] / w.nt;
-    w.j = sc[9] % w.nt;
-
     if (warp == NW) {
         // ======================= producer: one thread feeds the ring =======================
         if (lane == 0) {
@@ -508,30 +625,30 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
             for (; it < n_tiles; ++it, w.next(p)) {
                 const int s = it % STAGES;
                 if (*dead) break;
+                if (!w.valid(p)) {                               // ran past the last unit: len[] changed under the kernel
+                    *dead = 1; atomicOr(p.status, PHOTON_DEV_BAD_INDEX); break;
+                }
                 // row of the tile's first key in the cache tensor; for a paged cache through the page table
                 // (looked up before the wait for a free stage, which hides the load's latency)
-                int y = (w.u * p.Hkv + w.h) * p.cap + w.j * BN;
-                if (p.page_table) {
-                    const int row = w.j * BN;
-                    int id = __ldg(p.page_table + (size_t)w.u * p.pages_per_unit + row / p.page_rows);
-                    if (id < 0 || id >= p.n_pages) { atomicOr(p.status, PHOTON_DEV_BAD_INDEX); id = 0; }
-                    y = (id * p.Hkv + w.h) * p.page_rows + row % p.page_rows;
-                }
-                if (!ptx::mbar_wait(bars + 16 * s + 8, ((it / STAGES) & 1) ^ 1)) {
+                int y = tile_row(p, w);
+                if (y < 0) { atomicOr(p.status, PHOTON_DEV_BAD_INDEX); y = w.h * (p.page_table ? p.page_rows : p.cap); }
+                // the ring starts empty: only from its second turn on is there a stage to wait for
+                if (it >= STAGES && !ptx::mbar_wait(bars + 16 * s + 8, ((it / STAGES) & 1) ^ 1)) {
                     *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
                 }
                 const uint32_t full = bars + 16 * s;
                 const uint32_t kd = base + s * R::STAGE_BYTES, vd = kd + R::TILE_BYTES;
                 const int rows = min(BN, w.len - w.j * BN);
-                const int nbox = (rows + BOX - 1) / BOX;
                 const bool first = (it == 0 || w.j == 0);
-                ptx::mbar_arrive_expect_tx(full, nbox * R::HALVES * BOX_BYTES * 2 + (first ? G * DH * 2 : 0));
-                for (int b = 0; b < nbox; ++b)
+                // a tile of more than BOX rows comes as one box of BN rows per 64 features (what lies past the end
+                // of the cache is never used), a shorter one as one box of BOX rows
+                const bool tall = rows > BOX;
+                ptx::mbar_arrive_expect_tx(full, R::HALVES * (tall ? HALF_BYTES : BOX_BYTES) * 2 + (first ? G * DH * 2 : 0));
 #pragma unroll
-                    for (int hh = 0; hh < R::HALVES; ++hh) {
-                        ptx::tma_load_2d(kd + hh * HALF_BYTES + b * BOX_BYTES, &tm_k, hh * 64, y + b * BOX, full);
-                        ptx::tma_load_2d(vd + hh * HALF_BYTES + b * BOX_BYTES, &tm_v, hh * 64, y + b * BOX, full);
-                    }
+                for (int hh = 0; hh < R::HALVES; ++hh) {
+                    ptx::tma_load_2d(kd + hh * HALF_BYTES, tall ? &tm_k : &tm_k_end, hh * 64, y, full);
+                    ptx::tma_load_2d(vd + hh * HALF_BYTES, tall ? &tm_v : &tm_v_end, hh * 64, y, full);
+                }
                 if (first)
                     ptx::bulk_load(q_base + s * QB, p.q + ((size_t)w.u * p.Hq + (size_t)w.h * G) * DH, G * DH * 2, full);
             }
@@ -587,14 +704,18 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         {
             const uint32_t kt = base + s * R::STAGE_BYTES, vt = kt + R::TILE_BYTES;
             const int v = min(BN, w.len - w.j * BN) - 16 * warp;
-            if (v > 0) process_block<DH, NT8>(kt, vt, warp, min(v, 16), qb, o, m, l, p.scale_log2, lane);
+            if (v > 0 && !*dead) process_block<DH, NT8>(kt, vt, warp, min(v, 16), qb, o, m, l, p.scale_log2, lane);
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(bars + 16 * s + 8);
 
         const bool stream_end = (w.j == w.nt - 1);
         if (stream_end || it == n_tiles - 1) {
-            // ---- hand this warp's state to the finishing warp through `red`
+            // ---- this warp's state goes into `red`: for the finishing warp, or, when this is the CTA's last
+            // stream and it is complete, for the consumer warps themselves (each takes a quarter of the rows:
+            // nothing else is left to do, and four warps are through sooner than one)
+            const bool whole = stream_end && seg_j0 == 0, final_seg = (it == n_tiles - 1);
+            const bool direct = whole && final_seg && p.splits_sh == 0;
 #pragma unroll
             for (int nt = 0; nt < NT8; ++nt)
 #pragma unroll
@@ -622,16 +743,51 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                     }
                 }
             if (warp == 0 && lane == 0) {
-                // CTAs that hold a piece of this stream: first and last
-                const long long te = seg_t + w.nt;
                 meta[0] = w.u; meta[1] = w.h;
-                meta[2] = ((stream_end && seg_j0 == 0) ? 1 : 0) | (it == n_tiles - 1 ? 2 : 0);
-                meta[3] = (int)(((seg_t + 1) * n_cta - 1) / T);
-                meta[4] = (int)((te * n_cta - 1) / T);
+                meta[2] = (whole ? 1 : 0) | (final_seg ? 2 : 0) | (direct ? 4 : 0);
+                meta[3] = meta[4] = cta;
+                if (!whole) {
+                    // CTAs that hold a piece of this stream: first and last
+                    const long long te = seg_t + w.nt;
+                    meta[3] = (int)(((seg_t + 1) * n_cta - 1) / T);
+                    meta[4] = (int)((te * n_cta - 1) / T);
+                }
             }
+            if (direct) ptx::named_bar_sync(1, NW * 32);
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(red_full);
             ++sidx;
+            if (direct && !*dead) {
+                // thread -> four consecutive features of one query head; same arithmetic as the finishing warp's
+                for (int e = (warp * 32 + lane) * 4; e < G * DH; e += NW * 32 * 4) {
+                    const int r = e / DH, d0 = e % DH;
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f}, M = -CUDART_INF_F, L = 0.f;
+#pragma unroll
+                    for (int ww = 0; ww < NW; ++ww) {
+                        const float *src = red + ((size_t)ww * G + r) * (DH + 2);
+                        if (src[DH + 1] > 0.f) M = fmaxf(M, src[DH]);
+                    }
+#pragma unroll
+                    for (int ww = 0; ww < NW; ++ww) {
+                        const float *src = red + ((size_t)ww * G + r) * (DH + 2);
+                        const float lw = src[DH + 1];
+                        if (lw > 0.f) {
+                            const float f = exp2f(src[DH] - M);
+                            L += lw * f;
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                const float2 a = *reinterpret_cast<const float2 *>(src + d0 + 2 * i);
+                                acc[2 * i] += a.x * f; acc[2 * i + 1] += a.y * f;
+                            }
+                        }
+                    }
+                    const float inv = L > 0.f ? 1.f / L : 0.f;
+                    const size_t qh = (size_t)w.u * p.Hq + (size_t)w.h * G + r;
+                    *reinterpret_cast<uint2 *>(p.out + qh * DH + d0) =
+                        make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
+                    if (d0 == 0 && p.lse) p.lse[qh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
+                }
+            }
         }
         w.next(p);
     }
@@ -644,15 +800,20 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     static size_t smem_set[kMaxDevices] = {};
     if (const cudaError_t e = ensure_dynamic_smem(coarse_attn_kernel<DH, GP>, smem, ctx->device, smem_set)) return e;
     const CUtensorMap *t;
-    CUtensorMap mk, mv;
+    CUtensorMap mk, mv, mk_end, mv_end;
     const uint64_t pool_rows = p.page_table ? (uint64_t)p.n_pages * p.Hkv * p.page_rows : (uint64_t)p.n_units * p.Hkv * p.cap;
-    if (!(t = ctx->tmaps.get(p.k, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
+    if (!(t = ctx->tmaps.get(p.k, pool_rows, DH, BN))) return cudaErrorInvalidValue;
     mk = *t;
-    if (!(t = ctx->tmaps.get(p.v, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
+    if (!(t = ctx->tmaps.get(p.v, pool_rows, DH, BN))) return cudaErrorInvalidValue;
     mv = *t;
+    if (!(t = ctx->tmaps.get(p.k, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
+    mk_end = *t;
+    if (!(t = ctx->tmaps.get(p.v, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
+    mv_end = *t;
     const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
-    const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, ctx->max_ctas));
-    const cudaError_t e = launch_dependent(coarse_attn_kernel<DH, GP>, dim3(grid), dim3(THREADS), smem, st, 0, p, mk, mv);
+    const long long cap = ctx->attn_ctas > 0 ? ctx->attn_ctas : coarse_attn_grid(ctx->max_ctas, (long long)p.n_units * p.Hkv);
+    const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, cap));
+    const cudaError_t e = launch_dependent(coarse_attn_kernel<DH, GP>, dim3(grid), dim3(THREADS), smem, st, 0, p, mk, mv, mk_end, mv_end);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -660,6 +821,28 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
 }  // namespace
 
 int coarse_attn_ctas_per_sm() { return CTAS_PER_SM; }
+
+// The grid when the caller sets none.  Not every CTA slot of the device is taken: the kernel is bound by
+// HBM well below that, and a slot left free lets a CTA of the next kernel in the stream start, and get
+// through its set-up, while this one still runs (measured on caches of 64 to 256 MiB: 7/8 of the slots is 1 to 4 %
+// faster than all of them).  Below that bound the grid is a multiple or a near-divisor of the number of
+// (unit, KV head) streams, so that in a batch of equal lengths every stream falls to the same whole
+// number of CTAs, or every CTA to the same whole number of streams, and the cuts of the even deal line
+// up with the streams' ends; with ragged lengths the deal is even whatever the grid.
+int coarse_attn_grid(int resident_ctas, long long n_streams) {
+    const int top = std::max(1, resident_ctas * 7 / 8);
+    if (n_streams <= 0) return 1;
+    if (n_streams <= top) return (int)(n_streams * (top / n_streams));
+    // more streams than CTAs: the grid within the upper quarter that wastes the fewest stream slots
+    int best = top;
+    long long best_waste = -1;
+    for (int g = top; g >= top - top / 4; --g) {
+        const long long waste = (n_streams + g - 1) / g * g - n_streams;
+        if (best_waste < 0 || waste < best_waste) { best = g; best_waste = waste; }
+        if (waste == 0) break;
+    }
+    return best;
+}
 
 cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st, long long *launches) {
     if (p.n_q == 0) return cudaSuccess;

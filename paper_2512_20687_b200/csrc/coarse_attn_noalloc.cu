@@ -82,6 +82,7 @@ extern "C" photon_status photon_coarse_attn_noalloc(const photon_config *cfg, co
             s.ctx.device = dev;
             s.ctx.sm_count = prop.multiProcessorCount;
             s.ctx.max_ctas = std::min(kMaxCtas, prop.multiProcessorCount * coarse_attn_ctas_per_sm());
+            s.ctx.attn_ctas = 0;
             s.ctx.max_splits = 1;
             s.ctx.partials = nullptr;
             s.ctx.partial_floats = 0;

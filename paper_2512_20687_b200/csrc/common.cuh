@@ -34,7 +34,8 @@ struct photon_ctx {
     float *partials;         // shared-prefix partials: [max_queries * Hq][dh + 2] floats (acc, m, l)
     size_t partial_floats;
     float *cta_partials;     // partials of streams cut by a CTA boundary: [2 * max_ctas][16][dh + 2] floats
-    int max_ctas;            // grid of the persistent attention kernel
+    int max_ctas;            // most CTAs the persistent attention kernel can hold: two per SM
+    int attn_ctas;           // the caller's cap on that grid (photon_set_attention_ctas), 0: the launcher chooses
     int32_t *tickets;        // one arrival counter per (unit, kv head); zero between calls
     size_t n_tickets;
     int32_t *status;         // device status word
@@ -156,6 +157,7 @@ cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t 
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                            long long *launches);
 int coarse_attn_ctas_per_sm();
+int coarse_attn_grid(int resident_ctas, long long n_streams);
 int shared_prefix_units_per_cta(int G);
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);

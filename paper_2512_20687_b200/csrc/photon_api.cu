@@ -131,6 +131,7 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
     ctx->partial_floats = size_t(c.max_queries) * c.Hq * (c.dh + 2);      // one shared-prefix partial per query head
     ctx->n_tickets = size_t(c.max_queries) * c.Hkv;
     ctx->max_ctas = ctx->sm_count * coarse_attn_ctas_per_sm();
+    ctx->attn_ctas = 0;
     if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->cta_partials, size_t(2) * ctx->max_ctas * 16 * (c.dh + 2) * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->tickets, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
@@ -628,8 +629,7 @@ int64_t photon_launch_count(const photon_ctx *ctx) { return ctx ? ctx->launches 
 
 photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n) {
     if (!ctx || n < 0) return PHOTON_ERR_INVALID_ARG;
-    const int full = ctx->sm_count * coarse_attn_ctas_per_sm();
-    ctx->max_ctas = (n == 0 || n > full) ? full : n;
+    ctx->attn_ctas = (n <= 0 || n > ctx->max_ctas) ? 0 : n;
     return PHOTON_OK;
 }
 
