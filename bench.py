@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--max-splits", type=int, default=0)
     ap.add_argument("--hierarchy", default="",
                     help="chunk lengths C_1,...,C_L instead of 4,4 (e.g. 2,2): same model and context, other stream lengths")
+    ap.add_argument("--attention-ctas", type=int, default=0,
+                    help="persistent grid of the coarse attention (0: the library's choice)")
     ap.add_argument("--batch", type=int, default=0,
                     help="shrink the workload to this many sequences (for profiler captures of a small case)")
     return ap.parse_args()
@@ -233,6 +235,8 @@ def run_gpu(args, cfg) -> None:
                       shared_id=torch.from_numpy(co["shared_id"]).to(dev))
     ctx = ph.photon_create(cfg.Hq, cfg.Hkv, cfg.dh, cfg.D, cfg.P, cfg.C, max(cfg.B, cfg.Nc),
                            args.max_splits)
+    if args.attention_ctas:
+        ph.photon_set_attention_ctas(ctx, args.attention_ctas)
     reps = []
     for r in range(R):
         t = {n: (b if r == 0 else b.clone()) for n, b in base.items()}

@@ -46,7 +46,7 @@ chunk_attn_kernel(const AttnParams p) {
     const int G = p.Hq / p.Hkv;
     const int col = lane % VEC, rsub = lane / VEC;
 
-    const int u = p.slot ? p.slot[i] : i;
+    const int u = p.slot ? __ldcg(p.slot + i) : i;               // index arrays through the L2: another kernel may have just written them
     bf16 *out_base = p.out + ((size_t)i * p.Hq + (size_t)kvh * G) * DH + col * 8;
     if (u < 0 || u >= p.n_units) {
         if (lane == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
@@ -55,7 +55,7 @@ chunk_attn_kernel(const AttnParams p) {
                 *reinterpret_cast<uint4 *>(out_base + (size_t)g * DH) = make_uint4(0u, 0u, 0u, 0u);
         return;
     }
-    const int len = max(0, min(p.len[u], p.cap));
+    const int len = max(0, min(__ldcg(p.len + u), p.cap));
     const size_t base = ((size_t)u * p.Hkv + kvh) * p.cap * DH;
     const uint4 *kp = reinterpret_cast<const uint4 *>(p.k + base) + lane;     // row rsub, vector col
     const uint4 *vp = reinterpret_cast<const uint4 *>(p.v + base) + lane;

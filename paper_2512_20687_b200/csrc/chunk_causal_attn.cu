@@ -173,10 +173,10 @@ chunk_causal_attn_kernel(const CausalParams p) {
     auto get_item = [&](int x) {
         Item it;
         where(x, it.i, it.kvh, it.g0);
-        it.u = p.slot ? __ldg(p.slot + it.i) : it.i;
+        it.u = p.slot ? __ldcg(p.slot + it.i) : it.i;           // index arrays through the L2: another kernel may have just written them
         const bool bad = it.u < 0 || it.u >= p.n_units;
         if (bad && lane == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
-        it.len = bad ? 0 : max(0, min(__ldg(p.len + it.u), p.cap));
+        it.len = bad ? 0 : max(0, min(__ldcg(p.len + it.u), p.cap));
         it.n_keys = p.row0 < it.len ? min(it.len, p.row0 + p.R) : 0;   // rows any query of this call can see
         it.kt_all = (it.n_keys + 15) >> 4;
         return it;

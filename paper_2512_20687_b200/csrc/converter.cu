@@ -101,33 +101,56 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    ptx::grid_dep_wait();                   // x may be the output of the kernel before this one
     ptx::grid_dep_launch();                 // at most one CTA per SM and one wave
 
     if (warp == 0) {
-        int s = 0;
-        uint32_t phase = 0;
-        for (int st = 0; st < n_steps; ++st) {
+        // The weights never come from the kernel before this one, x may: the ring's first turn requests
+        // its weight atoms at once, and its x atoms once the dependency wait has returned, so that the
+        // weight stream already runs under the tail of the predecessor.  Everything else this kernel does
+        // with global memory follows from x having landed.
+        auto load_w = [&](int st, int s) {
+            const int atoms = min(KA, n_atoms - st * KA);
+            const uint32_t full = bars + 16 * s;
+            const uint32_t b_dst = base + s * stage_bytes + KA * a_bytes;
+            for (int j = 0; j < atoms; ++j) {
+                const int k0 = (a_lo + st * KA + j) * BK;
+                if (!W_IN_MAJOR) {
+                    ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);       // W[n0.., k0..]  (K-major)
+                } else {
+#pragma unroll
+                    for (int jj = 0; jj < NT / 64; ++jj)                                 // W[k0.., n0+64jj..] (N-major)
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES + jj * (BK * 128), &tm_w, n0 + 64 * jj, k0, full);
+                }
+            }
+        };
+        auto load_x = [&](int st, int s) {
+            const int atoms = min(KA, n_atoms - st * KA);
+            const uint32_t a_dst = base + s * stage_bytes;
+            for (int j = 0; j < atoms; ++j)
+                ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, (a_lo + st * KA + j) * BK, m0, bars + 16 * s);   // x[m0.., k0..]
+        };
+        const int ahead = min(n_steps, n_stages);          // the ring starts empty: no stage to wait for
+        if (ptx::elect_one())
+            for (int st = 0; st < ahead; ++st) {
+                ptx::mbar_arrive_expect_tx(bars + 16 * st, min(KA, n_atoms - st * KA) * (a_bytes + T::B_BYTES));
+                load_w(st, st);
+            }
+        __syncwarp();
+        ptx::grid_dep_wait();               // x may be the output of the kernel before this one
+        if (ptx::elect_one())
+            for (int st = 0; st < ahead; ++st) load_x(st, st);
+        __syncwarp();
+        int s = ahead == n_stages ? 0 : ahead;
+        uint32_t phase = ahead == n_stages ? 1 : 0;
+        for (int st = ahead; st < n_steps; ++st) {
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(bars + 16 * s + 8, phase ^ 1))) {
                 if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
                 break;
             }
-            const int atoms = min(KA, n_atoms - st * KA);
-            const uint32_t full = bars + 16 * s;
-            const uint32_t a_dst = base + s * stage_bytes, b_dst = a_dst + KA * a_bytes;
             if (ptx::elect_one()) {
-                ptx::mbar_arrive_expect_tx(full, atoms * (a_bytes + T::B_BYTES));
-                for (int j = 0; j < atoms; ++j) {
-                    const int k0 = (a_lo + st * KA + j) * BK;
-                    ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, k0, m0, full);              // x[m0.., k0..]
-                    if (!W_IN_MAJOR) {
-                        ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);       // W[n0.., k0..]  (K-major)
-                    } else {
-#pragma unroll
-                        for (int jj = 0; jj < NT / 64; ++jj)                                 // W[k0.., n0+64jj..] (N-major)
-                            ptx::tma_load_2d(b_dst + j * T::B_BYTES + jj * (BK * 128), &tm_w, n0 + 64 * jj, k0, full);
-                    }
-                }
+                ptx::mbar_arrive_expect_tx(bars + 16 * s, min(KA, n_atoms - st * KA) * (a_bytes + T::B_BYTES));
+                load_x(st, s);
+                load_w(st, s);
             }
             __syncwarp();
             if (++s == n_stages) { s = 0; phase ^= 1; }
@@ -183,6 +206,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
         ok = ptx::mbar_wait(bar_acc, 0);
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
+        ptx::grid_dep_wait();               // long since over; these warps read the residual and write the output
     }
     if (ks > 1) ptx::cluster_sync();        // every CTA of the cluster is done with its ring
     if (epi) {
@@ -224,7 +248,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     uint32_t w[4];
-                    const uint4 rv = res ? res[v] : make_uint4(0u, 0u, 0u, 0u);
+                    const uint4 rv = res ? __ldcg(res + v) : make_uint4(0u, 0u, 0u, 0u);
                     const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {

@@ -122,7 +122,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         const int i = unit0 + r / G;
         int s = -1;
         if (r < upt * G && i < p.n_q) {
-            s = p.sh_id[i];
+            s = __ldcg(p.sh_id + i);
             if (s >= p.n_shared || s < 0) s = -1;
         }
         sid[r] = s;
@@ -145,7 +145,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
             const int i = unit0 + r / G;
             qv[t] = make_uint4(0u, 0u, 0u, 0u);
             if (idx < BM * (DH / 8) && r < upt * G && i < p.n_q)
-                qv[t] = __ldg(reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8));
+                qv[t] = __ldcg(reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8));
         }
 #pragma unroll
         for (int t = 0; t < QV; ++t) {
@@ -187,7 +187,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         bool ok = true;
         for (int cur = next_sid(-1); cur != 0x7FFFFFFF && ok; cur = next_sid(cur)) {
             int r0, r1;
-            part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
+            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
             const int row_base = (cur * p.Hkv + h) * p.cap_sh;
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int s = it % KV_STAGES;
@@ -212,7 +212,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         int n_tiles = 0;
         for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
             int r0, r1;
-            part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
+            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
             n_tiles += (r1 - r0 + BN - 1) / BN;
         }
         bool ok = true;
@@ -272,7 +272,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         // keep meeting at the named barrier; the results are then void and the status says so.
         for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
             int r0, r1;
-            part_range(max(0, min(p.sh_len[cur], p.cap_sh)), p.splits_sh, part, r0, r1);
+            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
             const bool active = (my_sid == cur);
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int b = it & 1, st = it % KV_STAGES;
