@@ -6,9 +6,12 @@
 A step is one pass of the whole hot path (append -> coarse attention ->
 converter -> chunk attention) over one batch of seeded synthetic input.  The
 metric is decode tokens/s = token-level in-flight chunks per step / step time.
-With N > 1 (launched by torchrun) every rank runs an independent replica of
-the same per-GPU batch (weak scaling, no data-path collective); time is the
-max over ranks.  Rank 0 prints ONE JSON line.
+With N > 1 every rank runs an independent replica of the same per-GPU batch
+(weak scaling, no data-path collective); time is the max over ranks.  Under
+torchrun the ranks are there already; started plainly with --gpus N > 1 the
+script starts them itself (torch.distributed.run on 127.0.0.1).  Rank 0 prints
+ONE JSON line.  The K timed steps are repeated a few times and the median
+repetition is reported.
 
 `--impl reference` times the CPU oracle (a deliberately plain fp64 program)
 on the host cores on a bounded sample of the same workload.
@@ -301,16 +304,21 @@ def run_gpu(args, cfg) -> None:
 
     uuid = str(torch.cuda.get_device_properties(dev).uuid)
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    pd.barrier()
-    torch.cuda.synchronize()
+    # the K steps are timed REPS times over (each repetition bracketed by a barrier and a synchronize on both
+    # sides, device time by CUDA events, max over ranks); the median repetition is the one reported
+    REPS = 5 if K <= 4096 else 3
+    secs = []
     sampler.start()
-    e0.record()
-    replay()
-    e1.record()
-    torch.cuda.synchronize()
-    pd.barrier()
-    sec = e0.elapsed_time(e1) * 1e-3
+    for _ in range(REPS):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pd.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        replay()
+        e1.record()
+        torch.cuda.synchronize()
+        pd.barrier()
+        secs.append(pd.reduce_max(e0.elapsed_time(e1) * 1e-3))
     clocks = sampler.stop()
     if clocks["samples"] < 3:                     # region too short to sample: repeat it untimed under the sampler
         sampler = ClockSampler(sampler.uuid)
@@ -322,7 +330,7 @@ def run_gpu(args, cfg) -> None:
         clocks = sampler.stop()
         clocks["note"] = "timed region shorter than the sampling period; sampled on an untimed repeat of it"
     assert ph.photon_device_status(ctx) == 0, "device status word set during the timed region"
-    sec_max = pd.reduce_max(sec)
+    sec_max = statistics.median(secs)
     tokens_total = pd.reduce_sum(cfg.tokens_per_step * K)
     value = tokens_total / sec_max
 
@@ -385,6 +393,99 @@ def run_gpu(args, cfg) -> None:
             parts[name]["frac_of_own_roofline"] = t_roof / us
     lens.copy_(lens0)
     torch.cuda.synchronize()
+    def time_calls(fns, replays=6):
+        """us per call of a CUDA graph that runs the given calls back to back, replayed `replays` times."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for fn in fns:
+                    fn()
+        g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(replays):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / (replays * len(fns))
+
+    def read_ceiling(nbytes):
+        """The read-ceiling probe of the library on buffers of nbytes (rotating, more than 3x L2 in all): a kernel with
+        the attention's launch, grid and ring that only brings the bytes into shared memory.  Best of three grids."""
+        nbytes -= nbytes % 16
+        n_buf = max(4, -(-3 * L2_BYTES // nbytes))
+        bufs = [torch.empty(nbytes, dtype=torch.uint8, device=dev).random_() for _ in range(n_buf)]
+        best = None
+        for ctas in (0, 2 * torch.cuda.get_device_properties(dev).multi_processor_count,
+                     torch.cuda.get_device_properties(dev).multi_processor_count):
+            us = time_calls([(lambda b=b, c=ctas: ph.photon_read_probe(ctx, b, nbytes, c)) for b in bufs * max(1, 32 // n_buf)])
+            if best is None or us < best["us"]:
+                best = {"us": us, "ctas": ctas}
+        del bufs
+        torch.cuda.empty_cache()
+        return best
+
+    def other_workload(idx):
+        """The dominant attention part of another of the target workloads, timed in this run the same way as `parts`
+        (its caches only feed a timing: drawn on the device from a fixed seed, lengths as in the workload)."""
+        oc = wl.CONFIGS[idx]
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(777 + idx)
+        octx = ph.photon_create(oc.Hq, oc.Hkv, oc.dh, oc.D, oc.P, oc.C, max(oc.B, oc.Nc), args.max_splits)
+        o_scale = oc.dh ** -0.5
+
+        def draw(*shape):
+            return torch.empty(*shape, dtype=torch.bfloat16, device=dev).normal_(generator=gen)
+
+        res = {}
+        if idx == 4:
+            # chunk attention over every in-flight chunk; lengths P + (in-chunk position + 1) as the workload draws them
+            ln = torch.from_numpy(wl.chunk_inputs(wl.scaled(oc, B=1))["len"][:oc.chunks_per_seq]).repeat(oc.B).to(dev)
+            cap = oc.P + oc.C
+            kc, vc = draw(oc.Nc, oc.Hkv, cap, oc.dh), draw(oc.Nc, oc.Hkv, cap, oc.dh)
+            qq = draw(oc.Nc, oc.Hq, oc.dh)
+            oo = torch.empty_like(qq)
+            kvc = ph.make_kv(kc, vc, ln.to(torch.int32))
+            nbytes = int(ln.sum().item()) * oc.Hkv * oc.dh * 4 + 2 * oc.Nc * oc.Hq * oc.dh * 2
+            us = time_calls([lambda: ph.photon_chunk_attn(octx, kvc, qq, None, oo, scale=o_scale)] * 8)
+            res = {"kernel": "chunk_attn", "l2": "one set of chunk buffers of %.0f MiB, larger than L2" % (nbytes / 2**20)}
+        else:
+            kvb = oc.B * oc.Hkv * oc.S * oc.dh * 4
+            n_rep = max(4, -(-3 * L2_BYTES // kvb))
+            k0, v0 = draw(oc.B, oc.Hkv, oc.S, oc.dh), draw(oc.B, oc.Hkv, oc.S, oc.dh)
+            ks, vs = [k0] + [k0.clone() for _ in range(n_rep - 1)], [v0] + [v0.clone() for _ in range(n_rep - 1)]
+            qq = draw(oc.B, oc.Hq, oc.dh)
+            oo = [torch.empty_like(qq) for _ in range(n_rep)]
+            ln = torch.full((oc.B,), oc.S, dtype=torch.int32, device=dev)
+            sh = {}
+            if oc.shared_S:
+                sh = dict(k_shared=draw(1, oc.Hkv, oc.shared_S, oc.dh), v_shared=draw(1, oc.Hkv, oc.shared_S, oc.dh),
+                          shared_len=torch.full((1,), oc.shared_S, dtype=torch.int32, device=dev),
+                          shared_id=torch.zeros(oc.B, dtype=torch.int32, device=dev))
+            kvs = [ph.make_kv(ks[r], vs[r], ln, max_len=oc.S, **sh) for r in range(n_rep)]
+            nbytes = wl.coarse_kv_bytes(oc) + 2 * oc.B * oc.Hq * oc.dh * 2
+            us = time_calls([(lambda r=r: ph.photon_coarse_attn(octx, kvs[r], qq, oo[r], None, o_scale))
+                             for r in list(range(n_rep)) * max(1, 32 // n_rep)])
+            res = {"kernel": "coarse_attn", "l2": "%d replicas of the cache, %.0f MiB in all" % (n_rep, n_rep * kvb / 2**20)}
+            if oc.shared_S:
+                flops = 4.0 * oc.B * oc.Hq * oc.shared_S * oc.dh
+                logical = oc.B * (oc.S + oc.shared_S) * oc.Hkv * oc.dh * 4
+                t_roof = max(nbytes / (hbm_peak * 1e3), flops / (tensor_peak * 1e6))
+                res.update({"prefix_flops": flops, "TFLOPs": flops / us * 1e-6, "frac_of_own_roofline": t_roof / us,
+                            "logical_GBps": logical / us * 1e-3,
+                            "note": "two launches (prefix contraction on the tensor cores, then the own keys); the prefix "
+                                    "is read once, so the HBM fraction of the physical bytes says little: the own roofline "
+                                    "is the slower of bytes / HBM peak and prefix flops / bf16 peak; logical = bytes a "
+                                    "cache with the prefix copied into every branch would read"})
+        bits_o = ph.photon_device_status(octx)
+        ph.photon_destroy(octx)
+        torch.cuda.empty_cache()
+        res.update({"workload": oc.name, "us": us, "algorithmic_bytes": nbytes, "GBps": nbytes / us * 1e-3,
+                    "frac": nbytes / us * 1e-3 / hbm_peak, "frac_of_nominal_8TBs": nbytes / us * 1e-3 / 8000.0,
+                    "device_status": bits_o})
+        return res
+
     parts["note"] = ("each part timed as a CUDA graph of back-to-back calls rotating over the replicas; "
                      "kv_append's figure includes a %d-int length reset every %d calls" % (cfg.B * R, R))
 
@@ -672,6 +773,24 @@ def run_gpu(args, cfg) -> None:
                 # the replicas are meant to keep the reads in HBM: less DRAM traffic than 95 % of the
                 # algorithmic bytes would mean the L2 served part of them
                 "l2_assisted": None if traffic is None else bool(traffic < 0.95 * kernels[dom]["bytes"])}
+    ceil = read_ceiling(kernels[dom]["bytes"])
+    roofline.update({"read_ceiling_us": ceil["us"], "read_ceiling_ctas": ceil["ctas"],
+                     "frac_of_read_ceiling": ceil["us"] / kernels[dom]["us"],
+                     "read_ceiling_note": "photon_read_probe on buffers of the same size: the attention's launch, grid and "
+                                          "ring of bulk copies with nothing computed (best of three grids)"})
+    # the dominant attention part of every target workload (configs 1-4), this run's own workload from `parts`
+    by_workload = {}
+    if not args.no_parts and not args.batch and not args.hierarchy:
+        for idx in (1, 2, 3, 4):
+            if idx == cfg.index:
+                pc = parts[dom]
+                by_workload[f"config{idx}"] = {"workload": cfg.name, "kernel": dom, "us": pc["us"],
+                                               "algorithmic_bytes": pc["algorithmic_bytes"], "GBps": pc["GBps"],
+                                               "frac": pc["frac_hbm"], "frac_of_nominal_8TBs": pc["GBps"] / 8000.0}
+            else:
+                by_workload[f"config{idx}"] = other_workload(idx)
+        by_workload["note"] = ("dominant attention part per target workload, CUDA graph of back-to-back calls on inputs larger "
+                               "than L2, fraction of the measured copy peak (%s) and of the nominal 8 TB/s" % peak_src)
     if cfg.shared_S and "coarse_attn" in parts:
         # a shared prefix makes the coarse attention a contraction over the prefix plus a stream over the own
         # rows: its own roofline is the slower of the two, and the bytes a cache without sharing would read
@@ -699,7 +818,7 @@ def run_gpu(args, cfg) -> None:
 
     # end to end through the public API with host buffers: every step its inputs (new K/V row, both
     # query tensors, the cache lengths) travel from pinned host memory to the device and its results
-    # (both attention outputs) travel back.  The inputs live in one host buffer and one device buffer
+    # (both attention outputs and the converter's prefix vectors U) travel back.  The inputs live in one host buffer and one device buffer
     # (the tensors are views into it), so a step is one H2D copy, the decode step and one D2H copy.
     def pack(tensors):
         offs, total = [], 0
@@ -718,36 +837,42 @@ def run_gpu(args, cfg) -> None:
         h_in[o:o + nb].copy_(t.cpu().contiguous().view(-1).view(torch.uint8))
         views.append(d_in[o:o + nb].view(t.dtype).view(t.shape))
     e_k_new, e_v_new, e_q, e_len, e_qc = views
-    out_src = [reps[0]["out"], reps[0]["oc"]]
-    out_offs, out_total = pack(out_src)
-    d_out = torch.empty(out_total, dtype=torch.uint8, device=dev)
-    h_out = torch.empty(out_total, dtype=torch.uint8).pin_memory()
-    e_out, e_oc = [d_out[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for t, o in zip(out_src, out_offs)]
-    h2d, d2h = in_total, out_total
     n_e2e = max(3, min(K, 2000))
-    e2e_args = []
-    for r in range(R):
-        t = reps[r]
-        kv_e = ph.make_kv(t["k"], t["v"], e_len, max_len=cfg.S, **shared)
-        e2e_args.append(ph.make_step_args(kv_e, e_k_new, e_v_new, e_q, e_out, scale, t["w"], layout, t["U"], cfg.B,
-                                          chunks=t["ckv"], q_chunk=e_qc, out_chunk=e_oc, Nc=cfg.Nc, scale_chunk=scale))
 
-    host_io = ph.HostIO(h_in, d_in, d_out, h_out, in_split=in_offs[4], out_split=out_offs[1])
+    def run_e2e(with_U):
+        """tokens/s of host-driven steps and the bytes that come back per step.  with_U: the converter's prefix
+        vectors travel to the host as well (they lie between the two attention outputs in the staging area)."""
+        out_src = [reps[0]["out"]] + ([reps[0]["U"]] if with_U else []) + [reps[0]["oc"]]
+        out_offs, out_total = pack(out_src)
+        d_out = torch.empty(out_total, dtype=torch.uint8, device=dev)
+        h_out = torch.empty(out_total, dtype=torch.uint8).pin_memory()
+        vs = [d_out[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for t, o in zip(out_src, out_offs)]
+        e_out, e_oc = vs[0], vs[-1]
+        e2e_args = []
+        for r in range(R):
+            t = reps[r]
+            kv_e = ph.make_kv(t["k"], t["v"], e_len, max_len=cfg.S, **shared)
+            e2e_args.append(ph.make_step_args(kv_e, e_k_new, e_v_new, e_q, e_out, scale, t["w"], layout,
+                                              vs[1] if with_U else t["U"], cfg.B, chunks=t["ckv"], q_chunk=e_qc,
+                                              out_chunk=e_oc, Nc=cfg.Nc, scale_chunk=scale))
+        host_io = ph.HostIO(h_in, d_in, d_out, h_out, in_split=in_offs[4], out_split=out_offs[-1])
+        # one call of the library per step: host -> staging, the decode step, staging -> host, wait for the stream
+        for i in range(max(3, min(300, n_e2e // 5))):  # the first few hundred host-driven steps of a process run slower
+            ph.photon_decode_step_host(ctx, e2e_args[i % R], host_io)
+        pd.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            ph.photon_decode_step_host(ctx, e2e_args[i % R], host_io)
+        torch.cuda.synchronize()
+        sec = pd.reduce_max(time.perf_counter() - t0)
+        lens.copy_(lens0)
+        torch.cuda.synchronize()
+        return pd.reduce_sum(cfg.tokens_per_step * n_e2e) / sec, out_total
 
-    def e2e_step(i):
-        # one call of the library: host -> staging, the decode step, staging -> host, wait for the stream
-        ph.photon_decode_step_host(ctx, e2e_args[i % R], host_io)
-
-    for i in range(max(3, min(300, n_e2e // 5))):      # the first few hundred host-driven steps of a process run slower
-        e2e_step(i)
-    pd.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for i in range(n_e2e):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    e2e_sec = pd.reduce_max(time.perf_counter() - t0)
-    e2e_val = pd.reduce_sum(cfg.tokens_per_step * n_e2e) / e2e_sec
+    h2d = in_total
+    e2e_val, d2h = run_e2e(False)
+    e2e_val_U, d2h_U = run_e2e(True)
     lens.copy_(lens0)
     torch.cuda.synchronize()
     bits = ph.photon_device_status(ctx)
@@ -763,9 +888,17 @@ def run_gpu(args, cfg) -> None:
                        w_layout=args.layout),
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": n_e2e, "note": "photon_decode_step_host: one pinned host buffer -> device (new K/V row, queries, lengths), decode step, both outputs -> host, wait, every step; the chunk attention's query and output cross the bus beside the coarse part where that attention runs on the side stream"},
+                "steps": n_e2e,
+                "note": "photon_decode_step_host: one pinned host buffer -> device (new K/V row, queries, lengths), decode step, "
+                        "both attention outputs -> host, wait, every step; the chunk attention's query and output cross the bus "
+                        "beside the coarse part where that attention runs on the side stream, the coarse output leaves beside "
+                        "the converter.  The converter's output U stays on the device in this figure: its consumers are the "
+                        "local decoders (photon_decoder_prefill reads it from device memory), no host code of a serving loop "
+                        "reads prefix vectors; with_converter_output is the same loop with U copied back as well",
+                "with_converter_output": {"value": e2e_val_U, "unit": UNIT, "d2h_bytes_per_step": d2h_U}},
         "gpu_launches": launches_per_step * K,
         "roofline": roofline,
+        "roofline_by_workload": by_workload,
         "us_per_step": sec_max * 1e6 / K,
         "step_hbm": {"algorithmic_bytes": step_bytes, "GBps": step_bytes / (sec_max / K) * 1e-9,
                      "frac": step_bytes / (sec_max / K) * 1e-9 / hbm_peak},
@@ -790,8 +923,22 @@ def run_gpu(args, cfg) -> None:
     pd.shutdown()
 
 
+def spawn_ranks(n: int, argv: list[str]) -> int:
+    """Starts n ranks of this script on this node (one per GPU) the way a launcher would, and returns their
+    exit code: what `bench.py --gpus N` does when nobody has started the ranks for it."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
 def main():
     args = parse()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "photon":
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     cfg = wl.CONFIGS[args.config]
     if args.batch and args.batch < cfg.B:
         cfg = wl.scaled(cfg, B=args.batch, tokens_per_step=cfg.tokens_per_step * args.batch // cfg.B)

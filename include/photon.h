@@ -332,8 +332,12 @@ photon_status photon_decode_step(photon_ctx *ctx, const photon_step_args *args, 
  *                      the coarse attention and the converter read; the rest is
  *                      read by the chunk attention only (q_chunk, slot).
  *   out_split          bytes [0, out_split) of the output are written by the
- *                      coarse attention (out_coarse, lse_coarse); the rest by the
- *                      chunk attention (out_chunk).
+ *                      coarse attention (out_coarse, lse_coarse) and, when the
+ *                      caller wants it on the host, by the converter (U, which
+ *                      then comes after the coarse attention's arrays: what
+ *                      precedes U leaves beside the converter, U and what
+ *                      follows it after the converter); the rest by the chunk
+ *                      attention (out_chunk).
  * With in_split == in_bytes and out_split == out_bytes everything is copied in
  * before the step and out after it.  Otherwise, when the chunk attention runs
  * on the context's side stream (see photon_decode_step), the two parts of a
@@ -355,9 +359,10 @@ photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *a
                                       void *host_out, size_t out_bytes, size_t out_split, photon_stream stream);
 
 /* Reads (and optionally clears) the device status word.  Synchronises the
- * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT also
- * puts the context's arrival tickets back to zero, so the context stays
- * usable after a kernel that gave up on a wait. */
+ * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT or a
+ * PHOTON_DEV_BAD_INDEX also puts the context's arrival tickets back to zero,
+ * so the context stays usable after a kernel that gave up on a wait or
+ * stopped at an index out of range. */
 photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t clear);
 
 /* The paper has no counterpart to this call: it exists for hosts that must not
@@ -392,6 +397,29 @@ photon_status photon_coarse_attn_noalloc(const photon_config *cfg, const photon_
  * cache is cut and merged by log-sum-exp; a smaller grid leaves SMs free for
  * work on another stream.  Takes effect from the next call. */
 photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n);
+
+/* Two measurement and test aids without a counterpart in the paper; neither is
+ * part of a decode step.
+ *
+ * photon_read_probe streams `bytes` (a multiple of 16) of device memory at the
+ * 16-byte aligned pointer src into shared memory and computes nothing: same
+ * launch, grid and ring of bulk copies as the coarse attention, so its time on
+ * a buffer of the size an attention call reads is the ceiling that call can be
+ * held against beside the HBM peak (tens of megabytes are bound by start-up
+ * and drain, not by bandwidth).  ctas: the grid, 0 = the attention's default.
+ * sum_out: device uint32 (or NULL) to which the kernel adds the sum, modulo
+ * 2^32, of the first little-endian 32-bit word of every 128 bytes it read; the
+ * caller clears it.  One kernel on `stream`.
+ *
+ * photon_wait_probe launches one thread that waits on a barrier nobody
+ * arrives at, gives up after limit_ns nanoseconds (at most 1e8), sets
+ * PHOTON_DEV_TIMEOUT, leaves one arrival ticket of the context non-zero (as a
+ * kernel that stopped half way would) and returns by itself.  It exists so
+ * that a test can see the path every bounded wait of the library takes when it
+ * runs out, and that photon_device_status(clear) leaves the context usable. */
+photon_status photon_read_probe(photon_ctx *ctx, const void *src, size_t bytes, int32_t ctas, uint32_t *sum_out,
+                                photon_stream stream);
+photon_status photon_wait_probe(photon_ctx *ctx, int64_t limit_ns, photon_stream stream);
 
 /* Number of kernels the library has launched through this context so far. */
 int64_t photon_launch_count(const photon_ctx *ctx);

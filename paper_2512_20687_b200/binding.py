@@ -126,6 +126,10 @@ def load() -> ctypes.CDLL:
     lib.photon_device_status.argtypes = [c_void_p, POINTER(c_int32), c_int32]
     lib.photon_set_attention_ctas.restype = st
     lib.photon_set_attention_ctas.argtypes = [c_void_p, c_int32]
+    lib.photon_read_probe.restype = st
+    lib.photon_read_probe.argtypes = [c_void_p, c_void_p, c_size_t, c_int32, c_void_p, c_void_p]
+    lib.photon_wait_probe.restype = st
+    lib.photon_wait_probe.argtypes = [c_void_p, c_int64, c_void_p]
     lib.photon_launch_count.restype = c_int64
     lib.photon_launch_count.argtypes = [c_void_p]
     lib.photon_status_str.restype = c_char_p
@@ -382,6 +386,18 @@ def photon_device_status(ctx, clear=True) -> int:
 
 def photon_set_attention_ctas(ctx, n: int) -> None:
     _check(load().photon_set_attention_ctas(ctx, int(n)), "photon_set_attention_ctas")
+
+
+def photon_read_probe(ctx, src, nbytes=None, ctas=0, sum_out=None, stream=None) -> None:
+    """Streams the first nbytes of the device tensor src through the attention kernels' kind of ring (see photon.h)."""
+    if nbytes is None:
+        nbytes = src.numel() * src.element_size()
+    _check(load().photon_read_probe(ctx, _ptr(src), c_size_t(int(nbytes)), int(ctas), _ptr(sum_out), _stream(stream)),
+           "photon_read_probe")
+
+
+def photon_wait_probe(ctx, limit_ns=1_000_000, stream=None) -> None:
+    _check(load().photon_wait_probe(ctx, c_int64(int(limit_ns)), _stream(stream)), "photon_wait_probe")
 
 
 def photon_launch_count(ctx) -> int:

@@ -178,6 +178,9 @@ cudaError_t launch_rope_split_append(const bf16 *qkv, int n, int Hq, int Hkv, in
 cudaError_t launch_swiglu(const bf16 *gu, bf16 *out, int n, int F, cudaStream_t st, long long *launches);
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st,
                              long long *launches);
+cudaError_t launch_read_probe(photon_ctx *ctx, const void *src, size_t bytes, int ctas, unsigned int *sum_out,
+                              cudaStream_t st, long long *launches);
+cudaError_t launch_wait_probe(photon_ctx *ctx, unsigned long long limit_ns, cudaStream_t st, long long *launches);
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }

@@ -562,13 +562,18 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse, a->scale_coarse, stream);
     if (s == PHOTON_OK && a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;
+    // What the coarse attention wrote leaves beside the converter.  Where the converter's own output lies in the
+    // coarse part of the staging area, it and whatever follows it there leave after the converter.
+    size_t early_end = hp ? hp->out_split : 0;
+    if (hp && inside(a->U, (size_t)a->B * c.P * c.D * sizeof(photon_bf16), hp->dev_out, 0, hp->out_split))
+        early_end = (size_t)(reinterpret_cast<const char *>(a->U) - hp->dev_out);
     bool copying = false;
-    if (s == PHOTON_OK && (apart || direct) && hp->out_split > 0) {
+    if (s == PHOTON_OK && (apart || direct) && early_end > 0) {
         if (cudaEventRecord(ctx->ev_mid, st) != cudaSuccess || cudaStreamWaitEvent(ctx->copy, ctx->ev_mid, 0) != cudaSuccess)
             s = PHOTON_ERR_CUDA;
         else {
             copying = true;
-            if (!copy_out(hp, 0, hp->out_split, ctx->copy)) s = PHOTON_ERR_CUDA;
+            if (!copy_out(hp, 0, early_end, ctx->copy)) s = PHOTON_ERR_CUDA;
             if (cudaEventRecord(ctx->ev_copy, ctx->copy) != cudaSuccess) s = PHOTON_ERR_CUDA;
         }
     }
@@ -580,7 +585,8 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         s = photon_chunk_attn(ctx, a->chunks, q_chunk, slot, out_chunk, a->Nc, a->scale_chunk, stream);
     }
     if (copying && cudaStreamWaitEvent(st, ctx->ev_copy, 0) != cudaSuccess && s == PHOTON_OK) s = PHOTON_ERR_CUDA;
-    if (s == PHOTON_OK && hp && !copying && !copy_out(hp, 0, apart || direct ? hp->out_split : hp->out_bytes, st)) s = PHOTON_ERR_CUDA;
+    if (s == PHOTON_OK && hp && !copy_out(hp, copying ? early_end : 0, apart || direct ? hp->out_split : hp->out_bytes, st))
+        s = PHOTON_ERR_CUDA;
     return s;
 }
 }  // namespace
@@ -618,11 +624,25 @@ photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t c
     if (cudaMemcpy(bits_out, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
         return PHOTON_ERR_CUDA;
     if (clear && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return PHOTON_ERR_CUDA;
-    // a kernel that gave up on a wait may have left arrival tickets behind; they must read zero again
-    if (clear && (*bits_out & PHOTON_DEV_TIMEOUT) &&
+    // a kernel that gave up on a wait, or stopped at an index that was out of range, may have left arrival
+    // tickets behind; they must read zero again
+    if (clear && (*bits_out & (PHOTON_DEV_TIMEOUT | PHOTON_DEV_BAD_INDEX)) &&
         cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess)
         return PHOTON_ERR_CUDA;
     return PHOTON_OK;
+}
+
+photon_status photon_read_probe(photon_ctx *ctx, const void *src, size_t bytes, int32_t ctas, uint32_t *sum_out,
+                                photon_stream stream) {
+    if (!ctx || ctas < 0 || (bytes && !src) || !aligned16(src) || bytes % 16 != 0) return PHOTON_ERR_INVALID_ARG;
+    const cudaError_t e = launch_read_probe(ctx, src, bytes, ctas, sum_out, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+}
+
+photon_status photon_wait_probe(photon_ctx *ctx, int64_t limit_ns, photon_stream stream) {
+    if (!ctx || limit_ns < 0 || limit_ns > 100000000) return PHOTON_ERR_INVALID_ARG;       // a tenth of a second at most
+    const cudaError_t e = launch_wait_probe(ctx, (unsigned long long)limit_ns, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
 }
 
 int64_t photon_launch_count(const photon_ctx *ctx) { return ctx ? ctx->launches : 0; }

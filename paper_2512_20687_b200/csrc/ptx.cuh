@@ -39,16 +39,16 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after about two seconds and returns false.  Every
-// wait in this library goes through here, so no kernel can spin for ever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after limit_ns (about two seconds unless the caller says otherwise) and
+// returns false.  Every wait in this library goes through here, so no kernel can spin for ever.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 1024; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (globaltimer_ns() - t0 > 2000000000ull) return false;
+        if (globaltimer_ns() - t0 > limit_ns) return false;
     }
 }
 __device__ __forceinline__ void fence_proxy_async() {
@@ -64,26 +64,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, 
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-// The same load with an L2 eviction policy for the lines it touches (from l2_policy_evict_first()).
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *m, int x, int y, uint32_t bar,
-                                                 uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
-}
-// Policy for data that is read once: its lines are the first to leave the L2.
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-// Asks the L2 to fetch `bytes` (a multiple of 16) from the 16-byte aligned global address `src`.  Nothing
-// reaches the SM: the L2 is the point of coherence, so the request is safe before the data's final value
-// is known to be written, and a later load finds the line there or on its way.
-__device__ __forceinline__ void l2_prefetch(const void *src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
 }
 
 // Untiled bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16 bytes.

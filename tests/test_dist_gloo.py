@@ -43,3 +43,21 @@ def test_two_gloo_ranks_reduce_time_by_max_and_units_by_sum():
     assert [(r[1], r[2]) for r in res] == [(0, 51), (51, 101)]
     for r in res:
         assert r[3] == 2.0 and r[4] == 101.0 and abs(r[5] - 101.0 / 2.0) < 1e-12
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`bench.py --gpus N` started plainly launches N ranks of itself; here through the CPU arm of the script
+    (the oracle on the tiny workload), which rank 0 alone runs while the other rank exits 0: one JSON line,
+    and it names both ranks."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import sys, bench; sys.exit(bench.spawn_ranks(2, ['--impl', 'reference', '--gpus', '2', '--config', '0', "
+            "'--steps', '1', '--warmup', '0']))")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["value"] > 0

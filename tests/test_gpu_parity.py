@@ -102,7 +102,7 @@ def test_level1_cache_of_hierarchical_generation(oracle):
     assert np.abs(lse - want_lse).max() < 2e-3
 
 
-@pytest.mark.parametrize("n_ctas", [1, 2, 3, 7, 37, 101, 0])
+@pytest.mark.parametrize("n_ctas", [1, 2, 3, 7, 37, 101, 259, 296, 0])
 def test_grid_size_and_cut_points_do_not_change_the_result(oracle, n_ctas):
     """Ragged lengths incl. 0 and 1; the grid size moves the points where caches
     are cut and merged (one CTA: no cut at all; many: most units cut, some CTAs idle)."""
@@ -145,9 +145,14 @@ def test_coarse_attention_other_group_sizes(oracle, G, dh):
     assert np.abs(lse - want_lse).max() < 2e-3
 
 
-def test_shared_prefix_variants(oracle):
+# group sizes and head sizes the shared-prefix kernel accepts: a row tile of 128 query rows holds 128 / G units
+# (126 of its rows are used for G = 3); the batch is never a whole number of tiles
+@pytest.mark.parametrize("max_splits", [1, 0])
+@pytest.mark.parametrize("G,dh,B", [(4, 128, 37), (1, 64, 150), (2, 128, 75), (3, 64, 50), (8, 128, 21), (16, 64, 13)])
+def test_shared_prefix_variants(oracle, G, dh, B, max_splits):
     """Two shared segments of different length, units without a prefix, empty own caches."""
-    cfg = cfg_small(3, B=37, S=40, shared_S=300)
+    Hkv = 4 if G == 4 else 2
+    cfg = cfg_small(3, B=B, S=40, shared_S=300, Hq=G * Hkv, Hkv=Hkv, dh=dh, D=G * Hkv * dh)
     co = wl.coarse_inputs(cfg, poison=True)
     ks = wl.normal_bf16(3, "ks2", (2, cfg.Hkv, 300, cfg.dh))
     vs = wl.normal_bf16(3, "vs2", (2, cfg.Hkv, 300, cfg.dh))
@@ -163,10 +168,10 @@ def test_shared_prefix_variants(oracle):
     scale = cfg.dh ** -0.5
     want, want_lse = oracle.attention(co["q"], co["k"], co["v"], lens, scale, shared=shared_of(co),
                                       n_threads=NT)
-    with Ctx(cfg) as c:
+    with Ctx(cfg, max_splits=max_splits) as c:
         got, lse, _ = run_coarse(c, co, scale)
         assert c.status() == 0
-    assert_close(got, want, "shared prefix")
+    assert_close(got, want, f"shared prefix G={G} dh={dh} splits={max_splits}")
     empty = (lens == 0) & (sh_id < 0)
     assert empty.any() and np.all(got[empty] == 0) and np.all(np.isneginf(lse[empty]))
     fin = np.isfinite(want_lse)
@@ -492,6 +497,46 @@ def test_decode_step_chain_matches_oracle(oracle, idx, layout):
         assert_close(host_f64(U), r["U"], "step: U")
         assert_close(host_f64(oc), r["chunk_out"], "step: chunk out")
         assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
+
+
+@pytest.mark.parametrize("idx", [2, 3, 4])
+def test_decode_step_chain_at_full_size(oracle, idx):
+    """The step as the benchmark times it on the long-context, shared-prefix and chunk-parallel workloads: one
+    call at full size.  The append is checked in full and bit for bit, the coarse attention in full; of the
+    converter and the chunk attention the oracle recomputes a seeded sample of rows / chunks (every row of U
+    depends on its own latent only, every chunk on its own buffer only)."""
+    cfg = wl.CONFIGS[idx]
+    s = wl.step_inputs(cfg, poison=True)
+    co, cv, chk = s["coarse"], s["converter"], s["chunks"]
+    scale = cfg.dh ** -0.5
+    rng = np.random.default_rng(40 + idx)
+    rows = np.sort(rng.choice(cfg.B, min(cfg.B, 24), replace=False))
+    pick = np.sort(rng.choice(cfg.Nc, min(cfg.Nc, 400), replace=False)).astype(np.int32)
+    pick[0], pick[-1] = 0, cfg.Nc - 1
+    with Ctx(cfg) as c:
+        d, dc = coarse_to_dev(co), chunks_to_dev(chk)
+        out = torch.empty_like(d["q"])
+        lse = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device="cuda")
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        oc = torch.empty_like(dc["q"])
+        args = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out, scale, dev_bf16(cv["w_out_major"]),
+                                 ph.PHOTON_W_OUT_MAJOR, U, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc,
+                                 Nc=cfg.Nc, scale_chunk=scale, lse_coarse=lse)
+        ph.photon_decode_step(c.h, args)
+        assert c.status() == 0
+        assert oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"]) == 0
+        assert np.array_equal(host_bits(d["k"]), co["k"]) and np.array_equal(host_bits(d["v"]), co["v"])
+        assert np.array_equal(d["len"].cpu().numpy(), co["len"])
+        want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, shared=shared_of(co),
+                                          n_threads=NT)
+        assert_close(host_f64(out), want, f"step cfg{idx}: coarse out")
+        assert np.abs(lse.cpu().numpy() - want_lse).max() < 2e-3
+        x = oracle.round_bf16(want).reshape(cfg.B, -1)[rows]
+        want_U = oracle.converter(x, cv["w_out_major"], None, w_out_major=True, n_threads=NT)
+        assert_close(host_f64(U)[rows], want_U.reshape(len(rows), cfg.P, cfg.D), f"step cfg{idx}: U rows")
+        want_c, _ = oracle.chunk_attention(chk["q"][pick], chk["kc"], chk["vc"], chk["len"], scale, slot=pick,
+                                           n_threads=NT)
+        assert_close(host_f64(oc)[pick], want_c, f"step cfg{idx}: chunk sample")
 
 
 # chunk attention beside the coarse part with little / with more than 1 MiB to move, and in line after it

@@ -1,6 +1,7 @@
 """photon_coarse_attn_noalloc: the context-free coarse attention for callers that cannot allocate
 device memory (its workspace is an array inside the library image).  Called through the C boundary
-twice in a row and compared with photon_coarse_attn on the same inputs.  Collected last on purpose."""
+twice in a row and compared with photon_coarse_attn and with the CPU oracle on the same inputs.
+Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
@@ -24,7 +25,7 @@ def _inputs(seed_shift):
     return cfg, co
 
 
-def test_no_alloc_entry_point_matches_the_context_one_twice_in_a_row():
+def test_no_alloc_entry_point_matches_the_context_one_twice_in_a_row(oracle):
     for call in range(2):                                  # second call finds the first one's leftovers
         cfg, co = _inputs(call)
         scale = cfg.dh ** -0.5
@@ -46,6 +47,37 @@ def test_no_alloc_entry_point_matches_the_context_one_twice_in_a_row():
         fin = np.isfinite(b)
         assert np.abs(a[fin] - b[fin]).max() < 2e-3
         assert np.all(host_f64(got)[1] == 0)               # the empty unit
+        ref, ref_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, n_threads=16)
+        assert_close(host_f64(got), ref, f"no-alloc call {call} against the oracle")
+        assert np.abs(a[fin] - ref_lse[fin]).max() < 2e-3
+
+
+def test_no_alloc_entry_point_allocates_nothing_and_takes_wide_groups(oracle):
+    """Sixteen query heads per KV head of 64 features and one long unit among short ones, so that many CTAs
+    hold a piece of the same cache and both partial slots of a CTA are in use; the status word is the one
+    inside the array (dev_status = None).  Once the first call has looked up the array, a call leaves the
+    device's free memory and torch's own counters where they were."""
+    Hkv, G, dh = 2, 16, 64
+    cfg = wl.scaled(wl.CONFIGS[1], B=6, S=6000, Hq=G * Hkv, Hkv=Hkv, dh=dh, D=G * Hkv * dh, seed=321)
+    co = wl.coarse_inputs(cfg, poison=True)
+    lens = np.array([5999, 3, 70, 0, 129, 640], np.int32)
+    for u, n in enumerate(lens):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0x7FC1
+    co["len"] = lens
+    scale = dh ** -0.5
+    d = coarse_to_dev(co)
+    got = torch.empty_like(d["q"])
+    ph.photon_coarse_attn_noalloc(cfg.Hq, Hkv, dh, d["kv"], d["q"], got, None, scale)      # looks the array up
+    torch.cuda.synchronize()
+    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    got.fill_(7.0)
+    ph.photon_coarse_attn_noalloc(cfg.Hq, Hkv, dh, d["kv"], d["q"], got, None, scale)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    want, _ = oracle.attention(co["q"], co["k"], co["v"], lens, scale, n_threads=16)
+    assert_close(host_f64(got), want, "no-alloc, G = 16, dh = 64")
 
 
 def test_no_alloc_entry_point_rejects_sizes_beyond_its_array():
