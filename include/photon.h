@@ -358,6 +358,16 @@ photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *a
                                       void *dev_in, size_t in_bytes, size_t in_split, const void *dev_out,
                                       void *host_out, size_t out_bytes, size_t out_split, photon_stream stream);
 
+/* Two host-side habits of photon_decode_step_host, both found by measurement on
+ * one machine and therefore adjustable per context: pause_ns (default 1500, at
+ * most 1e6, 0 = none) is how long the call waits between enqueuing its first
+ * host-to-device copy and its first kernel launch (launches that follow the
+ * copy within a microsecond made the whole step end later there); poll_us
+ * (default 2000, at most 1e7, 0 = block at once) is how long the call polls
+ * the stream for the step's end before it falls back to a blocking wait.
+ * Neither changes what the step computes. */
+photon_status photon_set_host_step_tuning(photon_ctx *ctx, int64_t pause_ns, int64_t poll_us);
+
 /* Reads (and optionally clears) the device status word.  Synchronises the
  * whole device; the only call that does.  Clearing a PHOTON_DEV_TIMEOUT or a
  * PHOTON_DEV_BAD_INDEX also puts the context's arrival tickets back to zero,

@@ -130,6 +130,8 @@ def load() -> ctypes.CDLL:
     lib.photon_read_probe.argtypes = [c_void_p, c_void_p, c_size_t, c_int32, c_void_p, c_void_p]
     lib.photon_wait_probe.restype = st
     lib.photon_wait_probe.argtypes = [c_void_p, c_int64, c_void_p]
+    lib.photon_set_host_step_tuning.restype = st
+    lib.photon_set_host_step_tuning.argtypes = [c_void_p, c_int64, c_int64]
     lib.photon_launch_count.restype = c_int64
     lib.photon_launch_count.argtypes = [c_void_p]
     lib.photon_status_str.restype = c_char_p
@@ -398,6 +400,11 @@ def photon_read_probe(ctx, src, nbytes=None, ctas=0, sum_out=None, stream=None) 
 
 def photon_wait_probe(ctx, limit_ns=1_000_000, stream=None) -> None:
     _check(load().photon_wait_probe(ctx, c_int64(int(limit_ns)), _stream(stream)), "photon_wait_probe")
+
+
+def photon_set_host_step_tuning(ctx, pause_ns: int = 1500, poll_us: int = 2000) -> None:
+    _check(load().photon_set_host_step_tuning(ctx, c_int64(int(pause_ns)), c_int64(int(poll_us))),
+           "photon_set_host_step_tuning")
 
 
 def photon_launch_count(ctx) -> int:

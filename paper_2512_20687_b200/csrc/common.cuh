@@ -43,6 +43,8 @@ struct photon_ctx {
     long long launches;
     cudaStream_t side;       // lowest-priority stream for the chunk attention of a decode step
     cudaEvent_t ev_fork, ev_join;
+    long long host_pause_ns; // photon_decode_step_host: pause between the first host-to-device copy and the first launch
+    long long host_poll_us;  // photon_decode_step_host: how long the call polls the stream before it blocks on it
     cudaStream_t copy;       // carries the coarse results to the host beside the converter (photon_decode_step_host)
     cudaEvent_t ev_mid, ev_copy;
     TmapCache tmaps;

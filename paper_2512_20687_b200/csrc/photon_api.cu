@@ -132,6 +132,8 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
     ctx->n_tickets = size_t(c.max_queries) * c.Hkv;
     ctx->max_ctas = ctx->sm_count * coarse_attn_ctas_per_sm();
     ctx->attn_ctas = 0;
+    ctx->host_pause_ns = 1500;
+    ctx->host_poll_us = 2000;
     if (cudaMalloc(&ctx->partials, ctx->partial_floats * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->cta_partials, size_t(2) * ctx->max_ctas * 16 * (c.dh + 2) * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->tickets, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
@@ -538,11 +540,12 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     }
     if (hp) {
         if (!copy_in(hp, 0, apart || direct ? hp->in_split : hp->in_bytes, st)) return PHOTON_ERR_CUDA;
-        if (hp->in_bytes) {
-            // Measured: launches enqueued within a microsecond of the copy make the whole step finish about 5 us later
-            // than launches that follow 1.5 us behind it (a stream query in between does not help, a pause does).
+        if (hp->in_bytes && ctx->host_pause_ns > 0) {
+            // Measured on one host: launches enqueued within a microsecond of the copy make the whole step finish about
+            // 5 us later than launches that follow 1.5 us behind it (a stream query in between does not help, a pause
+            // does).  The length of the pause is the context's (photon_set_host_step_tuning; 0 switches it off).
             const auto g0 = std::chrono::steady_clock::now();
-            while (std::chrono::steady_clock::now() - g0 < std::chrono::nanoseconds(1500)) {}
+            while (std::chrono::steady_clock::now() - g0 < std::chrono::nanoseconds(ctx->host_pause_ns)) {}
         }
     }
     if (beside) {
@@ -607,11 +610,12 @@ photon_status photon_decode_step_host(photon_ctx *ctx, const photon_step_args *a
     const photon_status s = step_impl(ctx, args, stream, &hp);
     if (s != PHOTON_OK) return s;
     // a step is tens of microseconds: poll for its end (a blocking wait pays a wake-up of several microseconds),
-    // and hand over to the blocking wait when the stream turns out to hold much more work than that
+    // and hand over to the blocking wait when the stream turns out to hold much more work than that (how long to
+    // poll is the context's: photon_set_host_step_tuning; 0 blocks at once)
     const auto t0 = std::chrono::steady_clock::now();
     cudaError_t e;
     while ((e = cudaStreamQuery(st)) == cudaErrorNotReady)
-        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(2)) {
+        if (std::chrono::steady_clock::now() - t0 >= std::chrono::microseconds(ctx->host_poll_us)) {
             e = cudaStreamSynchronize(st);
             break;
         }
@@ -650,6 +654,13 @@ int64_t photon_launch_count(const photon_ctx *ctx) { return ctx ? ctx->launches 
 photon_status photon_set_attention_ctas(photon_ctx *ctx, int32_t n) {
     if (!ctx || n < 0) return PHOTON_ERR_INVALID_ARG;
     ctx->attn_ctas = (n <= 0 || n > ctx->max_ctas) ? 0 : n;
+    return PHOTON_OK;
+}
+
+photon_status photon_set_host_step_tuning(photon_ctx *ctx, int64_t pause_ns, int64_t poll_us) {
+    if (!ctx || pause_ns < 0 || pause_ns > 1000000 || poll_us < 0 || poll_us > 10000000) return PHOTON_ERR_INVALID_ARG;
+    ctx->host_pause_ns = pause_ns;
+    ctx->host_poll_us = poll_us;
     return PHOTON_OK;
 }
 
