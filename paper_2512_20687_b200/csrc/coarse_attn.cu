@@ -62,7 +62,7 @@ __host__ __device__ inline int q_slot_bytes(int G, int dh) { return (G * dh * 2 
 
 template <int DH>
 size_t smem_bytes(int G) {
-    return 1024 /*alignment slack*/ + size_t(STAGES) * (Ring<DH>::STAGE_BYTES + q_slot_bytes(G, DH)) +
+    return size_t(STAGES) * (Ring<DH>::STAGE_BYTES + q_slot_bytes(G, DH) + 2 * DH * 2 /*a new K and V row*/) +
            size_t(NW) * G * (DH + 2) * sizeof(float) + 128 /*barriers*/ + 128 /*scalars*/ + NLEN * sizeof(int);
 }
 
@@ -72,7 +72,13 @@ __device__ __forceinline__ int tiles_of(int len) { return (len + BN - 1) / BN; }
 // Index arrays (lengths, page ids, prefix ids) are read through the L2 only: another kernel may have
 // written them just before this one, and a line of them left in an SM's L1 by an earlier kernel is not
 // refreshed by a dependent launch.
-__device__ __forceinline__ int ld_len(const AttnParams &p, int u) { return clamp_len(__ldcg(p.len + u), p.cap); }
+//
+// A length is kept as it was read, clamped to [-1, cap] (-1: any negative value).  With the step's append
+// folded into this kernel (p.k_new set) a unit with room grows by the one row the kernel itself installs:
+// the keys it attends are those of the grown cache.
+__device__ __forceinline__ int ld_len(const AttnParams &p, int u) { return max(-1, min(__ldcg(p.len + u), p.cap)); }
+__device__ __forceinline__ bool appends(const AttnParams &p, int raw) { return p.k_new && raw >= 0 && raw < p.cap; }
+__device__ __forceinline__ int eff_len(const AttnParams &p, int raw) { return appends(p, raw) ? raw + 1 : max(raw, 0); }
 
 constexpr int LPT = NLEN / THREADS;        // lengths per thread when a batch fits the shared-memory copy
 static_assert(NLEN % THREADS == 0, "a thread's units must fit its registers");
@@ -82,7 +88,7 @@ __device__ __forceinline__ void load_lengths(const AttnParams &p, int ub, int ue
 #pragma unroll
     for (int i = 0; i < LPT; ++i) len[i] = ub + i < ue ? __ldcg(p.len + ub + i) : 0;
 #pragma unroll
-    for (int i = 0; i < LPT; ++i) len[i] = clamp_len(len[i], p.cap);
+    for (int i = 0; i < LPT; ++i) len[i] = max(-1, min(len[i], p.cap));
 }
 
 // A CTA's part of the tile sequence.
@@ -97,14 +103,17 @@ struct Share {
 // [0, NLEN) sit in shared memory, read once per CTA; those of later units come from the L2.
 struct Walker {
     int u, h, j, nt, len;
+    bool app;                // the unit's last row is the one this kernel installs
     const int *slen;
     __device__ __forceinline__ void load(const AttnParams &p) {
-        len = u < NLEN ? slen[u] : ld_len(p, u);
+        const int raw = u < NLEN ? slen[u] : ld_len(p, u);
+        len = eff_len(p, raw);
+        app = appends(p, raw);
         nt = tiles_of(len);
     }
     // false: the share does not start at a tile of unit u0 (the lengths changed under the kernel)
     __device__ __forceinline__ bool start(const AttnParams &p, const Share &sh, const int *lens) {
-        slen = lens; u = sh.u0; h = 0; j = 0; nt = 0; len = 0;
+        slen = lens; u = sh.u0; h = 0; j = 0; nt = 0; len = 0; app = false;
         if (u < 0 || u >= p.n_units) return false;
         load(p);
         if (nt == 0 || sh.rem < 0 || sh.rem >= nt * p.Hkv) return false;
@@ -118,7 +127,7 @@ struct Walker {
         if (++h < p.Hkv) return;
         h = 0;
         do {
-            if (++u >= p.n_units) { u = p.n_units; nt = 0; len = 0; return; }
+            if (++u >= p.n_units) { u = p.n_units; nt = 0; len = 0; app = false; return; }
             load(p);
         } while (nt == 0);
     }
@@ -309,7 +318,7 @@ __device__ __forceinline__ void process_block(uint32_t kt, uint32_t vt, int kb, 
 // cut.  sc: [0..5] warp sums, [8] u0, [9] rem, [12] t0, [14] t1.
 __device__ __forceinline__ Share deal(const AttnParams &p, int *sc, int *slen, int cta) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    auto len_of = [&](int u) { return u < NLEN ? slen[u] : ld_len(p, u); };
+    auto len_of = [&](int u) { return eff_len(p, u < NLEN ? slen[u] : ld_len(p, u)); };
     const int per = (p.n_units + THREADS - 1) / THREADS;
     const int ub = min(p.n_units, (int)threadIdx.x * per), ue = min(p.n_units, ub + per);
     int mine = 0;
@@ -318,12 +327,12 @@ __device__ __forceinline__ Share deal(const AttnParams &p, int *sc, int *slen, i
         load_lengths(p, ub, ue, len);
 #pragma unroll
         for (int i = 0; i < LPT; ++i)
-            if (ub + i < ue) { slen[ub + i] = len[i]; mine += tiles_of(len[i]); }
+            if (ub + i < ue) { slen[ub + i] = len[i]; mine += tiles_of(eff_len(p, len[i])); }
     } else {
         for (int u = ub; u < ue; ++u) {
             const int len = ld_len(p, u);
             if (u < NLEN) slen[u] = len;
-            mine += tiles_of(len);
+            mine += tiles_of(eff_len(p, len));
         }
     }
     int incl = mine;
@@ -405,13 +414,15 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_k_end, const __grid_constant__ CUtensorMap tm_v_end) {
     using R = Ring<DH>;
     constexpr int NT8 = GP > 8 ? 2 : 1;
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];      // the swizzled tiles want 1024-byte alignment
     const int G = p.Hq / p.Hkv;
     const int QB = q_slot_bytes(G, DH);
-    const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
+    constexpr int NB = 2 * DH * 2;                              // a new K row and a new V row
+    const uint32_t base = ptx::smem_u32(smem_raw);
+    uint8_t *gen = smem_raw;
     const uint32_t q_base = base + STAGES * R::STAGE_BYTES;
-    float *red = reinterpret_cast<float *>(gen + STAGES * (R::STAGE_BYTES + QB));      // [NW][G][DH + 2]
+    const uint32_t n_base = q_base + STAGES * QB;               // per stage: the row a folded-in append installs
+    float *red = reinterpret_cast<float *>(gen + STAGES * (R::STAGE_BYTES + QB + NB));  // [NW][G][DH + 2]
     uint8_t *tail = reinterpret_cast<uint8_t *>(red) + (size_t)NW * G * (DH + 2) * sizeof(float);
     const uint32_t bars = ptx::smem_u32(tail);                  // full[s] at +16s, empty[s] at +16s+8
     const uint32_t red_full = bars + 16 * STAGES, red_empty = red_full + 8;
@@ -422,6 +433,10 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
+    if (base & 1023u) {                                         // never expected: the ring would be misplaced
+        if (threadIdx.x == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -462,7 +477,7 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
 #pragma unroll
         for (int i = 0; i < LPT; ++i)
             if (ub + i < ue) {
-                diff |= (tiles_of(len[i]) != tiles_of(slen[ub + i]));
+                diff |= (tiles_of(eff_len(p, len[i])) != tiles_of(eff_len(p, slen[ub + i])));
                 slen[ub + i] = len[i];
             }
         redo = __syncthreads_or(diff);
@@ -477,11 +492,32 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     const long long T = sh.T, t0 = sh.t0, t1 = sh.t1;
     const int n_cta = sh.n_cta;
 
+    // ---- a folded-in append: from here on this CTA reads lengths from shared memory only (the host takes
+    // this path for batches of at most NLEN units), and says so on a counter; the CTA that finds every
+    // other one already there writes the grown lengths, and flags the units that had no room, with the
+    // checks of the append kernel.  Its finishing warp does that while the first tiles are on their way.
+    if (p.k_new && warp == NW + 1) {
+        int last = 0;
+        if (lane == 0) {
+            last = (atomicAdd(p.readers, 1) == (int)gridDim.x - 1);
+            if (last) *p.readers = 0;                          // zero again for the next call
+        }
+        if (__shfl_sync(0xffffffffu, last, 0)) {
+            bool full = false;
+            for (int u = lane; u < p.n_units; u += 32) {
+                const int raw = slen[u];
+                if (appends(p, raw)) p.len_w[u] = raw + 1;
+                else full = true;
+            }
+            if (full) atomicOr(p.status, PHOTON_DEV_CAPACITY);
+        }
+    }
+
     // ---- units without own keys are visited by no tile: they are finished by whoever has time for it
     // (the whole CTA when it has no tiles, else the finishing warp before its first stream arrives)
     auto finish_empty_units = [&](int tid, int nthreads) {
         for (int u = cta; u < p.n_units; u += gridDim.x) {
-            if ((u < NLEN ? slen[u] : ld_len(p, u)) != 0) continue;
+            if (eff_len(p, u < NLEN ? slen[u] : ld_len(p, u)) != 0) continue;
             for (int idx = tid; idx < p.Hq * DH; idx += nthreads)
                 emit<DH>(p, u, idx / DH, idx % DH, 0.f, -CUDART_INF_F, 0.f);
         }
@@ -643,7 +679,9 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 // a tile of more than BOX rows comes as one box of BN rows per 64 features (what lies past the end
                 // of the cache is never used), a shorter one as one box of BOX rows
                 const bool tall = rows > BOX;
-                ptx::mbar_arrive_expect_tx(full, R::HALVES * (tall ? HALF_BYTES : BOX_BYTES) * 2 + (first ? G * DH * 2 : 0));
+                const bool grows = w.app && w.j == w.nt - 1;    // the row this kernel installs lies in this tile
+                ptx::mbar_arrive_expect_tx(full, R::HALVES * (tall ? HALF_BYTES : BOX_BYTES) * 2 + (first ? G * DH * 2 : 0) +
+                                                     (grows ? NB : 0));
 #pragma unroll
                 for (int hh = 0; hh < R::HALVES; ++hh) {
                     ptx::tma_load_2d(kd + hh * HALF_BYTES, tall ? &tm_k : &tm_k_end, hh * 64, y, full);
@@ -651,6 +689,11 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 }
                 if (first)
                     ptx::bulk_load(q_base + s * QB, p.q + ((size_t)w.u * p.Hq + (size_t)w.h * G) * DH, G * DH * 2, full);
+                if (grows) {
+                    const size_t at = ((size_t)w.u * p.Hkv + w.h) * DH;                   // k_new, v_new: [n_units, Hkv, dh]
+                    ptx::bulk_load(n_base + s * NB, p.k_new + at, DH * 2, full);
+                    ptx::bulk_load(n_base + s * NB + DH * 2, p.v_new + at, DH * 2, full);
+                }
             }
             if (*dead) {
                 // loads already issued still land in this CTA's shared memory: give them time to finish
@@ -699,6 +742,25 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
                 for (int mt = 0; mt < DH / 16; ++mt)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) o[nt][mt][e] = 0.f;
+            }
+        }
+        if (w.app && w.j == w.nt - 1 && !*dead) {
+            // The append of the step, folded in: the unit's newest row is not in the cache yet.  The warp whose
+            // keys include it copies it from where it landed beside the tile into the tile (at its swizzled
+            // place) and into the cache; no other warp reads those 16 keys.  Lane -> one 16-byte piece of K or V.
+            const int r = w.len - 1 - w.j * BN;
+            if ((r >> 4) == warp) {
+                constexpr int PIECES = DH / 8;
+                if (lane < 2 * PIECES) {
+                    const bool is_v = lane >= PIECES;
+                    const int cf = lane % PIECES;
+                    const uint4 piece = ptx::lds128(n_base + s * NB + lane * 16);
+                    const uint32_t tile = base + s * R::STAGE_BYTES + (is_v ? R::TILE_BYTES : 0);
+                    ptx::sts128(tile + (cf >> 3) * HALF_BYTES + r * 128 + (((cf & 7) ^ (r & 7)) << 4), piece);
+                    const size_t row = ((size_t)w.u * p.Hkv + w.h) * p.cap + (w.len - 1);
+                    *reinterpret_cast<uint4 *>((is_v ? p.v_w : p.k_w) + row * DH + cf * 8) = piece;
+                }
+                __syncwarp();
             }
         }
         {
@@ -810,7 +872,8 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     mk_end = *t;
     if (!(t = ctx->tmaps.get(p.v, pool_rows, DH, BOX))) return cudaErrorInvalidValue;
     mv_end = *t;
-    const long long t_max = (long long)p.n_units * p.Hkv * ((p.max_len + BN - 1) / BN);
+    const int max_len = p.k_new ? std::min(p.max_len + 1, p.cap) : p.max_len;     // a folded-in append grows every unit by a row
+    const long long t_max = (long long)p.n_units * p.Hkv * ((max_len + BN - 1) / BN);
     const long long cap = ctx->attn_ctas > 0 ? ctx->attn_ctas : coarse_attn_grid(ctx->max_ctas, (long long)p.n_units * p.Hkv);
     const int grid = (int)std::max<long long>(1, std::min<long long>(t_max, cap));
     const cudaError_t e = launch_dependent(coarse_attn_kernel<DH, GP>, dim3(grid), dim3(THREADS), smem, st, 0, p, mk, mv, mk_end, mv_end);
@@ -821,6 +884,7 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
 }  // namespace
 
 int coarse_attn_ctas_per_sm() { return CTAS_PER_SM; }
+int coarse_attn_fold_limit() { return NLEN; }
 
 // The grid when the caller sets none.  Not every CTA slot of the device is taken: the kernel is bound by
 // HBM well below that, and a slot left free lets a CTA of the next kernel in the stream start, and get

@@ -40,6 +40,7 @@ struct photon_ctx {
     size_t n_tickets;
     int32_t *status;         // device status word
     int32_t *work;           // two counters of the whole-chunk attention's item hand-out; zero between calls
+    int32_t *readers;        // arrival counter of an attention with the append folded in; zero between calls
     long long launches;
     cudaStream_t side;       // lowest-priority stream for the chunk attention of a decode step
     cudaEvent_t ev_fork, ev_join;
@@ -76,6 +77,13 @@ struct AttnParams {
     float *cta_partials;
     int32_t *tickets;
     int32_t *status;
+    // The step's append folded into the attention over the unit's own keys (all NULL otherwise): one new row per unit,
+    // k_new, v_new [n_units, Hkv, dh], installed at row len[u] of a contiguous cache (k_w, v_w: the cache, writable),
+    // len_w[u] += 1 by the last CTA to arrive on `readers` (a counter that is zero between calls).
+    const bf16 *k_new, *v_new;
+    bf16 *k_w, *v_w;
+    int32_t *len_w;
+    int32_t *readers;
 };
 
 // Whole-chunk causal attention: query t of item i (q, out: [n, R, Hq, dh]) stands at row row0 + t of
@@ -159,6 +167,7 @@ cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t 
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                            long long *launches);
 int coarse_attn_ctas_per_sm();
+int coarse_attn_fold_limit();     // largest batch for which the step's append can be folded into the attention
 int coarse_attn_grid(int resident_ctas, long long n_streams);
 int shared_prefix_units_per_cta(int G);
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,

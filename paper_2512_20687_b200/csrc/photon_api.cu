@@ -35,9 +35,11 @@ bool kv_ok(const photon_ctx *ctx, const photon_kv *c, bool allow_shared) {
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 
+// k_new, v_new: the step's append folded into the attention over the units' own keys (see AttnParams), or NULL.
 photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const photon_bf16 *q,
                                const int32_t *slot, int n_q, photon_bf16 *out, float *lse,
-                               float scale, bool chunk, cudaStream_t st) {
+                               float scale, bool chunk, cudaStream_t st, const photon_bf16 *k_new = nullptr,
+                               const photon_bf16 *v_new = nullptr) {
     if (!ctx) return PHOTON_ERR_INVALID_ARG;
     if (!kv_ok(ctx, cache, !chunk) || (chunk && cache->page_table)) return PHOTON_ERR_INVALID_ARG;
     if (n_q < 0 || (n_q > 0 && (!q || !out))) return PHOTON_ERR_INVALID_ARG;
@@ -71,6 +73,14 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
     p.status = ctx->status;
 
     p.cta_partials = ctx->cta_partials;
+    if (k_new) {
+        p.k_new = reinterpret_cast<const bf16 *>(k_new);
+        p.v_new = reinterpret_cast<const bf16 *>(v_new);
+        p.k_w = reinterpret_cast<bf16 *>(cache->k);
+        p.v_w = reinterpret_cast<bf16 *>(cache->v);
+        p.len_w = cache->len;
+        p.readers = ctx->readers;
+    }
     p.max_len = cache->max_len ? cache->max_len : cache->cap;
     p.splits_sh = 0;
     if (!chunk) {
@@ -146,6 +156,7 @@ photon_status photon_create(photon_ctx **out, const photon_config *cfg) {
         return PHOTON_ERR_CUDA;
     }
     ctx->work = ctx->status + 32;
+    ctx->readers = ctx->status + 40;
     int lo = 0, hi = 0;
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, lo) != cudaSuccess ||
@@ -558,11 +569,18 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return PHOTON_ERR_CUDA;
         if (s != PHOTON_OK) { cudaStreamWaitEvent(st, ctx->ev_join, 0); return s; }
     }
-    s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr, a->coarse->n_units, 1, stream);
+    // The append is one row per unit, in place: for a contiguous cache of a batch whose lengths fit the attention
+    // kernel's shared memory it is folded into that kernel (the warp that reaches a unit's last tile installs the
+    // new row in the tile and in the cache; the lengths grow once every CTA has read them), which takes a launch
+    // and the wait between two launches out of the step.  Otherwise the append is its own kernel.
+    const bool fold = !a->coarse->page_table && a->coarse->n_units <= coarse_attn_fold_limit();
+    if (!fold) s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr, a->coarse->n_units, 1, stream);
     if (s == PHOTON_OK && a->ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_begin), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;
     if (s == PHOTON_OK)
-        s = photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse, a->scale_coarse, stream);
+        s = fold ? attention_common(ctx, a->coarse, a->q_coarse, nullptr, a->coarse->n_units, a->out_coarse, a->lse_coarse,
+                                    a->scale_coarse, false, st, a->k_new, a->v_new)
+                 : photon_coarse_attn(ctx, a->coarse, a->q_coarse, a->out_coarse, a->lse_coarse, a->scale_coarse, stream);
     if (s == PHOTON_OK && a->ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_end), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;
     // What the coarse attention wrote leaves beside the converter.  Where the converter's own output lies in the

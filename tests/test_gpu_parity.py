@@ -499,6 +499,74 @@ def test_decode_step_chain_matches_oracle(oracle, idx, layout):
         assert np.abs(lse.cpu().numpy() - r["lse"]).max() < 2e-3
 
 
+@pytest.mark.parametrize("shared", [False, True])
+def test_step_with_the_append_folded_into_the_attention_equals_append_then_attention(oracle, shared):
+    """For a contiguous cache the step installs the new row inside the attention kernel instead of launching the
+    append first.  Cache, lengths, status bits and the attention output must be what photon_kv_append followed
+    by photon_coarse_attn gives, bit for bit: lengths that open a new tile (64, 128), that fill the last slot, and
+    a unit without room, which is flagged and attends its full cache unchanged."""
+    cfg = cfg_small(3, B=13, S=330, shared_S=200) if shared else cfg_small(1, B=13, S=330)
+    s = wl.step_inputs(cfg, poison=True)
+    co, cv, chk = s["coarse"], s["converter"], s["chunks"]
+    lens = np.array([0, 1, 63, 64, 65, 127, 128, 300, 328, 329, 330, 200, 5], np.int32)
+    co["k"] = wl.normal_bf16(9, "k", co["k"].shape)
+    co["v"] = wl.normal_bf16(9, "v", co["v"].shape)
+    for u, n in enumerate(lens):
+        if n < 330:                                      # the slot the new row goes to, and everything behind it
+            co["k"][u, :, n:] = 0x7FC1
+            co["v"][u, :, n:] = 0xFFC1
+    co["len"] = lens
+    scale = cfg.dh ** -0.5
+    with Ctx(cfg) as c:
+        # append, then attention, as two calls
+        d1 = coarse_to_dev(co)
+        out1 = torch.empty_like(d1["q"])
+        lse1 = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device="cuda")
+        n0 = ph.photon_launch_count(c.h)
+        ph.photon_kv_append(c.h, d1["kv"], d1["k_new"], d1["v_new"])
+        ph.photon_coarse_attn(c.h, d1["kv"], d1["q"], out1, lse1, scale)
+        two_calls = ph.photon_launch_count(c.h) - n0
+        assert c.status() == ph.PHOTON_DEV_CAPACITY
+        # the step
+        d2, dc = coarse_to_dev(co), chunks_to_dev(chk)
+        out2 = torch.empty_like(d2["q"])
+        lse2 = torch.empty_like(lse1)
+        U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+        oc = torch.empty_like(dc["q"])
+        args = ph.make_step_args(d2["kv"], d2["k_new"], d2["v_new"], d2["q"], out2, scale, dev_bf16(cv["w_out_major"]),
+                                 ph.PHOTON_W_OUT_MAJOR, U, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc,
+                                 Nc=cfg.Nc, scale_chunk=scale, lse_coarse=lse2)
+        n0 = ph.photon_launch_count(c.h)
+        ph.photon_decode_step(c.h, args)
+        assert ph.photon_launch_count(c.h) - n0 == two_calls - 1 + 2       # no append launch; converter and chunk attention
+        assert c.status() == ph.PHOTON_DEV_CAPACITY
+        ph.photon_decode_step(c.h, args)                                    # the counters are back at zero: a second step works
+        assert c.status() == ph.PHOTON_DEV_CAPACITY
+        for name in ("k", "v"):
+            got1 = host_bits(d1[name])
+        assert np.array_equal(d1["len"].cpu().numpy(), np.minimum(lens + 1, 330))
+        assert np.array_equal(d2["len"].cpu().numpy(), np.minimum(lens + 2, 330))
+    # first step of the folded path against the two calls: redo it on fresh buffers (the second step above moved on)
+    with Ctx(cfg) as c:
+        d3, dc = coarse_to_dev(co), chunks_to_dev(chk)
+        out3 = torch.empty_like(d3["q"])
+        lse3 = torch.empty_like(lse1)
+        args = ph.make_step_args(d3["kv"], d3["k_new"], d3["v_new"], d3["q"], out3, scale, dev_bf16(cv["w_out_major"]),
+                                 ph.PHOTON_W_OUT_MAJOR, U, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc,
+                                 Nc=cfg.Nc, scale_chunk=scale, lse_coarse=lse3)
+        ph.photon_decode_step(c.h, args)
+        assert c.status() == ph.PHOTON_DEV_CAPACITY
+        assert np.array_equal(host_bits(d3["k"]), host_bits(d1["k"])) and np.array_equal(host_bits(d3["v"]), host_bits(d1["v"]))
+        assert np.array_equal(d3["len"].cpu().numpy(), d1["len"].cpu().numpy())
+        assert np.array_equal(host_bits(out3), host_bits(out1))
+        assert np.array_equal(lse3.cpu().numpy(), lse1.cpu().numpy())
+    flags = oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"])
+    assert flags == ph.PHOTON_DEV_CAPACITY
+    assert np.array_equal(host_bits(d3["k"]), co["k"]) and np.array_equal(host_bits(d3["v"]), co["v"])
+    want, _ = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, shared=shared_of(co), n_threads=NT)
+    assert_close(host_f64(out3), want, "folded append")
+
+
 @pytest.mark.parametrize("idx", [2, 3, 4])
 def test_decode_step_chain_at_full_size(oracle, idx):
     """The step as the benchmark times it on the long-context, shared-prefix and chunk-parallel workloads: one
