@@ -66,7 +66,6 @@ size_t smem_bytes(int G) {
            size_t(NW) * G * (DH + 2) * sizeof(float) + 128 /*barriers*/ + 128 /*scalars*/ + NLEN * sizeof(int);
 }
 
-__device__ __forceinline__ int clamp_len(int len, int cap) { return max(0, min(len, cap)); }
 __device__ __forceinline__ int tiles_of(int len) { return (len + BN - 1) / BN; }
 
 // Index arrays (lengths, page ids, prefix ids) are read through the L2 only: another kernel may have
