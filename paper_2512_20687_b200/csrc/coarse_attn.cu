@@ -910,8 +910,12 @@ int coarse_attn_grid(int resident_ctas, long long n_streams) {
 cudaError_t launch_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st, long long *launches) {
     if (p.n_q == 0) return cudaSuccess;
     if (p.splits_sh > 0) {
-        const cudaError_t e = launch_shared_prefix_attention(ctx, p, st, launches);
-        if (e != cudaSuccess) return e;
+        // Short own caches (at most one TMA box of rows per unit, by the caller's bound) ride along in the
+        // shared-prefix kernel as extra key tiles, and that kernel writes the result: one launch instead of two.
+        AttnParams ps = p;
+        ps.own_rows = (!p.page_table && !p.k_new && p.max_len <= shared_prefix_own_rows()) ? shared_prefix_own_rows() : 0;
+        const cudaError_t e = launch_shared_prefix_attention(ctx, ps, st, launches);
+        if (e != cudaSuccess || ps.own_rows) return e;
     }
     const int G = p.Hq / p.Hkv;
     int gp = 1;

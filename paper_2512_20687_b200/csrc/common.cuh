@@ -72,6 +72,8 @@ struct AttnParams {
     int n_q, Hq, Hkv, dh;
     int splits_sh;           // key ranges of a shared prefix = cluster size of its kernel (0: no shared prefix)
     int upc;                 // filled by the launcher: units per CTA on shared keys
+    int own_rows;            // filled by the launcher: the units' own keys (at most this many rows each) are read by the
+                             // shared-prefix kernel, which then writes the final result; 0: a second kernel reads them
     float scale_log2;        // scale * log2(e): logits are kept in the base-2 domain
     float *partials;
     float *cta_partials;
@@ -170,6 +172,12 @@ int coarse_attn_ctas_per_sm();
 int coarse_attn_fold_limit();     // largest batch for which the step's append can be folded into the attention
 int coarse_attn_grid(int resident_ctas, long long n_streams);
 int shared_prefix_units_per_cta(int G);
+int shared_prefix_own_rows();
+// Whether an attention call on this cache is one launch: a shared prefix, and own caches short enough (by the caller's
+// max_len) for their keys to ride along in the shared-prefix kernel.
+inline bool own_keys_ride_with_prefix(const photon_kv *c) {
+    return c->k_shared && !c->page_table && (c->max_len ? c->max_len : c->cap) <= shared_prefix_own_rows();
+}
 cudaError_t launch_chunk_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                    long long *launches);
 cudaError_t launch_chunk_causal_attention(photon_ctx *ctx, const CausalParams &p, cudaStream_t st,

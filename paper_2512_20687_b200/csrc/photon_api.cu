@@ -573,7 +573,9 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
     // kernel's shared memory it is folded into that kernel (the warp that reaches a unit's last tile installs the
     // new row in the tile and in the cache; the lengths grow once every CTA has read them), which takes a launch
     // and the wait between two launches out of the step.  Otherwise the append is its own kernel.
-    const bool fold = !a->coarse->page_table && a->coarse->n_units <= coarse_attn_fold_limit();
+    // (Not where short own caches ride along in the shared-prefix kernel: that path has no kernel of own keys to fold into.)
+    const bool fold = !a->coarse->page_table && a->coarse->n_units <= coarse_attn_fold_limit() &&
+                      !own_keys_ride_with_prefix(a->coarse);
     if (!fold) s = photon_kv_append(ctx, a->coarse, a->k_new, a->v_new, nullptr, a->coarse->n_units, 1, stream);
     if (s == PHOTON_OK && a->ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(a->ev_attn_begin), st) != cudaSuccess)
         s = PHOTON_ERR_CUDA;

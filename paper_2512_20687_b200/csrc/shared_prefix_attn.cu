@@ -37,6 +37,8 @@ constexpr int KV_STAGES = 2;
 constexpr int SW = 8;                      // softmax warps: warp w works on TMEM lanes 32*(w%4).., keys 64*(w/4)..
 constexpr int SP_THREADS = (SW + 3) * 32;  // + K loader (8) + MMA warp and TMEM owner (9) + V loader (10)
 constexpr float RESCALE_GAP = 8.f;         // log2 of the largest factor P may carry
+constexpr int OWN = 32;                    // own rows per unit that can ride along (one TMA box); 128 / OWN units per key tile
+constexpr int LIST = BM + BM / (BN / OWN); // entries of a CTA's tile list: distinct prefixes, then tiles of own keys
 
 template <int DH>
 struct SpTile {
@@ -49,8 +51,10 @@ struct SpTile {
     static constexpr int OFF_V = OFF_K + KV_STAGES * KV_BYTES;
     static constexpr int OFF_TAIL = OFF_V + KV_STAGES * KV_BYTES;
     // after the tiles: barriers (256), scalars (64), prefix ids (BM ints), maxima exchange (2 x 2 x BM floats),
-    // sums exchange (2 x BM floats)
-    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 + 64 + BM * 4 + 4 * BM * 4 + 2 * BM * 4;
+    // sums exchange (2 x BM floats), the tile's distinct prefix ids with this CTA's key range of each (3 x BM ints),
+    // lengths of the first 32 prefixes (32 ints)
+    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 + 64 + BM * 4 + 4 * BM * 4 + 2 * BM * 4 +
+                                3 * LIST * 4 + 32 * 4 + BM * 4 /*own lengths per unit of the tile*/;
     static constexpr int TMEM_COLS = 512;                       // S0, S1 (128 each), O (DH): next power of two
     static constexpr int COL_O = 2 * BN;
 };
@@ -68,8 +72,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 template <int DH>
 __global__ void __launch_bounds__(SP_THREADS, 1)
-shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_ks,
-                     const __grid_constant__ CUtensorMap tm_vs) {
+shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_ks, const __grid_constant__ CUtensorMap tm_vs,
+                     const __grid_constant__ CUtensorMap tm_ko, const __grid_constant__ CUtensorMap tm_vo) {
     using T = SpTile<DH>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -84,6 +88,10 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     int *sid = sc + 16;                                                          // [BM] prefix id per query row's unit
     float *xch_m = reinterpret_cast<float *>(sid + BM);                          // [2 tiles in flight][2 halves][BM]
     float *xch_l = xch_m + 4 * BM;                                               // [2 halves][BM]
+    int *ids = reinterpret_cast<int *>(xch_l + 2 * BM);                          // [BM] distinct prefix ids of the tile, ascending
+    int *rng0 = ids + LIST, *rng1 = rng0 + LIST;                                 // this CTA's key range of each
+    int *shl = rng1 + LIST;                                                      // [32] lengths of prefixes 0..31
+    int *ulen = shl + 32;                                                        // [BM] own length of unit unit0 + i (0: none)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = p.Hq / p.Hkv;
@@ -123,11 +131,59 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         int s = -1;
         if (r < upt * G && i < p.n_q) {
             s = __ldcg(p.sh_id + i);
-            if (s >= p.n_shared || s < 0) s = -1;
+            if (s >= p.n_shared) s = -2;       // a prefix that does not exist voids the query
+            else if (s < 0) s = -1;
         }
         sid[r] = s;
     }
-    __syncthreads();                           // barriers and ids are ready: the TMA warp starts loading at once
+    // With the units' own keys riding along (p.own_rows = OWN: every unit holds at most OWN rows), their lengths.
+    for (int i = threadIdx.x; i < BM; i += SP_THREADS) {
+        const int u = unit0 + i;
+        int n = 0;
+        if (p.own_rows && i < upt && u < p.n_q) {
+            n = max(0, min(__ldcg(p.len + u), p.cap));
+            if (n > OWN) { n = OWN; atomicOr(p.status, PHOTON_DEV_BAD_INDEX); }   // beyond what the caller's max_len promised
+        }
+        ulen[i] = n;
+    }
+    // (the lengths of the first prefixes travel with the ids: one trip to the L2 for both)
+    if (threadIdx.x >= SP_THREADS - 32) {
+        const int i = threadIdx.x - (SP_THREADS - 32);
+        shl[i] = i < p.n_shared ? max(0, min(__ldcg(p.sh_len + i), p.cap_sh)) : 0;
+    }
+    __syncthreads();
+    // The list every role walks: the distinct prefix ids of the tile's units in ascending order, each with
+    // this CTA's key range of that prefix.  One warp finds it (a minimum over the lanes per distinct id).
+    if (warp == 0) {
+        int n = 0, last = -1;
+        for (;;) {
+            int cand = 0x7FFFFFFF;
+            for (int r = lane * G; r < BM; r += 32 * G) {
+                const int s = sid[r];
+                if (s > last && s < cand) cand = s;
+            }
+            const int cur = __reduce_min_sync(0xffffffffu, cand);
+            if (cur == 0x7FFFFFFF) break;
+            if (lane == 0) {
+                const int L = cur < 32 ? shl[cur] : max(0, min(__ldcg(p.sh_len + cur), p.cap_sh));
+                int r0, r1;
+                part_range(L, p.splits_sh, part, r0, r1);
+                ids[n] = cur; rng0[n] = r0; rng1[n] = r1;
+            }
+            ++n;
+            last = cur;
+        }
+        // then the tiles of own keys: tile t holds the rows of units 4t .. 4t + 3 of this row tile; the key ranges of
+        // the cluster take them in turn.  An entry with a negative id -1 - t stands for own tile t.
+        if (p.own_rows) {
+            const int n_own = (upt + BN / OWN - 1) / (BN / OWN);
+            for (int t = part; t < n_own; t += p.splits_sh, ++n)
+                if (lane == 0) { ids[n] = -1 - t; rng0[n] = 0; rng1[n] = BN; }
+        }
+        if (lane == 0) sc[3] = n;
+    }
+    __syncthreads();                           // barriers, ids and key ranges are ready: the TMA warps start loading at once
+    const int n_ids = sc[3];
 
     uint32_t tmem = 0;
     if (warp != SW && warp != SW + 2) {
@@ -161,17 +217,6 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         tmem = *reinterpret_cast<volatile uint32_t *>(sc);
     }
 
-    // Every role walks the same list of tiles: for each distinct prefix id of the tile's units
-    // (ascending), the 128-key tiles of this CTA's key range of that prefix.
-    auto next_sid = [&](int last) {
-        int cur = 0x7FFFFFFF;
-        for (int r = 0; r < BM; r += G) {
-            const int s = sid[r];
-            if (s > last && s < cur) cur = s;
-        }
-        return cur;
-    };
-
     // what a softmax thread carries out of the key loop for its row
     float fin_m = -CUDART_INF_F, fin_l = 0.f;
     bool fin_have = false, fin_any = false;
@@ -183,11 +228,33 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         const bool is_k = warp == SW;
         const uint32_t full0 = is_k ? k_full : v_full, empty0 = is_k ? k_empty : v_empty, dst0 = is_k ? sK : sV;
         const CUtensorMap *tm = is_k ? &tm_ks : &tm_vs;
+        const CUtensorMap *tm_own = is_k ? &tm_ko : &tm_vo;
         int it = 0;
         bool ok = true;
-        for (int cur = next_sid(-1); cur != 0x7FFFFFFF && ok; cur = next_sid(cur)) {
-            int r0, r1;
-            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
+        for (int n = 0; n < n_ids && ok; ++n) {
+            const int cur = ids[n], r0 = rng0[n], r1 = rng1[n];
+            if (cur < 0) {
+                // a tile of own keys: one box of OWN rows per unit (a unit past the batch reads as zeros)
+                const int s = it % KV_STAGES;
+                if (!__all_sync(0xffffffffu, ptx::mbar_wait(empty0 + 8 * s, ((it / KV_STAGES) & 1) ^ 1))) {
+                    if (lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+                if (ptx::elect_one()) {
+                    ptx::mbar_arrive_expect_tx(full0 + 8 * s, T::KV_BYTES);
+                    for (int i = 0; i < BN / OWN; ++i) {
+                        const int u = unit0 + (-1 - cur) * (BN / OWN) + i;
+                        const int y = u < p.n_units ? (u * p.Hkv + h) * p.cap : p.n_units * p.Hkv * p.cap;
+#pragma unroll
+                        for (int hh = 0; hh < T::HALVES; ++hh)
+                            ptx::tma_load_2d(dst0 + s * T::KV_BYTES + hh * (BN * 128) + i * (OWN * 128), tm_own, hh * 64, y, full0 + 8 * s);
+                    }
+                }
+                __syncwarp();
+                ++it;
+                continue;
+            }
             const int row_base = (cur * p.Hkv + h) * p.cap_sh;
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int s = it % KV_STAGES;
@@ -210,11 +277,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(BM, BN, false, false);
         constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(BM, DH, false, true);
         int n_tiles = 0;
-        for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
-            int r0, r1;
-            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
-            n_tiles += (r1 - r0 + BN - 1) / BN;
-        }
+        for (int n = 0; n < n_ids; ++n) n_tiles += (rng1[n] - rng0[n] + BN - 1) / BN;
         bool ok = true;
         auto issue_qk = [&](int i) {           // S[i % 2] = Q K_i^T
             const int s = i % KV_STAGES, b = i & 1;
@@ -270,13 +333,24 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         bool ok = true;
         // After a wait has run out (ok = false) the loop goes on without waiting, so that the warps
         // keep meeting at the named barrier; the results are then void and the status says so.
-        for (int cur = next_sid(-1); cur != 0x7FFFFFFF; cur = next_sid(cur)) {
-            int r0, r1;
-            part_range(max(0, min(__ldcg(p.sh_len + cur), p.cap_sh)), p.splits_sh, part, r0, r1);
-            const bool active = (my_sid == cur);
+        for (int n = 0; n < n_ids; ++n) {
+            const int cur = ids[n], r0 = rng0[n], r1 = rng1[n];
+            const bool own = cur < 0;                              // a tile of own keys: OWN rows of each of BN / OWN units
+            bool active = (my_sid == cur);
+            int own_lo = 0, own_hi = 0;                            // my valid keys within my half of an own tile
+            if (own) {
+                const int ur = row / G, blk = ur % (BN / OWN);     // my unit in the row tile, its block of keys in its tile
+                const bool mine = row < upt * G && my_sid != -2 && ur / (BN / OWN) == -1 - cur;
+                active = mine && ulen[ur] > 0;
+                if (active && blk / (CH / OWN) == hf) {
+                    own_lo = (blk % (CH / OWN)) * OWN;
+                    own_hi = own_lo + ulen[ur];
+                }
+            }
             for (int k0 = r0; k0 < r1; k0 += BN, ++it) {
                 const int b = it & 1, st = it % KV_STAGES;
-                const int nvalid = min(BN, r1 - k0) - hf * CH;     // keys of my half that are in range (may be <= 0)
+                // keys [lo, hi) of my half are in range (hi may be <= lo)
+                const int lo = own ? own_lo : 0, hi = own ? own_hi : min(BN, r1 - k0) - hf * CH;
                 if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(s_ready + 8 * b, (it >> 1) & 1))) ok = false;
                 ptx::tc_fence_after();
                 uint32_t sr[CH];
@@ -288,22 +362,25 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(s_free + 8 * b);          // the tensor pipe may overwrite this S
 
-                float mx = -CUDART_INF_F;
-                if (nvalid >= CH) {
+                // four running maxima (and, below, four running sums): one chain of 64 dependent operations
+                // would cost this thread more than the arithmetic itself
+                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                if (lo == 0 && hi >= CH) {
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {
                         const float v = __uint_as_float(sr[c]) * p.scale_log2;
                         sr[c] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
+                        mx4[c & 3] = fmaxf(mx4[c & 3], v);
                     }
                 } else {
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {
-                        const float v = c < nvalid ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
+                        const float v = (c >= lo && c < hi) ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
                         sr[c] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
+                        mx4[c & 3] = fmaxf(mx4[c & 3], v);
                     }
                 }
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // the two threads of a row exchange their maxima; a row whose maximum outgrows its reference
                 // by more than the gap makes the whole CTA rescale its accumulators
                 xch_m[(b * 2 + hf) * BM + row] = mx;
@@ -340,7 +417,17 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 }
                 // rows of V past the end of the range may hold anything: clear them (P is 0 there, 0 * NaN is not)
                 const int tile_valid = min(BN, r1 - k0);
-                if (tile_valid < BN) {
+                if (own) {
+                    // every row at or past its unit's length, unit by unit
+                    if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
+                    for (int idx = threadIdx.x; idx < BN * T::HALVES * 8; idx += SW * 32) {
+                        const int r = idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
+                        const int uu = (-1 - cur) * (BN / OWN) + r / OWN;
+                        if (r % OWN >= (uu < BM ? ulen[uu] : 0))
+                            ptx::sts128(sV + st * T::KV_BYTES + (c16 >> 3) * (BN * 128) + r * 128 + ((c16 & 7) << 4),
+                                        make_uint4(0u, 0u, 0u, 0u));
+                    }
+                } else if (tile_valid < BN) {
                     if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
                     for (int idx = threadIdx.x; idx < (BN - tile_valid) * T::HALVES * 8; idx += SW * 32) {
                         const int r = tile_valid + idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
@@ -349,7 +436,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                     }
                 }
                 // probabilities of my 64 keys, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
-                float ls = 0.f;
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t prow = sP + hf * (BM * 128) + row * 128;
                 if (active) {
 #pragma unroll
@@ -358,7 +445,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             e[j] = exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref);
-                            ls += e[j];
+                            ls4[j & 3] += e[j];
                         }
                         ptx::sts128(prow + ((ch ^ (row & 7)) << 4),
                                     make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])));
@@ -367,7 +454,7 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
 #pragma unroll
                     for (int ch = 0; ch < CH / 8; ++ch) ptx::sts128(prow + ((ch ^ (row & 7)) << 4), make_uint4(0u, 0u, 0u, 0u));
                 }
-                l_half += ls;
+                l_half += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
                 ptx::fence_proxy_async();
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -473,7 +560,21 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 }
             }
             (void)mine;
-            float *out = p.partials + ((size_t)i * p.Hq + (size_t)h * G + rr % G) * (DH + 2);
+            const size_t qh = (size_t)i * p.Hq + (size_t)h * G + rr % G;
+            if (p.own_rows) {
+                // the units' own keys rode along: this is the whole result of the query head
+                const bool gone = sid[rr] == -2;                  // its prefix does not exist
+                if (gone && lane == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+                const float inv = (L > 0.f && !gone) ? 1.f / L : 0.f;
+#pragma unroll
+                for (int k = 0; k < NK; ++k)
+                    if (4 * lane + 128 * k < DH)
+                        *reinterpret_cast<uint2 *>(p.out + qh * DH + 4 * lane + 128 * k) =
+                            make_uint2(pack_bf16(acc[k].x * inv, acc[k].y * inv), pack_bf16(acc[k].z * inv, acc[k].w * inv));
+                if (lane == 0 && p.lse) p.lse[qh] = (L > 0.f && !gone) ? (M + log2f(L)) * 0.6931471805599453f : -CUDART_INF_F;
+                continue;
+            }
+            float *out = p.partials + qh * (DH + 2);
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
                 if (4 * lane + 128 * k < DH) {
@@ -500,13 +601,18 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
     const int upt = BM / G;
     const int groups = (p.n_q + upt - 1) / upt;
     const CUtensorMap *t;
-    CUtensorMap mks, mvs;
+    CUtensorMap mks, mvs, mko, mvo;
     if (!(t = ctx->tmaps.get(p.ks, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mks = *t;
     if (!(t = ctx->tmaps.get(p.vs, (uint64_t)p.n_shared * p.Hkv * p.cap_sh, DH, BN))) return cudaErrorInvalidValue;
     mvs = *t;
+    // the units' own caches in boxes of OWN rows (used when their keys ride along)
+    if (!(t = ctx->tmaps.get(p.k, (uint64_t)p.n_units * p.Hkv * p.cap, DH, OWN))) return cudaErrorInvalidValue;
+    mko = *t;
+    if (!(t = ctx->tmaps.get(p.v, (uint64_t)p.n_units * p.Hkv * p.cap, DH, OWN))) return cudaErrorInvalidValue;
+    mvo = *t;
     const cudaError_t e = launch_dependent(shared_prefix_kernel<DH>, dim3(groups * p.Hkv * p.splits_sh), dim3(SP_THREADS), T::SMEM, st,
-                                           p.splits_sh /* the key ranges of a row tile form a cluster */, p, mks, mvs);
+                                           p.splits_sh /* the key ranges of a row tile form a cluster */, p, mks, mvs, mko, mvo);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -514,6 +620,7 @@ cudaError_t run(photon_ctx *ctx, AttnParams p, cudaStream_t st, long long *launc
 }  // namespace
 
 int shared_prefix_units_per_cta(int G) { return BM / G; }
+int shared_prefix_own_rows() { return OWN; }
 
 cudaError_t launch_shared_prefix_attention(photon_ctx *ctx, const AttnParams &p, cudaStream_t st,
                                            long long *launches) {

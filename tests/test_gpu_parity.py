@@ -147,12 +147,14 @@ def test_coarse_attention_other_group_sizes(oracle, G, dh):
 
 # group sizes and head sizes the shared-prefix kernel accepts: a row tile of 128 query rows holds 128 / G units
 # (126 of its rows are used for G = 3); the batch is never a whole number of tiles
+# ... and own caches of at most 40 rows (a second kernel reads them) or at most 24 (they ride along in the first)
+@pytest.mark.parametrize("S", [40, 24])
 @pytest.mark.parametrize("max_splits", [1, 0])
 @pytest.mark.parametrize("G,dh,B", [(4, 128, 37), (1, 64, 150), (2, 128, 75), (3, 64, 50), (8, 128, 21), (16, 64, 13)])
-def test_shared_prefix_variants(oracle, G, dh, B, max_splits):
+def test_shared_prefix_variants(oracle, G, dh, B, max_splits, S):
     """Two shared segments of different length, units without a prefix, empty own caches."""
     Hkv = 4 if G == 4 else 2
-    cfg = cfg_small(3, B=B, S=40, shared_S=300, Hq=G * Hkv, Hkv=Hkv, dh=dh, D=G * Hkv * dh)
+    cfg = cfg_small(3, B=B, S=S, shared_S=300, Hq=G * Hkv, Hkv=Hkv, dh=dh, D=G * Hkv * dh)
     co = wl.coarse_inputs(cfg, poison=True)
     ks = wl.normal_bf16(3, "ks2", (2, cfg.Hkv, 300, cfg.dh))
     vs = wl.normal_bf16(3, "vs2", (2, cfg.Hkv, 300, cfg.dh))
@@ -160,7 +162,7 @@ def test_shared_prefix_variants(oracle, G, dh, B, max_splits):
     ks[1, :, 77:] = 0x7FC1
     vs[1, :, 77:] = 0x7FC1
     sh_id = (np.arange(cfg.B) % 3 - 1).astype(np.int32)       # -1, 0, 1, -1, ...
-    lens = (np.arange(cfg.B) % 5 * 9).astype(np.int32)        # 0, 9, 18, 27, 36
+    lens = (np.arange(cfg.B) % 5 * (S // 4 - 1)).astype(np.int32)        # 0, 9, 18, 27, 36 of 40 rows; 0 .. 20 of 24
     for u, n in enumerate(lens):
         co["k"][u, :, n:] = 0x7FC1
         co["v"][u, :, n:] = 0x7FC1
@@ -171,7 +173,7 @@ def test_shared_prefix_variants(oracle, G, dh, B, max_splits):
     with Ctx(cfg, max_splits=max_splits) as c:
         got, lse, _ = run_coarse(c, co, scale)
         assert c.status() == 0
-    assert_close(got, want, f"shared prefix G={G} dh={dh} splits={max_splits}")
+    assert_close(got, want, f"shared prefix G={G} dh={dh} splits={max_splits} S={S}")
     empty = (lens == 0) & (sh_id < 0)
     assert empty.any() and np.all(got[empty] == 0) and np.all(np.isneginf(lse[empty]))
     fin = np.isfinite(want_lse)
