@@ -79,7 +79,12 @@ typedef struct {
  *               and never influence a result.
  *   len         [n_units] device int32.
  *   max_len     host-side upper bound on every len[u] during the call
- *               (0 = cap); only steers how many CTAs are launched.
+ *               (0 = cap).  It steers how many CTAs are launched and, for a
+ *               cache with shared prefixes, whether the units' own rows are
+ *               read by the shared-prefix kernel itself (at most 32 of them
+ *               per unit: one launch) or by a second kernel.  It has to hold:
+ *               a unit longer than max_len may have the rows beyond it
+ *               ignored, with PHOTON_DEV_BAD_INDEX set.
  * Optional shared prefixes (Section 1: long-context, multi-query serving; one
  * document, many query branches): unit u with shared_id[u] = s >= 0 attends
  * rows [0, shared_len[s]) of segment s followed by its own rows, exactly as

@@ -133,6 +133,11 @@ __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The same barrier without memory ordering: for when only the fact that every CTA has arrived matters.
+__device__ __forceinline__ void cluster_sync_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
 // Reads the float at shared-memory address `addr` (an address of this CTA's window) in CTA `rank` of the cluster.
 __device__ __forceinline__ float ld_cluster_f32(uint32_t addr, uint32_t rank) {
     uint32_t remote;

@@ -34,8 +34,10 @@ namespace {
 constexpr int BM = 128;                    // query rows per CTA (UMMA M; one TMEM lane each)
 constexpr int BN = 128;                    // keys per tile
 constexpr int KV_STAGES = 2;
-constexpr int SW = 8;                      // softmax warps: warp w works on TMEM lanes 32*(w%4).., keys 64*(w/4)..
-constexpr int SP_THREADS = (SW + 3) * 32;  // + K loader (8) + MMA warp and TMEM owner (9) + V loader (10)
+constexpr int SW = 16;                     // softmax warps: warp w works on TMEM lanes 32*(w%4).., keys CH*(w/4)..
+constexpr int KP = SW / 4;                 // threads that share a query row, each on CH keys of a tile
+constexpr int CH = BN / KP;
+constexpr int SP_THREADS = (SW + 3) * 32;  // + K loader + MMA warp and TMEM owner + V loader
 constexpr float RESCALE_GAP = 8.f;         // log2 of the largest factor P may carry
 constexpr int OWN = 32;                    // own rows per unit that can ride along (one TMA box); 128 / OWN units per key tile
 constexpr int LIST = BM + BM / (BN / OWN); // entries of a CTA's tile list: distinct prefixes, then tiles of own keys
@@ -53,7 +55,7 @@ struct SpTile {
     // after the tiles: barriers (256), scalars (64), prefix ids (BM ints), maxima exchange (2 x 2 x BM floats),
     // sums exchange (2 x BM floats), the tile's distinct prefix ids with this CTA's key range of each (3 x BM ints),
     // lengths of the first 32 prefixes (32 ints)
-    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 + 64 + BM * 4 + 4 * BM * 4 + 2 * BM * 4 +
+    static constexpr int SMEM = OFF_TAIL + 1024 /*alignment slack*/ + 256 + 64 + BM * 4 + 2 * KP * BM * 4 + KP * BM * 4 +
                                 3 * LIST * 4 + 32 * 4 + BM * 4 /*own lengths per unit of the tile*/;
     static constexpr int TMEM_COLS = 512;                       // S0, S1 (128 each), O (DH): next power of two
     static constexpr int COL_O = 2 * BN;
@@ -86,9 +88,9 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     const uint32_t p_ready = bars + 80, p_free = bars + 88, recv_bar = bars + 96;
     int *sc = reinterpret_cast<int *>(gen + T::OFF_TAIL + 256);                  // [0] tmem base, [1..2] rescale flags
     int *sid = sc + 16;                                                          // [BM] prefix id per query row's unit
-    float *xch_m = reinterpret_cast<float *>(sid + BM);                          // [2 tiles in flight][2 halves][BM]
-    float *xch_l = xch_m + 4 * BM;                                               // [2 halves][BM]
-    int *ids = reinterpret_cast<int *>(xch_l + 2 * BM);                          // [BM] distinct prefix ids of the tile, ascending
+    float *xch_m = reinterpret_cast<float *>(sid + BM);                          // [2 tiles in flight][KP key parts][BM]
+    float *xch_l = xch_m + 2 * KP * BM;                                          // [KP key parts][BM]
+    int *ids = reinterpret_cast<int *>(xch_l + KP * BM);                          // [BM] distinct prefix ids of the tile, ascending
     int *rng0 = ids + LIST, *rng1 = rng0 + LIST;                                 // this CTA's key range of each
     int *shl = rng1 + LIST;                                                      // [32] lengths of prefixes 0..31
     int *ulen = shl + 32;                                                        // [BM] own length of unit unit0 + i (0: none)
@@ -125,26 +127,38 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     }
     ptx::grid_dep_wait();                      // queries may come from the kernel before this one
     ptx::grid_dep_launch();                    // one wave: the kernel for the units' own keys may line up
-    // prefix id of every row's unit (>= 0 valid, -1 none / bad / past the batch); row r = (unit - unit0) * G + g
-    for (int r = threadIdx.x; r < BM; r += SP_THREADS) {
-        const int i = unit0 + r / G;
-        int s = -1;
-        if (r < upt * G && i < p.n_q) {
-            s = __ldcg(p.sh_id + i);
-            if (s >= p.n_shared) s = -2;       // a prefix that does not exist voids the query
-            else if (s < 0) s = -1;
+    // The Q tile goes to shared memory K-major with the 128-byte swizzle TMA would use.  Every warp but the two
+    // loaders takes part; all of a thread's loads are requested here, before anything else, and stored once the
+    // tile list below is done: one round trip to memory, under the one the ids make.
+    constexpr int NQT = SP_THREADS - 64;
+    constexpr int QV = (BM * (DH / 8) + NQT - 1) / NQT;
+    const int tq = threadIdx.x < SW * 32 ? threadIdx.x : threadIdx.x - 32;
+    uint4 qv[QV];
+    if (warp != SW && warp != SW + 2) {
+#pragma unroll
+        for (int t = 0; t < QV; ++t) {
+            const int idx = tq + t * NQT;
+            const int r = idx / (DH / 8), ch = idx % (DH / 8);                   // 16-byte chunk ch of row r
+            const int i = unit0 + r / G;
+            qv[t] = make_uint4(0u, 0u, 0u, 0u);
+            if (idx < BM * (DH / 8) && r < upt * G && i < p.n_q)
+                qv[t] = __ldcg(reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8));
         }
-        sid[r] = s;
     }
-    // With the units' own keys riding along (p.own_rows = OWN: every unit holds at most OWN rows), their lengths.
-    for (int i = threadIdx.x; i < BM; i += SP_THREADS) {
-        const int u = unit0 + i;
-        int n = 0;
-        if (p.own_rows && i < upt && u < p.n_q) {
-            n = max(0, min(__ldcg(p.len + u), p.cap));
-            if (n > OWN) { n = OWN; atomicOr(p.status, PHOTON_DEV_BAD_INDEX); }   // beyond what the caller's max_len promised
-        }
-        ulen[i] = n;
+    // prefix id of every row's unit (>= 0 valid, -1 none or past the batch, -2 no such prefix); row r = (unit - unit0)
+    // * G + g.  With the units' own keys riding along (p.own_rows = OWN: every unit holds at most OWN rows), the
+    // own length of unit unit0 + r as well.  Both loads are requested before either is used.
+    if (threadIdx.x < BM) {
+        const int r = threadIdx.x, i = unit0 + r / G, u = unit0 + r;
+        const bool has_row = r < upt * G && i < p.n_q, has_unit = p.own_rows && r < upt && u < p.n_q;
+        int s = has_row ? __ldcg(p.sh_id + i) : -1;
+        int n = has_unit ? __ldcg(p.len + u) : 0;
+        if (s >= p.n_shared) s = -2;           // a prefix that does not exist voids the query
+        else if (s < 0) s = -1;
+        n = max(0, min(n, p.cap));
+        if (n > OWN) { n = OWN; atomicOr(p.status, PHOTON_DEV_BAD_INDEX); }   // beyond what the caller's max_len promised
+        sid[r] = s;
+        ulen[r] = n;
     }
     // (the lengths of the first prefixes travel with the ids: one trip to the L2 for both)
     if (threadIdx.x >= SP_THREADS - 32) {
@@ -188,21 +202,6 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
     uint32_t tmem = 0;
     if (warp != SW && warp != SW + 2) {
         if (warp == SW + 1) ptx::tmem_alloc(ptx::smem_u32(sc), T::TMEM_COLS);
-        // the Q tile, stored K-major with the 128-byte swizzle TMA would use; all of a thread's loads are
-        // issued before its first store: one round trip to memory, not one per chunk
-        constexpr int NQT = SP_THREADS - 64;
-        constexpr int QV = (BM * (DH / 8) + NQT - 1) / NQT;
-        const int tq = threadIdx.x < SW * 32 ? threadIdx.x : threadIdx.x - 32;
-        uint4 qv[QV];
-#pragma unroll
-        for (int t = 0; t < QV; ++t) {
-            const int idx = tq + t * NQT;
-            const int r = idx / (DH / 8), ch = idx % (DH / 8);                   // 16-byte chunk ch of row r
-            const int i = unit0 + r / G;
-            qv[t] = make_uint4(0u, 0u, 0u, 0u);
-            if (idx < BM * (DH / 8) && r < upt * G && i < p.n_q)
-                qv[t] = __ldcg(reinterpret_cast<const uint4 *>(p.q + ((size_t)i * p.Hq + (size_t)h * G + r % G) * DH + ch * 8));
-        }
 #pragma unroll
         for (int t = 0; t < QV; ++t) {
             const int idx = tq + t * NQT;
@@ -323,12 +322,12 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
     } else {
         // ======================= softmax warps: two threads per query row =======================
-        const int quad = warp & 3, hf = warp >> 2;                 // TMEM lane quadrant; which 64 keys of a tile
+        const int quad = warp & 3, hf = warp >> 2;                 // TMEM lane quadrant; which CH keys of a tile
         const int row = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const int my_sid = sid[row];
-        constexpr int CH = BN / 2;                                 // keys per thread and tile
-        float m_ref = -CUDART_INF_F, l_half = 0.f;                 // m_ref is kept identical in both threads of a row
+        constexpr int RP = DH / 32 < KP ? DH / 32 : KP;            // threads of a row that move its accumulator, 32 or more columns each
+        float m_ref = -CUDART_INF_F, l_half = 0.f;                 // m_ref is kept identical in all threads of a row
         int it = 0;
         bool ok = true;
         // After a wait has run out (ok = false) the loop goes on without waiting, so that the warps
@@ -383,10 +382,11 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // the two threads of a row exchange their maxima; a row whose maximum outgrows its reference
                 // by more than the gap makes the whole CTA rescale its accumulators
-                xch_m[(b * 2 + hf) * BM + row] = mx;
+                xch_m[(b * KP + hf) * BM + row] = mx;
                 if (active && m_ref != -CUDART_INF_F && mx > m_ref + RESCALE_GAP) sc[1 + b] = 1;
                 ptx::named_bar_sync(1, SW * 32);
-                mx = fmaxf(mx, xch_m[(b * 2 + (hf ^ 1)) * BM + row]);
+#pragma unroll
+                for (int o = 1; o < KP; ++o) mx = fmaxf(mx, xch_m[(b * KP + (hf ^ o)) * BM + row]);
                 const bool rescale = sc[1 + b] != 0;
                 float corr = 1.f;
                 if (active) {
@@ -402,13 +402,13 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 if (rescale) {
                     ptx::tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < DH / 2; c0 += 32) {              // my half of the row's accumulator
+                    for (int c0 = 0; c0 < DH / RP && hf < RP; c0 += 32) {  // my part of the row's accumulator
                         uint32_t orow[32];
-                        ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + hf * (DH / 2) + c0, orow);
+                        ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + hf * (DH / RP) + c0, orow);
                         ptx::tmem_ld_wait();
 #pragma unroll
                         for (int e = 0; e < 32; ++e) orow[e] = __float_as_uint(__uint_as_float(orow[e]) * corr);
-                        ptx::tmem_st_32x32(tmem + lane_base + T::COL_O + hf * (DH / 2) + c0, orow);
+                        ptx::tmem_st_32x32(tmem + lane_base + T::COL_O + hf * (DH / RP) + c0, orow);
                     }
                     ptx::tmem_st_wait();
                     l_half *= corr;
@@ -437,7 +437,10 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 }
                 // probabilities of my 64 keys, bf16, into the swizzled P tile (K-major: 64 keys per 128-byte row)
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-                const uint32_t prow = sP + hf * (BM * 128) + row * 128;
+                // (a 128-byte row of P holds 64 keys: my CH keys start at 16-byte chunk pc0 of row `row` of half ph)
+                constexpr int CPH = 64 / CH;                               // key parts per 64-key half
+                const int ph = hf / CPH, pc0 = (hf % CPH) * (CH / 8);
+                const uint32_t prow = sP + ph * (BM * 128) + row * 128;
                 if (active) {
 #pragma unroll
                     for (int ch = 0; ch < CH / 8; ++ch) {
@@ -447,12 +450,12 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                             e[j] = exp2f(__uint_as_float(sr[ch * 8 + j]) - m_ref);
                             ls4[j & 3] += e[j];
                         }
-                        ptx::sts128(prow + ((ch ^ (row & 7)) << 4),
+                        ptx::sts128(prow + (((pc0 + ch) ^ (row & 7)) << 4),
                                     make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])));
                     }
                 } else {
 #pragma unroll
-                    for (int ch = 0; ch < CH / 8; ++ch) ptx::sts128(prow + ((ch ^ (row & 7)) << 4), make_uint4(0u, 0u, 0u, 0u));
+                    for (int ch = 0; ch < CH / 8; ++ch) ptx::sts128(prow + (((pc0 + ch) ^ (row & 7)) << 4), make_uint4(0u, 0u, 0u, 0u));
                 }
                 l_half += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
                 ptx::fence_proxy_async();
@@ -464,7 +467,9 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         // ---- what the row carries out: reference maximum and the sum over both halves
         xch_l[hf * BM + row] = l_half;
         ptx::named_bar_sync(1, SW * 32);
-        const float l_sum = l_half + xch_l[(hf ^ 1) * BM + row];
+        float l_sum = l_half;
+#pragma unroll
+        for (int o = 1; o < KP; ++o) l_sum += xch_l[(hf ^ o) * BM + row];
         if (ok && it > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(p_free, (it - 1) & 1));
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
         ptx::tc_fence_after();
@@ -486,8 +491,9 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         const int row = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float *stage = reinterpret_cast<float *>(gen) + (size_t)row * RS;
+        constexpr int RP = DH / 32 < KP ? DH / 32 : KP;
 #pragma unroll 1
-        for (int c0 = hf * (DH / 2); c0 < (hf + 1) * (DH / 2); c0 += 32) {
+        for (int c0 = hf * (DH / RP); c0 < (hf + 1) * (DH / RP) && hf < RP; c0 += 32) {
             uint32_t orow[32];
             if (fin_any) {                                                  // O was written by at least one P V
                 ptx::tmem_ld_32x32(tmem + lane_base + T::COL_O + c0, orow);
@@ -585,7 +591,10 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
             if (lane == 0) { out[DH] = M; out[DH + 1] = L; }
         }
     }
-    ptx::cluster_sync();                                           // every copy out of this CTA's staging area has landed
+    // Every copy out of this CTA's staging area has landed once its peers are past their own receive wait, which
+    // is where they come from: nothing but the order of arrival is needed of this barrier, no flush of the
+    // results written just before it.
+    ptx::cluster_sync_relaxed();
     if (warp == SW + 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, T::TMEM_COLS);
