@@ -23,6 +23,14 @@
  *  - q and k arrive already position-encoded; the library applies no rotary
  *    or other positional transform.
  *  - There is no CPU fallback: without a CUDA device photon_create fails.
+ *  - Host threads: the library keeps a little host-side state (tensor-map
+ *    caches, per-kernel launch attributes) that it does not lock.  Calls on
+ *    one context, and calls of photon_coarse_attn_noalloc on one device, must
+ *    not run concurrently with each other or with calls on another context;
+ *    a caller with several threads serialises its calls into the library.
+ *  - len, slot, shared_id and page_table must not change while a call that
+ *    reads them is in flight on the device (a kernel of the caller's that
+ *    writes them belongs before the call in the same stream).
  */
 #ifndef PHOTON_H
 #define PHOTON_H

@@ -336,8 +336,13 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
             const int cur = ids[n], r0 = rng0[n], r1 = rng1[n];
             const bool own = cur < 0;                              // a tile of own keys: OWN rows of each of BN / OWN units
             bool active = (my_sid == cur);
-            int own_lo = 0, own_hi = 0;                            // my valid keys within my half of an own tile
+            int own_lo = 0, own_hi = 0;                            // my valid keys within my part of an own tile
+            bool own_clear = false;                                // some unit of the tile ends before its box of rows does
             if (own) {
+                for (int i = 0; i < BN / OWN; ++i) {
+                    const int uu = (-1 - cur) * (BN / OWN) + i;
+                    own_clear |= uu < upt && unit0 + uu < p.n_q && ulen[uu] < OWN;
+                }
                 const int ur = row / G, blk = ur % (BN / OWN);     // my unit in the row tile, its block of keys in its tile
                 const bool mine = row < upt * G && my_sid != -2 && ur / (BN / OWN) == -1 - cur;
                 active = mine && ulen[ur] > 0;
@@ -418,14 +423,15 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
                 // rows of V past the end of the range may hold anything: clear them (P is 0 there, 0 * NaN is not)
                 const int tile_valid = min(BN, r1 - k0);
                 if (own) {
-                    // every row at or past its unit's length, unit by unit
-                    if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
-                    for (int idx = threadIdx.x; idx < BN * T::HALVES * 8; idx += SW * 32) {
-                        const int r = idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
-                        const int uu = (-1 - cur) * (BN / OWN) + r / OWN;
-                        if (r % OWN >= (uu < BM ? ulen[uu] : 0))
-                            ptx::sts128(sV + st * T::KV_BYTES + (c16 >> 3) * (BN * 128) + r * 128 + ((c16 & 7) << 4),
-                                        make_uint4(0u, 0u, 0u, 0u));
+                    if (own_clear) {                                       // every row at or past its unit's length, unit by unit
+                        if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
+                        for (int idx = threadIdx.x; idx < BN * T::HALVES * 8; idx += SW * 32) {
+                            const int r = idx / (T::HALVES * 8), c16 = idx % (T::HALVES * 8);
+                            const int uu = (-1 - cur) * (BN / OWN) + r / OWN;
+                            if (r % OWN >= (uu < BM ? ulen[uu] : 0))
+                                ptx::sts128(sV + st * T::KV_BYTES + (c16 >> 3) * (BN * 128) + r * 128 + ((c16 & 7) << 4),
+                                            make_uint4(0u, 0u, 0u, 0u));
+                        }
                     }
                 } else if (tile_valid < BN) {
                     if (ok && !__all_sync(0xffffffffu, ptx::mbar_wait(v_full + 8 * st, (it / KV_STAGES) & 1))) ok = false;
