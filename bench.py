@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--layout", default="out_major", choices=["out_major", "in_major"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parts", action="store_true")
+    ap.add_argument("--only-this-workload", action="store_true",
+                    help="skip the other target workloads' attention parts and the read-ceiling probe (profiler captures)")
     ap.add_argument("--max-splits", type=int, default=0)
     ap.add_argument("--hierarchy", default="",
                     help="chunk lengths C_1,...,C_L instead of 4,4 (e.g. 2,2): same model and context, other stream lengths")
@@ -773,14 +775,14 @@ def run_gpu(args, cfg) -> None:
                 # the replicas are meant to keep the reads in HBM: less DRAM traffic than 95 % of the
                 # algorithmic bytes would mean the L2 served part of them
                 "l2_assisted": None if traffic is None else bool(traffic < 0.95 * kernels[dom]["bytes"])}
-    ceil = read_ceiling(kernels[dom]["bytes"])
+    ceil = {"us": None, "ctas": 0} if args.only_this_workload else read_ceiling(kernels[dom]["bytes"])
     roofline.update({"read_ceiling_us": ceil["us"], "read_ceiling_ctas": ceil["ctas"],
-                     "frac_of_read_ceiling": ceil["us"] / kernels[dom]["us"],
+                     "frac_of_read_ceiling": ceil["us"] / kernels[dom]["us"] if ceil["us"] else None,
                      "read_ceiling_note": "photon_read_probe on buffers of the same size: the attention's launch, grid and "
                                           "ring of bulk copies with nothing computed (best of three grids)"})
     # the dominant attention part of every target workload (configs 1-4), this run's own workload from `parts`
     by_workload = {}
-    if not args.no_parts and not args.batch and not args.hierarchy:
+    if not args.no_parts and not args.batch and not args.hierarchy and not args.only_this_workload:
         for idx in (1, 2, 3, 4):
             if idx == cfg.index:
                 pc = parts[dom]

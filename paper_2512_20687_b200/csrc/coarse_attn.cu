@@ -464,8 +464,49 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
         if (sh.t0 < sh.t1) started = w.start(p, sh, slen);
     }
 
+    // One tile into stage it % STAGES: the walker's current tile, with the group's query rows if a stream starts
+    // there and the row a folded-in append installs if the stream ends there.  whole_box: fetch a box of BN
+    // rows whatever the length says (for loads that go out before the lengths are confirmed: a unit may have
+    // grown inside its last tile since they were read; what lies past the end of a cache is never used).
+    auto issue_tile = [&](int it, const Walker &tw, bool whole_box) {
+        const int s = it % STAGES;
+        // row of the tile's first key in the cache tensor; for a paged cache through the page table
+        int y = tile_row(p, tw);
+        if (y < 0) { atomicOr(p.status, PHOTON_DEV_BAD_INDEX); y = tw.h * (p.page_table ? p.page_rows : p.cap); }
+        const uint32_t full = bars + 16 * s;
+        const uint32_t kd = base + s * R::STAGE_BYTES, vd = kd + R::TILE_BYTES;
+        const int rows = min(BN, tw.len - tw.j * BN);
+        const bool first = (it == 0 || tw.j == 0);
+        // a tile of more than BOX rows comes as one box of BN rows per 64 features, a shorter one as one box of BOX rows
+        const bool tall = whole_box || rows > BOX;
+        const bool grows = tw.app && tw.j == tw.nt - 1;        // the row this kernel installs lies in this tile
+        ptx::mbar_arrive_expect_tx(full, R::HALVES * (tall ? HALF_BYTES : BOX_BYTES) * 2 + (first ? G * DH * 2 : 0) +
+                                             (grows ? NB : 0));
+#pragma unroll
+        for (int hh = 0; hh < R::HALVES; ++hh) {
+            ptx::tma_load_2d(kd + hh * HALF_BYTES, tall ? &tm_k : &tm_k_end, hh * 64, y, full);
+            ptx::tma_load_2d(vd + hh * HALF_BYTES, tall ? &tm_v : &tm_v_end, hh * 64, y, full);
+        }
+        if (first)
+            ptx::bulk_load(q_base + s * QB, p.q + ((size_t)tw.u * p.Hq + (size_t)tw.h * G) * DH, G * DH * 2, full);
+        if (grows) {
+            const size_t at = ((size_t)tw.u * p.Hkv + tw.h) * DH;                       // k_new, v_new: [n_units, Hkv, dh]
+            ptx::bulk_load(n_base + s * NB, p.k_new + at, DH * 2, full);
+            ptx::bulk_load(n_base + s * NB + DH * 2, p.v_new + at, DH * 2, full);
+        }
+    };
+
     ptx::grid_dep_wait();                   // lengths, caches and queries may come from the kernel before this one
     ptx::grid_dep_launch();                 // one wave of CTAs, all resident: the next kernel may line up behind them
+
+    // The ring's first turn goes out at once, from the deal made ahead, while the lengths are read again: keys,
+    // values and queries are final now, only the deal may turn out stale.  If it does (rare), these loads are
+    // left to land, the ring's barriers are made anew and everything starts over from the deal.
+    int n_early = 0;
+    if (ahead && started && warp == NW && lane == 0) {
+        const int n = (int)min((long long)STAGES, sh.t1 - sh.t0);
+        for (; n_early < n && w.valid(p); ++n_early, w.next(p)) issue_tile(n_early, w, !p.k_new);
+    }
 
     bool redo = !ahead;
     if (ahead) {
@@ -476,16 +517,32 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
 #pragma unroll
         for (int i = 0; i < LPT; ++i)
             if (ub + i < ue) {
-                diff |= (tiles_of(eff_len(p, len[i])) != tiles_of(eff_len(p, slen[ub + i])));
+                // (with the append folded in nothing else may change a length meanwhile: any difference counts,
+                // and the loads that went out early were sized by the lengths themselves)
+                diff |= p.k_new ? len[i] != slen[ub + i] : tiles_of(eff_len(p, len[i])) != tiles_of(eff_len(p, slen[ub + i]));
                 slen[ub + i] = len[i];
             }
         redo = __syncthreads_or(diff);
     }
     if (redo) {
+        if (ahead) {
+            // what went out early belongs to a deal that no longer holds: let it land, then new barriers
+            for (int b = 0; b < n_early; ++b)
+                if (!ptx::mbar_wait(bars + 16 * b, 0)) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
+            n_early = 0;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int s = 0; s < STAGES; ++s) {
+                    ptx::mbar_inval(bars + 16 * s);
+                    ptx::mbar_init(bars + 16 * s, 1);
+                }
+                ptx::mbar_fence_init();
+            }
+        }
         if (threadIdx.x == 0) { sc[8] = -1; sc[9] = 0; sc[12] = 0; sc[14] = -1; }
         sh = deal(p, sc, slen, cta);
         started = sh.t0 < sh.t1 && w.start(p, sh, slen);
-    } else if (started) {
+    } else if (started && w.valid(p)) {
         w.load(p);                          // same tile counts, but the unit may have grown within its last tile
     }
     const long long T = sh.T, t0 = sh.t0, t1 = sh.t1;
@@ -656,43 +713,18 @@ coarse_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k,
     if (warp == NW) {
         // ======================= producer: one thread feeds the ring =======================
         if (lane == 0) {
-            int it = 0;
+            int it = n_early;                                    // this thread's walker stands behind the tiles that went out early
             for (; it < n_tiles; ++it, w.next(p)) {
                 const int s = it % STAGES;
                 if (*dead) break;
                 if (!w.valid(p)) {                               // ran past the last unit: len[] changed under the kernel
                     *dead = 1; atomicOr(p.status, PHOTON_DEV_BAD_INDEX); break;
                 }
-                // row of the tile's first key in the cache tensor; for a paged cache through the page table
-                // (looked up before the wait for a free stage, which hides the load's latency)
-                int y = tile_row(p, w);
-                if (y < 0) { atomicOr(p.status, PHOTON_DEV_BAD_INDEX); y = w.h * (p.page_table ? p.page_rows : p.cap); }
                 // the ring starts empty: only from its second turn on is there a stage to wait for
                 if (it >= STAGES && !ptx::mbar_wait(bars + 16 * s + 8, ((it / STAGES) & 1) ^ 1)) {
                     *dead = 1; atomicOr(p.status, PHOTON_DEV_TIMEOUT); break;
                 }
-                const uint32_t full = bars + 16 * s;
-                const uint32_t kd = base + s * R::STAGE_BYTES, vd = kd + R::TILE_BYTES;
-                const int rows = min(BN, w.len - w.j * BN);
-                const bool first = (it == 0 || w.j == 0);
-                // a tile of more than BOX rows comes as one box of BN rows per 64 features (what lies past the end
-                // of the cache is never used), a shorter one as one box of BOX rows
-                const bool tall = rows > BOX;
-                const bool grows = w.app && w.j == w.nt - 1;    // the row this kernel installs lies in this tile
-                ptx::mbar_arrive_expect_tx(full, R::HALVES * (tall ? HALF_BYTES : BOX_BYTES) * 2 + (first ? G * DH * 2 : 0) +
-                                                     (grows ? NB : 0));
-#pragma unroll
-                for (int hh = 0; hh < R::HALVES; ++hh) {
-                    ptx::tma_load_2d(kd + hh * HALF_BYTES, tall ? &tm_k : &tm_k_end, hh * 64, y, full);
-                    ptx::tma_load_2d(vd + hh * HALF_BYTES, tall ? &tm_v : &tm_v_end, hh * 64, y, full);
-                }
-                if (first)
-                    ptx::bulk_load(q_base + s * QB, p.q + ((size_t)w.u * p.Hq + (size_t)w.h * G) * DH, G * DH * 2, full);
-                if (grows) {
-                    const size_t at = ((size_t)w.u * p.Hkv + w.h) * DH;                   // k_new, v_new: [n_units, Hkv, dh]
-                    ptx::bulk_load(n_base + s * NB, p.k_new + at, DH * 2, full);
-                    ptx::bulk_load(n_base + s * NB + DH * 2, p.v_new + at, DH * 2, full);
-                }
+                issue_tile(it, w, false);
             }
             if (*dead) {
                 // loads already issued still land in this CTA's shared memory: give them time to finish

@@ -91,6 +91,7 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
             p.sh_len = cache->shared_len; p.sh_id = cache->shared_id;
             p.n_shared = cache->n_shared; p.cap_sh = cache->cap_shared;
             const int ms = cache->max_shared_len ? cache->max_shared_len : cache->cap_shared;
+            p.max_sh = ms;
             if (size_t(n_q) * c.Hq * (c.dh + 2) > ctx->partial_floats) return PHOTON_ERR_WORKSPACE;
             const int G = c.Hq / c.Hkv;
             const int groups = ceil_div(n_q, shared_prefix_units_per_cta(G));     // tiles of 128 query rows
@@ -566,7 +567,8 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         if (s == PHOTON_OK)
             s = photon_chunk_attn(ctx, a->chunks, q_chunk, slot, out_chunk, a->Nc, a->scale_chunk, ctx->side);
         if (s == PHOTON_OK && apart && !direct && !copy_out(hp, hp->out_split, hp->out_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
-        if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return PHOTON_ERR_CUDA;
+        // every way out from here on joins the side stream again, failed calls included
+        if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) s = PHOTON_ERR_CUDA;
         if (s != PHOTON_OK) { cudaStreamWaitEvent(st, ctx->ev_join, 0); return s; }
     }
     // The append is one row per unit, in place: for a contiguous cache of a batch whose lengths fit the attention
