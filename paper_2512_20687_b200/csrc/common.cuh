@@ -66,7 +66,6 @@ struct AttnParams {
     const bf16 *ks, *vs;
     const int32_t *sh_len, *sh_id;
     int n_shared, cap_sh;
-    int max_sh;              // host-side bound on the prefixes' lengths (a hint: where a key range probably starts)
     const int32_t *slot;
     const int32_t *page_table;   // paged cache: [n_units, pages_per_unit] page ids, or NULL
     int page_rows, pages_per_unit, n_pages;

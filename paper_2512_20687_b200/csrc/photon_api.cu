@@ -91,7 +91,6 @@ photon_status attention_common(photon_ctx *ctx, const photon_kv *cache, const ph
             p.sh_len = cache->shared_len; p.sh_id = cache->shared_id;
             p.n_shared = cache->n_shared; p.cap_sh = cache->cap_shared;
             const int ms = cache->max_shared_len ? cache->max_shared_len : cache->cap_shared;
-            p.max_sh = ms;
             if (size_t(n_q) * c.Hq * (c.dh + 2) > ctx->partial_floats) return PHOTON_ERR_WORKSPACE;
             const int G = c.Hq / c.Hkv;
             const int groups = ceil_div(n_q, shared_prefix_units_per_cta(G));     // tiles of 128 query rows

@@ -69,13 +69,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, 
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 
-// Asks the L2 to fetch `bytes` (a multiple of 16) from the 16-byte aligned global address `src`.  Nothing
-// reaches the SM: the L2 is the point of coherence, so the request is harmless whatever is written there
-// later, and a load that follows finds the line there or on its way.
-__device__ __forceinline__ void l2_prefetch(const void *src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
-}
-
 // Untiled bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16 bytes.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile(

@@ -125,19 +125,6 @@ shared_prefix_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_
         else ptx::mbar_arrive(recv_bar);
         ptx::prefetch_tmap(&tm_ks); ptx::prefetch_tmap(&tm_vs);
     }
-    // A guess at the first key tile this CTA will want (prefix 0, cut as if it had the length the host
-    // names as its bound) goes to the L2 as a request, ahead of everything: nothing but the L2 keeps what
-    // it brings, so a wrong guess costs a little bandwidth and a right one most of the first tile's latency.
-    if (threadIdx.x == 32 && p.max_sh > 0) {
-        int g0, g1;
-        part_range(min(p.max_sh, p.cap_sh), p.splits_sh, part, g0, g1);
-        const int rows = min(BN, g1 - g0);
-        if (rows > 0) {
-            const size_t at = ((size_t)h * p.cap_sh + g0) * DH;
-            ptx::l2_prefetch(p.ks + at, rows * DH * 2);
-            ptx::l2_prefetch(p.vs + at, rows * DH * 2);
-        }
-    }
     ptx::grid_dep_wait();                      // queries may come from the kernel before this one
     ptx::grid_dep_launch();                    // one wave: the kernel for the units' own keys may line up
     // The Q tile goes to shared memory K-major with the 128-byte swizzle TMA would use.  Every warp but the two
