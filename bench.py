@@ -763,7 +763,8 @@ def run_gpu(args, cfg) -> None:
             pass
         return None, note
 
-    traffic, traffic_note = recorded_traffic(dom)
+    # (with a shared prefix the coarse attention is the shared-prefix kernel, recorded under that name)
+    traffic, traffic_note = recorded_traffic("shared_prefix" if cfg.shared_S and dom == "coarse_attn" else dom)
     if "chunk_causal_attn" in widened:
         widened["chunk_causal_attn"]["traffic"], widened["chunk_causal_attn"]["traffic_note"] = recorded_traffic(
             "chunk_causal_attn")
