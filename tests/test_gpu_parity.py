@@ -180,6 +180,57 @@ def test_shared_prefix_variants(oracle, G, dh, B, max_splits, S):
     assert np.abs(lse[fin] - want_lse[fin]).max() < 2e-3
 
 
+@pytest.mark.parametrize("folded", [False, True])
+def test_attention_that_lined_up_behind_an_append_which_opens_new_tiles(oracle, folded):
+    """The attention's CTAs start, and deal the tiles, while the kernels before it in the stream still run: a long
+    read (the probe) holds the stream, the append behind it has not run yet, so the lengths the deal is made from are
+    the old ones.  Units at 64 and 128 rows open a new tile with the append: after the dependency wait the deal is
+    found stale, the loads that went out early are left to land and everything is dealt again.  The result must be
+    what the oracle gives for the grown caches, and the same bits as a run with nothing in front of it.  folded: the
+    same start behind a long read for the step's attention with the append folded in (its lengths do not change
+    under it)."""
+    cfg = cfg_small(1, B=21, S=400)
+    s_in = wl.step_inputs(cfg, poison=True)
+    co, cv, chk = s_in["coarse"], s_in["converter"], s_in["chunks"]
+    lens = np.array([64, 128, 63, 0, 399, 192, 1, 127, 256, 320, 64, 64, 128, 5, 300, 191, 255, 64, 383, 128, 2], np.int32)
+    co["k"] = wl.normal_bf16(11, "k", co["k"].shape)
+    co["v"] = wl.normal_bf16(11, "v", co["v"].shape)
+    for u, n in enumerate(lens):
+        co["k"][u, :, n:] = 0x7FC1
+        co["v"][u, :, n:] = 0xFFC1
+    co["len"] = lens
+    scale = cfg.dh ** -0.5
+    held = torch.empty(192 << 20, dtype=torch.uint8, device="cuda").random_()       # about 30 us of reading
+    outs = []
+    with Ctx(cfg) as c:
+        for hold in (True, False):
+            d, dc = coarse_to_dev(co), chunks_to_dev(chk)
+            out = torch.empty_like(d["q"])
+            lse = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device="cuda")
+            torch.cuda.synchronize()
+            if hold:
+                ph.photon_read_probe(c.h, held)
+            if folded:
+                U = torch.empty(cfg.B, cfg.P, cfg.D, dtype=torch.bfloat16, device="cuda")
+                oc = torch.empty_like(dc["q"])
+                args = ph.make_step_args(d["kv"], d["k_new"], d["v_new"], d["q"], out, scale, dev_bf16(cv["w_out_major"]),
+                                         ph.PHOTON_W_OUT_MAJOR, U, cfg.B, chunks=dc["kv"], q_chunk=dc["q"], out_chunk=oc,
+                                         Nc=cfg.Nc, scale_chunk=scale, lse_coarse=lse)
+                ph.photon_decode_step(c.h, args)
+            else:
+                ph.photon_kv_append(c.h, d["kv"], d["k_new"], d["v_new"])
+                ph.photon_coarse_attn(c.h, d["kv"], d["q"], out, lse, scale)
+            assert c.status() == 0
+            outs.append((host_bits(out), lse.cpu().numpy(), host_bits(d["k"]), d["len"].cpu().numpy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    assert oracle.kv_append(co["k"], co["v"], co["len"], co["k_new"], co["v_new"]) == 0
+    assert np.array_equal(outs[0][2], co["k"]) and np.array_equal(outs[0][3], co["len"])
+    want, want_lse = oracle.attention(co["q"], co["k"], co["v"], co["len"], scale, n_threads=NT)
+    assert_close(wl.bf16_bits_to_f64(outs[0][0]), want, "attention behind an append")
+    fin = np.isfinite(want_lse)
+    assert np.abs(outs[0][1][fin] - want_lse[fin]).max() < 2e-3
+
+
 @pytest.mark.parametrize("max_splits", [1, 0])
 def test_shared_prefix_with_logits_that_grow_along_the_prefix(oracle, max_splits):
     """Keys of later tiles score far higher than earlier ones for some query heads, so the reference
