@@ -103,11 +103,20 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     const uint32_t tmem = *tmem_slot;
     ptx::grid_dep_launch();                 // at most one CTA per SM and one wave
 
+    // The weights never come from the kernel before this one, x may: the ring's first turn requests its
+    // weight atoms at once (the TMA warp) and its x atoms once the dependency wait has returned (the first
+    // epilogue warp, idle until the accumulator is complete: where the wait is over already, the two go out
+    // side by side), so that the weight stream already runs under the tail of the predecessor.  Everything
+    // else this kernel does with global memory follows from x having landed.
+    auto load_x = [&](int st, int s) {
+        const int atoms = min(KA, n_atoms - st * KA);
+        const uint32_t a_dst = base + s * stage_bytes;
+        for (int j = 0; j < atoms; ++j)
+            ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, (a_lo + st * KA + j) * BK, m0, bars + 16 * s);   // x[m0.., k0..]
+    };
+    const int ahead = min(n_steps, n_stages);              // the ring starts empty: no stage to wait for
+
     if (warp == 0) {
-        // The weights never come from the kernel before this one, x may: the ring's first turn requests
-        // its weight atoms at once, and its x atoms once the dependency wait has returned, so that the
-        // weight stream already runs under the tail of the predecessor.  Everything else this kernel does
-        // with global memory follows from x having landed.
         auto load_w = [&](int st, int s) {
             const int atoms = min(KA, n_atoms - st * KA);
             const uint32_t full = bars + 16 * s;
@@ -123,13 +132,6 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
                 }
             }
         };
-        auto load_x = [&](int st, int s) {
-            const int atoms = min(KA, n_atoms - st * KA);
-            const uint32_t a_dst = base + s * stage_bytes;
-            for (int j = 0; j < atoms; ++j)
-                ptx::tma_load_2d(a_dst + j * a_bytes, &tm_x, (a_lo + st * KA + j) * BK, m0, bars + 16 * s);   // x[m0.., k0..]
-        };
-        const int ahead = min(n_steps, n_stages);          // the ring starts empty: no stage to wait for
         if (ptx::elect_one())
             for (int st = 0; st < ahead; ++st) {
                 ptx::mbar_arrive_expect_tx(bars + 16 * st, min(KA, n_atoms - st * KA) * (a_bytes + T::B_BYTES));
@@ -137,9 +139,6 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             }
         __syncwarp();
         ptx::grid_dep_wait();               // x may be the output of the kernel before this one
-        if (ptx::elect_one())
-            for (int st = 0; st < ahead; ++st) load_x(st, st);
-        __syncwarp();
         int s = ahead == n_stages ? 0 : ahead;
         uint32_t phase = ahead == n_stages ? 1 : 0;
         for (int st = ahead; st < n_steps; ++st) {
@@ -202,6 +201,12 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     const bool epi = warp >= 2 && warp <= 5;
     const int quad = warp & 3;
     bool ok = true;
+    if (warp == 2) {
+        ptx::grid_dep_wait();               // x may be the output of the kernel before this one
+        if (ptx::elect_one())
+            for (int st = 0; st < ahead; ++st) load_x(st, st);
+        __syncwarp();
+    }
     if (epi) {
         ok = ptx::mbar_wait(bar_acc, 0);
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);

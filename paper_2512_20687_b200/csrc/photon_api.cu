@@ -650,9 +650,11 @@ photon_status photon_device_status(photon_ctx *ctx, int32_t *bits_out, int32_t c
         return PHOTON_ERR_CUDA;
     if (clear && cudaMemset(ctx->status, 0, sizeof(int32_t)) != cudaSuccess) return PHOTON_ERR_CUDA;
     // a kernel that gave up on a wait, or stopped at an index that was out of range, may have left arrival
-    // tickets behind; they must read zero again
+    // tickets or counters behind (the hand-out counters of the whole-chunk attention, the readers' counter of
+    // a folded-in append); they must read zero again
     if (clear && (*bits_out & (PHOTON_DEV_TIMEOUT | PHOTON_DEV_BAD_INDEX)) &&
-        cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess)
+        (cudaMemset(ctx->tickets, 0, ctx->n_tickets * sizeof(int32_t)) != cudaSuccess ||
+         cudaMemset(ctx->work, 0, 32 * sizeof(int32_t)) != cudaSuccess))       // words 32..63 of the status block
         return PHOTON_ERR_CUDA;
     return PHOTON_OK;
 }
