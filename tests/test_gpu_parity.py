@@ -461,6 +461,42 @@ def test_chunk_attention_at_the_largest_window(oracle, dh, Hq, Hkv):
     assert_close(got, want, f"chunk cap 64 dh={dh} G={Hq // Hkv}")
 
 
+@pytest.mark.parametrize("dh,Hq,Hkv,P,C", [(128, 8, 8, 8, 16), (128, 8, 2, 8, 24), (64, 6, 2, 8, 16), (64, 3, 3, 4, 4)])
+def test_chunk_attention_through_the_ring_of_bulk_copies(oracle, dh, Hq, Hkv, P, C):
+    """Enough (chunk, KV head) pairs for the persistent kernel whose warps keep their next items on their way
+    into shared memory: every length from 0 to the capacity (empty items take no slot turn), a number of items
+    that is no multiple of the grid, a gather through a permutation with two bad entries, poisoned rows past
+    the end, group sizes 1, 3 and 4.  Every output is compared."""
+    n_chunks = (8 * 148 * 8 + Hkv - 1) // Hkv + 37
+    cfg = cfg_small(4, B=n_chunks, chunks_per_seq=1, P=P, C=C, Hq=Hq, Hkv=Hkv, dh=dh, D=Hq * dh)
+    assert cfg.Nc == n_chunks
+    ch = wl.chunk_inputs(cfg, poison=True)
+    cap = P + C
+    lens = ((np.arange(cfg.Nc) * 7) % (cap + 1)).astype(np.int32)
+    bad = np.arange(cap)[None, :] >= lens[:, None]
+    fresh_k = wl.normal_bf16(21, "k", ch["kc"].shape)
+    fresh_v = wl.normal_bf16(22, "v", ch["vc"].shape)
+    gone = np.broadcast_to(bad[:, None, :, None], ch["kc"].shape)
+    ch["kc"] = np.where(gone, np.uint16(0x7FC1), fresh_k)
+    ch["vc"] = np.where(gone, np.uint16(0xFFC1), fresh_v)
+    ch["len"] = lens
+    scale = cfg.dh ** -0.5
+    slot = np.random.default_rng(dh + Hq).permutation(cfg.Nc).astype(np.int32)
+    slot[5] = -1
+    slot[cfg.Nc - 2] = cfg.Nc
+    want, _, flags = oracle.attention(ch["q"], ch["kc"], ch["vc"], lens, scale, slot=slot, n_threads=NT, want_flags=True)
+    with Ctx(cfg) as c:
+        d = chunks_to_dev(ch)
+        out = torch.full_like(d["q"], 5.0)
+        ph.photon_chunk_attn(c.h, d["kv"], d["q"], dev_i32(slot), out, scale=scale)
+        assert c.status() == flags == ph.PHOTON_DEV_BAD_INDEX
+    got = host_f64(out)
+    assert np.all(got[5] == 0) and np.all(got[cfg.Nc - 2] == 0)
+    empty = lens[np.clip(slot, 0, cfg.Nc - 1)] == 0
+    assert np.all(got[empty] == 0)
+    assert_close(got, want, f"chunk ring dh={dh} G={Hq // Hkv} cap={cap}")
+
+
 @pytest.mark.parametrize("idx,lengths,B", [(1, (2, 2), 16), (1, (4, 4, 4), 64), (3, (2, 2), 64), (4, (2, 2), 8)])
 def test_decode_step_under_other_hierarchies(oracle, idx, lengths, B):
     """The whole step on the shapes another hierarchy gives the same model: (2, 2) makes
