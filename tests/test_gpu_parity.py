@@ -697,7 +697,7 @@ def test_decode_step_chain_at_full_size(oracle, idx):
 
 
 # chunk attention beside the coarse part with little / with more than 1 MiB to move, and in line after it
-@pytest.mark.parametrize("idx,B,S", [(1, 24, 300), (1, 130, 200), (4, 12, 128)])
+@pytest.mark.parametrize("idx,B,S", [(1, 24, 300), (1, 130, 200), (4, 12, 128), (4, 40, 64)])
 @pytest.mark.parametrize("pinned,split", [(True, True), (True, False), (False, True), (False, False)])
 def test_decode_step_from_host_buffers(oracle, pinned, split, idx, B, S):
     """The step whose inputs (new K/V rows, both query tensors, the lengths) start in host memory and
