@@ -476,7 +476,8 @@ def run_gpu(args, cfg) -> None:
                 t_roof = max(nbytes / (hbm_peak * 1e3), flops / (tensor_peak * 1e6))
                 res.update({"prefix_flops": flops, "TFLOPs": flops / us * 1e-6, "frac_of_own_roofline": t_roof / us,
                             "logical_GBps": logical / us * 1e-3,
-                            "note": "two launches (prefix contraction on the tensor cores, then the own keys); the prefix "
+                            "note": "one launch: the prefix contraction on the tensor cores with the branches' short own caches "
+                                    "riding along as extra key tiles (two launches once an own cache exceeds 32 rows); the prefix "
                                     "is read once, so the HBM fraction of the physical bytes says little: the own roofline "
                                     "is the slower of bytes / HBM peak and prefix flops / bf16 peak; logical = bytes a "
                                     "cache with the prefix copied into every branch would read"})

@@ -9,7 +9,7 @@
 // in fp32, and the G query heads of the group reuse the rows.  One launch, no
 // workspace: the result is rounded once to bf16 and stored.
 //
-// Two kernels share that arithmetic and differ in how the rows arrive:
+// Two kernels do that arithmetic and differ in how the rows arrive:
 //  - chunk_attn_kernel: 128-bit loads into registers, all issued before the
 //    first use (up to 2 * RP rows in flight per warp), one item per warp, many
 //    small CTAs.  For small calls, and for buffers too large for the ring.
@@ -41,11 +41,11 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&t);
 }
 
-// DH: head size; RP: rows fetched per pass (a pass covers rows [pass*RP, pass*RP + RP));
+// The ring kernel's arithmetic.  DH: head size; RP: rows per pass (a pass covers rows [pass*RP, pass*RP + RP));
 // GT: query heads evaluated together against the rows in registers.
 //
-// One item (query i, KV head kvh; numbered i * Hkv + kvh) against the first len rows of its buffer.  ldk(off) and ldv(off) give this lane
-// the 16-byte vector that lies `off` vectors past its own place in the first rows (row lane / VEC, vector lane % VEC);
+// One item (query i, KV head kvh; numbered i * Hkv + kvh) against the first len rows of its buffer.  ldk(off) and
+// ldv(off) give this lane the 16-byte vector that lies `off` vectors past its own place in the first rows (row lane / VEC, vector lane % VEC);
 // ldq(off) likewise in the G query rows of the pair, from vector lane % VEC of the first.  `ok` says whether the row
 // exists: a missing V row must come back as zeros (its weight is zero, but zero times whatever lies there need not
 // be); a missing K row may come back as anything that can be read, its logit is replaced.
@@ -104,7 +104,9 @@ __device__ __forceinline__ void attend(const AttnParams &p, long long item, int 
                     s[g][t] = a;
                 }
             }
-            // (step by step over all logits: shuffles keep their order, so a logit at a time would be one long chain)
+            // Step by step over all logits: shuffles keep their order, a logit at a time would be one long chain, and
+            // with few warps per SM nothing else fills the gaps.  (The register kernel, 16 warps per SM, is faster
+            // with a logit at a time and fewer values live: measured both ways in both kernels.)
 #pragma unroll
             for (int o = 1; o < VEC; o <<= 1)
 #pragma unroll
@@ -178,26 +180,144 @@ __device__ __forceinline__ void bad_index(const AttnParams &p, long long item, i
                 make_uint4(0u, 0u, 0u, 0u);
 }
 
+// The register kernel: one item per warp, rows loaded straight into registers.  It has the arithmetic of `attend`
+// written out once more (a logit at a time in the reduction, predicated loads, four heads at a time): sharing the
+// function cost this kernel 15-20 % on small calls.
+// DH: head size; RP: rows fetched per pass (a pass covers rows [pass*RP, pass*RP + RP));
+// GT: query heads evaluated together against the rows in registers.
 template <int DH, int RP, int GT>
 __global__ void __launch_bounds__(CH_WARPS * 32)
 chunk_attn_kernel(const AttnParams p) {
+    constexpr int VEC = DH / 8;             // 16-byte vectors (= lanes) per row
+    constexpr int RPL = 32 / VEC;           // rows covered by one warp-wide load
+    constexpr int NI = RP / RPL;            // loads per lane per pass
+    static_assert(RP % RPL == 0, "pass height must be a whole number of warp loads");
+
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * CH_WARPS + (threadIdx.x >> 5);
     if (item >= (long long)p.n_q * p.Hkv) return;
     const int kvh = (int)(item % p.Hkv);
     const int i = (int)(item / p.Hkv);
+    const int G = p.Hq / p.Hkv;
+    const int col = lane % VEC, rsub = lane / VEC;
+
     const int u = p.slot ? __ldcg(p.slot + i) : i;               // index arrays through the L2: another kernel may have just written them
+    bf16 *out_base = p.out + ((size_t)i * p.Hq + (size_t)kvh * G) * DH + col * 8;
     if (u < 0 || u >= p.n_units) {
-        bad_index<DH>(p, item, lane);
+        if (lane == 0) atomicOr(p.status, PHOTON_DEV_BAD_INDEX);
+        if (rsub == 0)
+            for (int g = 0; g < G; ++g)
+                *reinterpret_cast<uint4 *>(out_base + (size_t)g * DH) = make_uint4(0u, 0u, 0u, 0u);
         return;
     }
     const int len = max(0, min(__ldcg(p.len + u), p.cap));
     const size_t base = ((size_t)u * p.Hkv + kvh) * p.cap * DH;
-    const uint4 *kp = reinterpret_cast<const uint4 *>(p.k + base) + lane;
+    const uint4 *kp = reinterpret_cast<const uint4 *>(p.k + base) + lane;     // row rsub, vector col
     const uint4 *vp = reinterpret_cast<const uint4 *>(p.v + base) + lane;
-    const uint4 *qp = reinterpret_cast<const uint4 *>(p.q + (size_t)item * (p.Hq / p.Hkv) * DH) + lane % (DH / 8);
-    attend<DH, RP, GT>(p, item, len, lane, [=](int off) { return qp[off]; }, [=](int off, bool ok) { return ok ? __ldg(kp + off) : make_uint4(0u, 0u, 0u, 0u); },
-                       [=](int off, bool ok) { return ok ? __ldg(vp + off) : make_uint4(0u, 0u, 0u, 0u); });
+    const int n_pass = (len + RP - 1) / RP;
+
+    for (int g0 = 0; g0 < G; g0 += GT) {
+        float qf[GT][8];
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            const uint4 qv = *reinterpret_cast<const uint4 *>(
+                p.q + ((size_t)i * p.Hq + (size_t)kvh * G + g0 + g) * DH + col * 8);
+            unpack8(qv, qf[g]);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) qf[g][e] *= p.scale_log2;
+        }
+        float m[GT], l[GT], acc[GT][8];
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            m[g] = -CUDART_INF_F; l[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
+        }
+
+        for (int pass = 0; pass < n_pass; ++pass) {
+            const int r0 = pass * RP + rsub;
+            uint4 kr[NI], vr[NI];
+#pragma unroll
+            for (int t = 0; t < NI; ++t) {
+                const bool ok = r0 + t * RPL < len;
+                kr[t] = ok ? __ldg(kp + (size_t)(pass * RP + t * RPL) * VEC) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int t = 0; t < NI; ++t) {
+                const bool ok = r0 + t * RPL < len;
+                vr[t] = ok ? __ldg(vp + (size_t)(pass * RP + t * RPL) * VEC) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            // logits of this lane's rows for each head of the group
+            float s[GT][NI];
+#pragma unroll
+            for (int t = 0; t < NI; ++t) {
+                float kf[8];
+                unpack8(kr[t], kf);
+#pragma unroll
+                for (int g = 0; g < GT; ++g) {
+                    float a = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) a = fmaf(qf[g][e], kf[e], a);
+                    s[g][t] = a;
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < GT; ++g)
+#pragma unroll
+                for (int t = 0; t < NI; ++t) {
+#pragma unroll
+                    for (int o = 1; o < VEC; o <<= 1) s[g][t] += __shfl_xor_sync(0xffffffffu, s[g][t], o);
+                    if (r0 + t * RPL >= len) s[g][t] = -CUDART_INF_F;
+                }
+            // online softmax; the running maximum is uniform across the warp
+            float w[GT][NI];
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                float mx = s[g][0];
+#pragma unroll
+                for (int t = 1; t < NI; ++t) mx = fmaxf(mx, s[g][t]);
+#pragma unroll
+                for (int o = VEC; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                const float mn = fmaxf(m[g], mx);                 // finite: a pass holds >= 1 valid row
+                const float corr = exp2f(m[g] - mn);              // first pass: exp2(-inf) = 0
+                float ls = 0.f;
+#pragma unroll
+                for (int t = 0; t < NI; ++t) { w[g][t] = exp2f(s[g][t] - mn); ls += w[g][t]; }
+                l[g] = l[g] * corr + ls;
+                m[g] = mn;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] *= corr;
+            }
+#pragma unroll
+            for (int t = 0; t < NI; ++t) {
+                float vf[8];
+                unpack8(vr[t], vf);
+#pragma unroll
+                for (int g = 0; g < GT; ++g)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(w[g][t], vf[e], acc[g][e]);
+            }
+        }
+        // fold the row groups together, normalise, store
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+#pragma unroll
+            for (int o = VEC; o < 32; o <<= 1) {
+                l[g] += __shfl_xor_sync(0xffffffffu, l[g], o);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], o);
+            }
+            if (rsub == 0) {
+                const float inv = l[g] > 0.f ? 1.f / l[g] : 0.f;   // no valid key: zero row
+                uint4 o4;
+                o4.x = pack2(acc[g][0] * inv, acc[g][1] * inv);
+                o4.y = pack2(acc[g][2] * inv, acc[g][3] * inv);
+                o4.z = pack2(acc[g][4] * inv, acc[g][5] * inv);
+                o4.w = pack2(acc[g][6] * inv, acc[g][7] * inv);
+                *reinterpret_cast<uint4 *>(out_base + (size_t)(g0 + g) * DH) = o4;
+            }
+        }
+    }
 }
 
 constexpr int RING_DEPTH = 2;               // items a consumer warp holds in shared memory: one in use, the next on its way
