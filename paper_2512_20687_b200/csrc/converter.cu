@@ -38,10 +38,7 @@ constexpr int CONV_THREADS = 224;       // warp 0: TMA, warps 1 and 6: MMA (1 ow
 template <int NT> __host__ __device__ constexpr int mma_warps() { return NT <= 64 ? 2 : 1; }
 
 constexpr int MAX_STAGES = 12;
-constexpr int RING_BYTES = 192 * 1024;  // one CTA per SM
-// With more output tiles than SMs but no more than two per SM, two CTAs share an SM, each with a smaller
-// ring of single-atom stages, so that the tiles still run as one wave.
-constexpr int RING_BYTES_PAIR = 88 * 1024;
+constexpr int RING_BYTES = 192 * 1024;  // one CTA per SM; more output tiles than SMs run as further waves
 
 template <int NT>
 struct ConvTile {
@@ -57,13 +54,13 @@ __host__ __device__ inline int conv_stages(int ring_bytes, int a_bytes, int b_by
 
 // The loops of the TMA warp and of the MMA warp are run by the whole warp (so that their
 // address arithmetic stays warp-uniform); one elected lane issues the asynchronous operations.
-template <int NT, bool W_IN_MAJOR, bool PAIR, bool SPLIT>
+template <int NT, bool W_IN_MAJOR, bool SPLIT>
 __global__ void __launch_bounds__(CONV_THREADS, 1)
 converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
                       const __grid_constant__ CUtensorMap tm_w) {
     using T = ConvTile<NT>;
-    constexpr int KA = PAIR ? 1 : atoms_per_stage<NT>();
-    constexpr int RING = PAIR ? RING_BYTES_PAIR : RING_BYTES;
+    constexpr int KA = atoms_per_stage<NT>();
+    constexpr int RING = RING_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - ptx::smem_u32(smem_raw));
@@ -101,13 +98,14 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    ptx::grid_dep_launch();                 // at most one CTA per SM and one wave
+    ptx::grid_dep_launch();                 // one CTA per SM; the next kernel lines up once the last wave has started
 
     // The weights never come from the kernel before this one, x may: the ring's first turn requests its
-    // weight atoms at once (the TMA warp) and its x atoms once the dependency wait has returned (the first
-    // epilogue warp, idle until the accumulator is complete: where the wait is over already, the two go out
-    // side by side), so that the weight stream already runs under the tail of the predecessor.  Everything
-    // else this kernel does with global memory follows from x having landed.
+    // weight atoms at once and its x atoms once the dependency wait has returned, so that the weight stream
+    // already runs under the tail of the predecessor.  The same thread issues both, after it has told the
+    // stage's barrier how many bytes to expect: were another warp to issue the x atoms, then with no
+    // predecessor in flight (calls launched one by one) an x atom could land before its stage's byte count is
+    // posted.  Everything else this kernel does with global memory follows from x having landed.
     auto load_x = [&](int st, int s) {
         const int atoms = min(KA, n_atoms - st * KA);
         const uint32_t a_dst = base + s * stage_bytes;
@@ -139,6 +137,9 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             }
         __syncwarp();
         ptx::grid_dep_wait();               // x may be the output of the kernel before this one
+        if (ptx::elect_one())
+            for (int st = 0; st < ahead; ++st) load_x(st, st);
+        __syncwarp();
         int s = ahead == n_stages ? 0 : ahead;
         uint32_t phase = ahead == n_stages ? 1 : 0;
         for (int st = ahead; st < n_steps; ++st) {
@@ -201,12 +202,6 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     const bool epi = warp >= 2 && warp <= 5;
     const int quad = warp & 3;
     bool ok = true;
-    if (warp == 2) {
-        ptx::grid_dep_wait();               // x may be the output of the kernel before this one
-        if (ptx::elect_one())
-            for (int st = 0; st < ahead; ++st) load_x(st, st);
-        __syncwarp();
-    }
     if (epi) {
         ok = ptx::mbar_wait(bar_acc, 0);
         if (!ok && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
@@ -287,14 +282,14 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     }
 }
 
-template <int NT, bool IN_MAJOR, bool PAIR, bool SPLIT>
+template <int NT, bool IN_MAJOR, bool SPLIT>
 cudaError_t run_as(photon_ctx *ctx, const ConvParams &p, const CUtensorMap &mx, const CUtensorMap &mw, dim3 grid,
                    cudaStream_t st) {
     using T = ConvTile<NT>;
-    constexpr size_t smem = (size_t)(PAIR ? RING_BYTES_PAIR : RING_BYTES) + T::extra;
+    constexpr size_t smem = (size_t)RING_BYTES + T::extra;
     static size_t smem_set[kMaxDevices] = {};
-    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR, PAIR, SPLIT>, smem, ctx->device, smem_set)) return e;
-    return launch_dependent(converter_umma_kernel<NT, IN_MAJOR, PAIR, SPLIT>, grid, dim3(CONV_THREADS), smem, st,
+    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR, SPLIT>, smem, ctx->device, smem_set)) return e;
+    return launch_dependent(converter_umma_kernel<NT, IN_MAJOR, SPLIT>, grid, dim3(CONV_THREADS), smem, st,
                             p.ksplit > 1 ? p.ksplit : 0, p, mx, mw);
 }
 
@@ -311,16 +306,11 @@ cudaError_t run(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launc
     mw = *t;
     if (p.ksplit < 1) p.ksplit = 1;
     dim3 grid(p.ksplit * (p.N / NT), (p.B + BM - 1) / BM);
-    const long long ctas = (long long)grid.x * grid.y;
     cudaError_t e;
-    if constexpr (NT == 64) {
-        const bool pair = p.ksplit == 1 && ctas > ctx->sm_count && ctas <= 2ll * ctx->sm_count;
-        e = pair ? run_as<NT, IN_MAJOR, true, false>(ctx, p, mx, mw, grid, st)
-                 : p.ksplit > 1 ? run_as<NT, IN_MAJOR, false, true>(ctx, p, mx, mw, grid, st)
-                                : run_as<NT, IN_MAJOR, false, false>(ctx, p, mx, mw, grid, st);
-    } else {
-        e = run_as<NT, IN_MAJOR, false, false>(ctx, p, mx, mw, grid, st);
-    }
+    if constexpr (NT == 64)
+        e = p.ksplit > 1 ? run_as<NT, IN_MAJOR, true>(ctx, p, mx, mw, grid, st) : run_as<NT, IN_MAJOR, false>(ctx, p, mx, mw, grid, st);
+    else
+        e = run_as<NT, IN_MAJOR, false>(ctx, p, mx, mw, grid, st);
     ++*launches;
     return e != cudaSuccess ? e : cudaGetLastError();
 }

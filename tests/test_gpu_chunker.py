@@ -42,7 +42,7 @@ def test_rmsnorm_matches_oracle(oracle, rows, cols, with_gamma):
 
 # (B, K, N): the 1B-class chunker (4 CTAs share a tile), the chunk-parallel one (wide batch),
 # a tile count that needs no split, odd batch sizes, the smallest K that is still split, K too short to split
-# and more tiles than SMs (two CTAs per SM with smaller rings)
+# and more tiles than SMs (a second wave of CTAs)
 SHAPES = [(64, 8192, 2048), (512, 4096, 1024), (64, 2048, 8192), (1, 1024, 64), (130, 1024, 128),
           (17, 512, 64), (200, 4096, 256), (64, 1024, 11264), (130, 512, 6400),
           # thousands of rows: the persistent kernel (one to several tiles per CTA, a ragged last row tile)
@@ -66,6 +66,28 @@ def test_linear_matches_oracle(oracle, B, K, N, out_major):
         assert c.status() == 0
     assert np.array_equal(host_bits(y), host_bits(y2))                  # the split of K adds in a fixed order
     assert_close(host_f64(y), want, f"linear {B}x{K}x{N}")
+
+
+def test_linear_with_more_tiles_than_sms_repeated_on_an_idle_device():
+    """128 rows and 176 output tiles (the gate/up projection of a layer step on 128 chunks): 200 calls, each on
+    an idle device with another kernel run in between, as a caller that launches one operation at a time does.
+    Every call gives the first call's bits and leaves the status word clear.  (A form of this kernel that put
+    two CTAs on an SM for such tile counts gave up on a wait, or failed, once in some tens of such calls.)"""
+    B, K, N = 128, 2048, 11264
+    x = dev_bf16(wl.normal_bf16(25, "x", (B, K)))
+    w = dev_bf16(wl.normal_bf16(25, "w", (K, N), std=K ** -0.5))
+    with Ctx(cfg_small(0)) as c:
+        y0 = torch.empty((B, N), dtype=torch.bfloat16, device="cuda")
+        ph.photon_linear(c.h, x, w, ph.PHOTON_W_IN_MAJOR, None, y0)
+        torch.cuda.synchronize()
+        y, n = torch.empty_like(y0), torch.empty_like(x)
+        for _ in range(200):
+            ph.photon_rmsnorm(c.h, x, None, 1e-5, n)
+            torch.cuda.synchronize()
+            ph.photon_linear(c.h, x, w, ph.PHOTON_W_IN_MAJOR, None, y)
+            torch.cuda.synchronize()
+            assert c.status() == 0
+            assert torch.equal(y.view(torch.int16), y0.view(torch.int16))
 
 
 def test_large_tile_kernel_adds_bias_and_residual_and_is_deterministic(oracle):
