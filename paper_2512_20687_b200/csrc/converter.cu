@@ -324,16 +324,19 @@ cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long l
     const int m_tiles = (p.B + BM - 1) / BM;
     const bool wide = p.B > 128 && p.N % 128 == 0 && (p.N / 128) * m_tiles * 2 >= ctx->sm_count;
     const bool wider = wide && p.N % 256 == 0 && (p.N / 256) * m_tiles >= 100;
-    const int nt = wider ? 256 : wide ? 128 : 64;
+    // narrow slabs that would need a second wave of CTAs: twice as wide, one wave
+    const bool second_wave = !wide && p.N % 128 == 0 && (long long)(p.N / 64) * m_tiles > ctx->sm_count &&
+                             (long long)(p.N / 128) * m_tiles <= ctx->sm_count;
+    const int nt = wider ? 256 : (wide || second_wave) ? 128 : 64;
     p.ksplit = 1;
     if (nt == 64)
         while (p.ksplit < 4 && (p.N / nt) * m_tiles * p.ksplit * 2 <= ctx->sm_count && (p.D / BK) / (p.ksplit * 2) >= 8)
             p.ksplit *= 2;
     if (p.w_out_major)
-        return wider ? run<256, false>(ctx, p, st, launches)
-                     : wide ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
-    return wider ? run<256, true>(ctx, p, st, launches)
-                 : wide ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
+        return nt == 256 ? run<256, false>(ctx, p, st, launches)
+                         : nt == 128 ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
+    return nt == 256 ? run<256, true>(ctx, p, st, launches)
+                     : nt == 128 ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
 }
 
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {

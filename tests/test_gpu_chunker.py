@@ -42,7 +42,7 @@ def test_rmsnorm_matches_oracle(oracle, rows, cols, with_gamma):
 
 # (B, K, N): the 1B-class chunker (4 CTAs share a tile), the chunk-parallel one (wide batch),
 # a tile count that needs no split, odd batch sizes, the smallest K that is still split, K too short to split
-# and more tiles than SMs (a second wave of CTAs)
+# and more narrow tiles than SMs (wider slabs, one wave)
 SHAPES = [(64, 8192, 2048), (512, 4096, 1024), (64, 2048, 8192), (1, 1024, 64), (130, 1024, 128),
           (17, 512, 64), (200, 4096, 256), (64, 1024, 11264), (130, 512, 6400),
           # thousands of rows: the persistent kernel (one to several tiles per CTA, a ragged last row tile)
@@ -69,7 +69,7 @@ def test_linear_matches_oracle(oracle, B, K, N, out_major):
 
 
 def test_linear_with_more_tiles_than_sms_repeated_on_an_idle_device():
-    """128 rows and 176 output tiles (the gate/up projection of a layer step on 128 chunks): 200 calls, each on
+    """128 rows and 176 slabs of 64 output columns (the gate/up projection of a layer step on 128 chunks): 200 calls, each on
     an idle device with another kernel run in between, as a caller that launches one operation at a time does.
     Every call gives the first call's bits and leaves the status word clear.  (A form of this kernel that put
     two CTAs on an SM for such tile counts gave up on a wait, or failed, once in some tens of such calls.)"""
