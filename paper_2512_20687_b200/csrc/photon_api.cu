@@ -549,6 +549,18 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
             }
         }
     }
+    // A chunk attention that reads its queries (and slots) from the host buffer itself and whose lengths lie outside the
+    // staging area needs nothing of this call's copy: its stream forks before the copy is enqueued, not after it.
+    bool forked = false;
+    if (beside && direct) {
+        const char *cl = reinterpret_cast<const char *>(a->chunks->len);
+        const bool len_off = cl + (size_t)a->chunks->n_units * sizeof(int32_t) <= hp->dev_in || cl >= hp->dev_in + hp->in_bytes;
+        if (len_off) {
+            if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+                return PHOTON_ERR_CUDA;
+            forked = true;
+        }
+    }
     if (hp) {
         if (!copy_in(hp, 0, apart || direct ? hp->in_split : hp->in_bytes, st)) return PHOTON_ERR_CUDA;
         if (hp->in_bytes && ctx->host_pause_ns > 0) {
@@ -560,7 +572,7 @@ photon_status step_impl(photon_ctx *ctx, const photon_step_args *a, photon_strea
         }
     }
     if (beside) {
-        if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+        if (!forked && (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess))
             return PHOTON_ERR_CUDA;
         if (apart && !direct && !copy_in(hp, hp->in_split, hp->in_bytes, ctx->side)) s = PHOTON_ERR_CUDA;
         if (s == PHOTON_OK)
