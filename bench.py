@@ -643,7 +643,7 @@ def run_gpu(args, cfg) -> None:
         torch.cuda.empty_cache()
 
         # STEP of one LLaMA layer of the top-level encoder (normalise, q/k/v, rotary, append, attention, output
-        # projection, MLP) on the step's own caches: nine launches; weights rotate over the replicas
+        # projection, MLP) on the step's own caches: eight or nine launches; weights rotate over the replicas
         if cfg.Hq * cfg.dh == cfg.D:
             li = wl.encoder_layer_inputs(cfg)
             F = li["F"]

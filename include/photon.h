@@ -218,9 +218,12 @@ photon_status photon_linear(photon_ctx *ctx, const photon_bf16 *x, const photon_
  * weights in the order w_layout names: wqkv [D, (Hq + 2 Hkv) dh], wo [Hq dh,
  * D], wgu [D, 2F], wdown [F, D]; g1, g2 [D].  F a multiple of 64.  The
  * caller owns the intermediates in `scratch` (sizes beside the fields); each
- * is rounded to bf16 where the next kernel reads it.  y may alias x.  With
- * thousands of rows the gate/up projection and the activation are one launch
- * and scratch->gu is left unwritten (eight launches).
+ * is rounded to bf16 where the next kernel reads it.  y may alias x.  Where
+ * the gate/up projection's slabs of 64 features occupy at least half of the
+ * GPU's SMs (F / 64 slabs per 128 rows), and with thousands of rows, that
+ * projection and the activation are one launch and scratch->gu is left
+ * unwritten (eight launches); both projections are rounded to bf16 before
+ * the activation either way.
  *
  * photon_decoder_step: the same layer of a local decoder G^(l) (Eq. 6-7) for
  * the newest in-chunk position of every in-flight chunk: `chunks` holds the

@@ -186,6 +186,8 @@ cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long l
 bool linear_wants_large_tiles(const photon_ctx *ctx, const ConvParams &p);
 cudaError_t launch_linear_large(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches);
 cudaError_t launch_gate_up_large(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches);
+bool gate_up_fits_small_tiles(const photon_ctx *ctx, const ConvParams &p);
+cudaError_t launch_gate_up(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches);
 cudaError_t launch_rmsnorm(const bf16 *x, const bf16 *gamma, float eps, bf16 *out, int rows, int cols,
                            cudaStream_t st, long long *launches);
 cudaError_t launch_rope_split(const bf16 *qkv, const int32_t *pos, int period, int n, int Hq, int Hkv, int dh,

@@ -54,7 +54,11 @@ __host__ __device__ inline int conv_stages(int ring_bytes, int a_bytes, int b_by
 
 // The loops of the TMA warp and of the MMA warp are run by the whole warp (so that their
 // address arithmetic stays warp-uniform); one elected lane issues the asynchronous operations.
-template <int NT, bool W_IN_MAJOR, bool SPLIT>
+// GATED (slabs of 128 columns only): the gate/up projection of the MLP with its activation folded in.  W is
+// [gate | up] with N = 2F columns; a CTA takes 64 gate columns and the 64 up columns of the same features, and
+// writes silu(gate) * up for them into U [B, F] (both projections rounded to bf16 first, as when they are
+// stored and read back by the activation kernel).  No bias, no residual, no split of K.
+template <int NT, bool W_IN_MAJOR, bool SPLIT, bool GATED = false>
 __global__ void __launch_bounds__(CONV_THREADS, 1)
 converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm_x,
                       const __grid_constant__ CUtensorMap tm_w) {
@@ -76,7 +80,9 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ks = SPLIT ? p.ksplit : 1;                         // CTAs (one cluster) that share an output tile
     const int zr = ks > 1 ? (int)(blockIdx.x % ks) : 0;          // = rank in the cluster: which slice of K
-    const int n0 = (int)(blockIdx.x / ks) * NT, m0 = blockIdx.y * BM;
+    static_assert(!GATED || (NT == 128 && !SPLIT), "the gated form takes 64 gate and 64 up columns, whole K");
+    const int n0 = (int)(blockIdx.x / ks) * (GATED ? NT / 2 : NT), m0 = blockIdx.y * BM;
+    const int up0 = p.N / 2 + n0;                                // GATED: first of this CTA's up columns
     constexpr int MMA_WARPS = mma_warps<NT>();
     const uint32_t stg_bytes = (uint32_t)p.x_rows * NT * 4;      // the fetched rows of one fp32 tile, stored [column][row]
     const int a_lo = (p.D / BK) * zr / ks, n_atoms = (p.D / BK) * (zr + 1) / ks - a_lo;
@@ -122,11 +128,17 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             for (int j = 0; j < atoms; ++j) {
                 const int k0 = (a_lo + st * KA + j) * BK;
                 if (!W_IN_MAJOR) {
-                    ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);       // W[n0.., k0..]  (K-major)
+                    if (GATED) {                                                         // two boxes of 64 rows: gate, then up
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES + 64 * 128, &tm_w, k0, up0, full);
+                    } else {
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES, &tm_w, k0, n0, full);   // W[n0.., k0..]  (K-major)
+                    }
                 } else {
 #pragma unroll
                     for (int jj = 0; jj < NT / 64; ++jj)                                 // W[k0.., n0+64jj..] (N-major)
-                        ptx::tma_load_2d(b_dst + j * T::B_BYTES + jj * (BK * 128), &tm_w, n0 + 64 * jj, k0, full);
+                        ptx::tma_load_2d(b_dst + j * T::B_BYTES + jj * (BK * 128), &tm_w,
+                                         GATED ? (jj == 0 ? n0 : up0) : n0 + 64 * jj, k0, full);
                 }
             }
         };
@@ -216,6 +228,33 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
             if (!got && lane == 0) atomicOr(p.status, PHOTON_DEV_TIMEOUT);
             ok = ok && got;
         }
+        if constexpr (GATED) {
+            const int F = p.N / 2;
+#pragma unroll 1
+            for (int c0 = 0; c0 < NT / 2; c0 += 32) {
+                uint32_t g[32], u[32];
+                ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + c0, g);
+                ptx::tmem_ld_32x32(tmem + ((uint32_t)(quad * 32) << 16) + NT / 2 + c0, u);
+                ptx::tmem_ld_wait();
+                if (ok && b < p.B) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.U + (size_t)b * F + n0 + c0);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float g0 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(g[v * 8 + 2 * e])));
+                            const float g1 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(g[v * 8 + 2 * e + 1])));
+                            const float u0 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(u[v * 8 + 2 * e])));
+                            const float u1 = __bfloat162float(__float2bfloat16_rn(__uint_as_float(u[v * 8 + 2 * e + 1])));
+                            __nv_bfloat162 o = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+                            w[e] = *reinterpret_cast<uint32_t *>(&o);
+                        }
+                        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        } else {
 #pragma unroll 1
         for (int c0 = 0; c0 < NT; c0 += 32) {
             uint32_t r[32];
@@ -265,6 +304,7 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
                 }
             }
         }
+        }                                                  // (not GATED)
         if (zr != 0) {
             ptx::fence_proxy_async();                      // the staged tile is read by the bulk copy
             ptx::named_bar_sync(1, 128);                   // the four epilogue warps
@@ -282,15 +322,34 @@ converter_umma_kernel(const ConvParams p, const __grid_constant__ CUtensorMap tm
     }
 }
 
-template <int NT, bool IN_MAJOR, bool SPLIT>
+template <int NT, bool IN_MAJOR, bool SPLIT, bool GATED = false>
 cudaError_t run_as(photon_ctx *ctx, const ConvParams &p, const CUtensorMap &mx, const CUtensorMap &mw, dim3 grid,
                    cudaStream_t st) {
     using T = ConvTile<NT>;
     constexpr size_t smem = (size_t)RING_BYTES + T::extra;
     static size_t smem_set[kMaxDevices] = {};
-    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR, SPLIT>, smem, ctx->device, smem_set)) return e;
-    return launch_dependent(converter_umma_kernel<NT, IN_MAJOR, SPLIT>, grid, dim3(CONV_THREADS), smem, st,
+    if (const cudaError_t e = ensure_dynamic_smem(converter_umma_kernel<NT, IN_MAJOR, SPLIT, GATED>, smem, ctx->device, smem_set)) return e;
+    return launch_dependent(converter_umma_kernel<NT, IN_MAJOR, SPLIT, GATED>, grid, dim3(CONV_THREADS), smem, st,
                             p.ksplit > 1 ? p.ksplit : 0, p, mx, mw);
+}
+
+// out [B, F] = silu(x Wg) * (x Wu) for w = [Wg | Wu] (N = 2F columns), 64 features per CTA.
+template <bool IN_MAJOR>
+cudaError_t run_gated(photon_ctx *ctx, ConvParams p, cudaStream_t st, long long *launches) {
+    p.x_rows = p.B > 64 ? 128 : p.B > 32 ? 64 : p.B > 16 ? 32 : 16;
+    p.ksplit = 1;
+    const CUtensorMap *t;
+    CUtensorMap mx, mw;
+    if (!(t = ctx->tmaps.get(p.x, (uint64_t)p.B, (uint64_t)p.D, p.x_rows))) return cudaErrorInvalidValue;
+    mx = *t;
+    // [K, N] in boxes of 64 k x 64 n, or [N, K] in boxes of 64 n x 64 k (gate rows and up rows are fetched apart)
+    t = IN_MAJOR ? ctx->tmaps.get(p.w, (uint64_t)p.D, (uint64_t)p.N, BK) : ctx->tmaps.get(p.w, (uint64_t)p.N, (uint64_t)p.D, 64);
+    if (!t) return cudaErrorInvalidValue;
+    mw = *t;
+    const dim3 grid(p.N / 128, (p.B + BM - 1) / BM);
+    const cudaError_t e = run_as<128, IN_MAJOR, false, true>(ctx, p, mx, mw, grid, st);
+    ++*launches;
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int NT, bool IN_MAJOR>
@@ -337,6 +396,18 @@ cudaError_t launch_linear(photon_ctx *ctx, ConvParams p, cudaStream_t st, long l
                          : nt == 128 ? run<128, false>(ctx, p, st, launches) : run<64, false>(ctx, p, st, launches);
     return nt == 256 ? run<256, true>(ctx, p, st, launches)
                      : nt == 128 ? run<128, true>(ctx, p, st, launches) : run<64, true>(ctx, p, st, launches);
+}
+
+// Whether the fused gate/up form serves this shape: whole slabs of 64 features, and enough of them to occupy most
+// of the GPU without a split of K (below that the plain projection, which can split K, and the activation kernel).
+bool gate_up_fits_small_tiles(const photon_ctx *ctx, const ConvParams &p) {
+    const long long tiles = (long long)(p.N / 128) * ((p.B + BM - 1) / BM);
+    return p.N % 128 == 0 && p.D % BK == 0 && tiles * 2 >= ctx->sm_count;
+}
+
+cudaError_t launch_gate_up(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {
+    if (p.B == 0) return cudaSuccess;
+    return p.w_out_major ? run_gated<false>(ctx, p, st, launches) : run_gated<true>(ctx, p, st, launches);
 }
 
 cudaError_t launch_converter(photon_ctx *ctx, const ConvParams &p, cudaStream_t st, long long *launches) {

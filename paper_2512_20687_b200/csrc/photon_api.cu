@@ -341,8 +341,9 @@ photon_status photon_swiglu(photon_ctx *ctx, const photon_bf16 *gu, photon_bf16 
 }
 
 namespace {
-// gate/up projection and activation: act [rows, F] = silu(n Wg) * (n Wu).  With thousands of rows one fused
-// launch of the large-tile kernel (gu is then not written); else the projection followed by photon_swiglu.
+// gate/up projection and activation: act [rows, F] = silu(n Wg) * (n Wu).  One fused launch (gu is then not written)
+// of the large-tile kernel with thousands of rows, of the slab kernel where 64-feature slabs occupy most of the GPU;
+// else the projection followed by photon_swiglu.
 photon_status gate_up(photon_ctx *ctx, const photon_layer *L, const photon_layer_scratch *sc, int rows,
                       photon_stream stream) {
     const photon_config &c = ctx->cfg;
@@ -355,6 +356,10 @@ photon_status gate_up(photon_ctx *ctx, const photon_layer *L, const photon_layer
     p.status = ctx->status;
     if (L->F % 128 == 0 && linear_wants_large_tiles(ctx, p)) {
         const cudaError_t e = launch_gate_up_large(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
+        return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
+    }
+    if (gate_up_fits_small_tiles(ctx, p)) {                                // one launch, gu is not written
+        const cudaError_t e = launch_gate_up(ctx, p, static_cast<cudaStream_t>(stream), &ctx->launches);
         return e == cudaSuccess ? PHOTON_OK : PHOTON_ERR_CUDA;
     }
     photon_status s = photon_linear(ctx, sc->n, L->wgu, L->w_layout, nullptr, nullptr, sc->gu, rows, c.D, 2 * L->F, stream);
